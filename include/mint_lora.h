@@ -1,0 +1,230 @@
+/*
+ * mint_lora.h -- C ABI of the mixed-adapter LoRA apply for NVIDIA B200 (sm_100a).
+ *
+ * One resident base model serves a batch in which every request names its own
+ * LoRA adapter revision (paper, section "Shared-Base Rollout and Serving").
+ * For every token t with adapter a(t), resident in GPU slot sigma:
+ *
+ *        y[t, :] += s_sigma * (x[t, :] . A_sigma) . B_sigma
+ *
+ * A_sigma is d x r_sigma, B_sigma is r_sigma x n, s_sigma a per-adapter scalar.
+ * The paper delegates the apply to its serving engine and prints no equation;
+ * this is the standard LoRA update it relies on (section "Related Work").
+ *
+ * General rules for every call
+ *  - Returns an int32_t status: MINT_OK or a negative MINT_ERR_* code.  Nothing
+ *    is thrown across the boundary; mint_last_error_string() gives the detail
+ *    for the calling thread.
+ *  - Pointers named *_dev are DEVICE pointers, everything else is HOST memory.
+ *  - All device buffers (activations, pools, tables, plans, workspaces, status
+ *    words) are allocated and owned by the caller.  The library allocates no
+ *    device memory.  Handles (mint_pool, mint_slot_table) are small host
+ *    objects freed by their *_destroy call.
+ *  - GPU work is enqueued on the caller's stream (a cudaStream_t passed as
+ *    void*) and the call returns without synchronising, except
+ *    mint_plan_fetch_summary, which waits for the stream.
+ *  - bf16 tensors: device pointers 16-byte aligned, d and n multiples of 8,
+ *    row strides (ldx, ldy, in elements) multiples of 8; otherwise
+ *    MINT_ERR_MISALIGNED / MINT_ERR_SHAPE_MISMATCH and nothing is launched.
+ *  - Problems only the device can see (an id that is not resident, an index out
+ *    of range, a stale plan, a bounded wait that ran out) are recorded in the
+ *    caller's status_dev words and the offending work is skipped; kernels never
+ *    trap.  status_dev is MINT_STATUS_WORDS int32 that the caller zeroes:
+ *      [0] first error code seen (sticky), [1] number of tokens whose id was
+ *      not resident, [2] detail of the first error (token or item index),
+ *      [3] reserved.
+ */
+#ifndef MINT_LORA_H
+#define MINT_LORA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *mint_stream_t; /* a cudaStream_t */
+
+enum {
+  MINT_OK = 0,
+  MINT_ERR_INVALID_ARG = -1,
+  MINT_ERR_NOT_RESIDENT = -2,        /* a token names an id bound to no slot          */
+  MINT_ERR_SHAPE_MISMATCH = -3,      /* pool / table / plan shapes do not agree       */
+  MINT_ERR_RANK_TOO_LARGE = -4,      /* rank exceeds the pool's configured r_max      */
+  MINT_ERR_WORKSPACE_TOO_SMALL = -5,
+  MINT_ERR_MISALIGNED = -6,
+  MINT_ERR_CUDA = -7,                /* a CUDA runtime call failed                    */
+  MINT_ERR_TIMEOUT = -8,             /* a bounded device-side wait ran out            */
+  MINT_ERR_UNSUPPORTED = -9,
+  MINT_ERR_STALE_PLAN = -10,         /* the slot table changed after the plan was made */
+  MINT_ERR_BAD_INDEX = -11           /* expert id or row index out of range           */
+};
+
+#define MINT_STATUS_WORDS 4
+
+/* Pool weight layouts.  Slots are allocated at the configured maximum rank
+ * r_max and smaller adapters are padded (paper, "Time-Sliced Multi-LoRA
+ * Training": slots at configured maximum shapes, smaller adapters padded and
+ * inactive rows masked).  Only rows/columns below a slot's true rank are ever
+ * read; padding may hold anything, NaN included.
+ *   MINT_LAYOUT_RANK_MAJOR : A[slot][r_max][d],       B[slot][r_max][n]        dense projections
+ *   MINT_LAYOUT_PACKED_MOE : A[slot][expert][d][r_max], B[slot][expert][r_max][n]
+ *     the packed MoE representation: the per-expert tensors of one projection
+ *     stacked along an expert axis (paper, packed MoE LoRA loader).           */
+enum { MINT_LAYOUT_RANK_MAJOR = 0, MINT_LAYOUT_PACKED_MOE = 1 };
+
+typedef struct {
+  int32_t d;            /* input width                                    */
+  int32_t n;            /* output width                                   */
+  int32_t r_max;        /* slot rank stride                               */
+  int32_t num_slots;
+  int32_t num_experts;  /* 0 for a dense projection                       */
+  int32_t layout;       /* MINT_LAYOUT_*                                  */
+  void *A_dev;          /* bf16, caller-owned, 16-byte aligned            */
+  void *B_dev;          /* bf16, caller-owned, 16-byte aligned            */
+} mint_pool_desc;
+
+typedef struct mint_pool mint_pool;
+typedef struct mint_slot_table mint_slot_table;
+
+const char *mint_last_error_string(void);
+const char *mint_status_name(int32_t status);
+
+/* ---- pool: the packed weights of ONE projection over all GPU slots -------
+ * The GPU-batch tier of the paper's three cache tiers (at most 64 distinct
+ * adapters resident for a decoding step; "Scale Out: Policy-Population
+ * Serving").  create copies the descriptor; the storage stays the caller's. */
+int32_t mint_pool_create(mint_pool **out, const mint_pool_desc *desc);
+int32_t mint_pool_destroy(mint_pool *pool);
+
+/* Admission of one adapter into a slot (the step that, in the paper's serving
+ * path, puts an exported adapter revision into a GPU slot before any request
+ * may use it): copy A_src (d x rank) and B_src (rank x n) into the slot, in the
+ * pool's layout; expert is ignored (pass -1) for dense pools.  Sources are in
+ * the pool's own element order with rank in place of r_max:
+ *   RANK_MAJOR: A_src[rank][d], B_src[rank][n];  PACKED_MOE: A_src[d][rank], B_src[rank][n].
+ * src_is_device selects host or device sources.  Padding is left untouched.  */
+int32_t mint_pool_write_slot(mint_pool *pool, int32_t slot, int32_t expert, const void *A_src,
+                             const void *B_src, int32_t rank, int32_t src_is_device,
+                             mint_stream_t stream);
+
+/* ---- slot table: catalog id -> slot, slot -> (rank, scale) ---------------
+ * The engine-local adapter id of the paper's serving map: a catalog of up to
+ * 10^6 addressable ids of which a bounded subset is resident.  The three device
+ * arrays are the caller's; create enqueues their initialisation (all ids
+ * unbound, all slots empty) on the stream.  A host mirror validates bind/evict
+ * and carries a generation counter that every bind/evict bumps; plans record
+ * it and an apply with an older plan reports MINT_ERR_STALE_PLAN.            */
+int32_t mint_slot_table_create(mint_slot_table **out, int64_t catalog_size, int32_t num_slots,
+                               int32_t *id_to_slot_dev /*[catalog_size]*/,
+                               int32_t *slot_rank_dev /*[num_slots]*/,
+                               float *slot_scale_dev /*[num_slots]*/, mint_stream_t stream);
+int32_t mint_slot_table_bind(mint_slot_table *table, int64_t catalog_id, int32_t slot, int32_t rank,
+                             float scale, mint_stream_t stream);
+/* count binds from host arrays, in order; stops at the first invalid one.   */
+int32_t mint_slot_table_bind_many(mint_slot_table *table, int64_t count, const int64_t *catalog_ids,
+                                  const int32_t *slots, const int32_t *ranks, const float *scales,
+                                  mint_stream_t stream);
+int32_t mint_slot_table_evict(mint_slot_table *table, int64_t catalog_id, mint_stream_t stream);
+int32_t mint_slot_table_destroy(mint_slot_table *table);
+int64_t mint_slot_table_generation(const mint_slot_table *table);
+
+/* ---- plan: token -> adapter segmentation, once per batch ------------------
+ * Groups the batch's work items by the adapter slot they use (paper: batch
+ * construction respects the same-batch adapter limit; a batch holds several
+ * adapters).  Items are tokens (dense: expert_ids_dev = NULL, K = 1) or
+ * (token, k) pairs p = t*K + k (MoE).  key = slot for dense, expert*num_slots +
+ * slot for MoE.  Canonical result: items with an adapter, ordered by key
+ * ascending and by item index ascending inside a key (the stable grouping);
+ * one segment per distinct key.  ids_dev[t] = -1 means "no adapter": the item
+ * is dropped and its output row is never touched.  An id that is not resident
+ * is dropped too, counted in status_dev[1], and status_dev[0] becomes
+ * MINT_ERR_NOT_RESIDENT.
+ *
+ * The plan is an opaque device blob of mint_lora_plan_bytes() bytes (plan
+ * arrays, derived tile lists for the kernels, and the sort scratch).  It is
+ * reused by every layer and projection of the step; the calls that consume it
+ * take the same T (and K) it was made with and report MINT_ERR_SHAPE_MISMATCH
+ * in status_dev when they differ.  mint_lora_plan_layout
+ * gives the byte offsets of the canonical arrays inside the blob:
+ *   perm int32[n_active], seg_start int32[S+1], seg_key int32[S].           */
+typedef struct {
+  int64_t total_bytes;
+  int64_t header_off;     /* int32[MINT_PLAN_HEADER_WORDS] */
+  int64_t perm_off;
+  int64_t seg_start_off;
+  int64_t seg_key_off;
+} mint_plan_layout;
+
+typedef struct {
+  int32_t num_items;      /* T*K                                            */
+  int32_t num_active;     /* items with a resident adapter                  */
+  int32_t num_segments;   /* S                                              */
+  int32_t max_segment;    /* longest segment                                */
+  int32_t sum_rank;       /* sum over segments of the slot's true rank      */
+  int32_t not_resident;   /* tokens whose id was not resident               */
+  int32_t bad_expert;     /* pairs whose expert id was out of range         */
+  int32_t reserved;
+  int64_t generation;     /* slot-table generation the plan was made under  */
+} mint_plan_summary;
+
+size_t mint_lora_plan_bytes(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts);
+int32_t mint_lora_plan_layout(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts,
+                              mint_plan_layout *out);
+int32_t mint_lora_plan(const mint_slot_table *table, const int64_t *ids_dev /*[T]*/, int32_t T,
+                       const int32_t *expert_ids_dev /*[T*K] or NULL*/, int32_t K,
+                       int32_t num_experts, void *plan_dev, size_t plan_bytes, int32_t *status_dev,
+                       mint_stream_t stream);
+/* Copies the plan's counters to the host; synchronises the stream.          */
+int32_t mint_plan_fetch_summary(const void *plan_dev, mint_plan_summary *host_out,
+                                mint_stream_t stream);
+
+/* ---- shrink: v[t, :r] = x[t, :] . A_sigma   (d -> r) ----------------------
+ * x_dev: bf16 [T][ldx].  v_dev: fp32 [T][r_max] in ORIGINAL token order; the
+ * call defines all of it: columns at or beyond the token's rank and rows of
+ * tokens without a resident adapter are written as 0.  Dense pools only.    */
+int32_t mint_lora_shrink(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                         int32_t T, const void *x_dev, int64_t ldx, float *v_dev,
+                         int32_t *status_dev, mint_stream_t stream);
+
+/* ---- expand: y[t, :] += s_sigma * (v[t, :r] . B_sigma)   (r -> n) ---------
+ * y_dev: bf16 [T][ldy], read-modified-written in place: one fp32 add of y and
+ * the scaled delta, one round-to-nearest-even store.  Rows of tokens without
+ * a resident adapter are neither read nor written.                           */
+int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                         int32_t T, const float *v_dev, void *y_dev, int64_t ldy,
+                         int32_t *status_dev, mint_stream_t stream);
+
+/* ---- fused apply: shrink + expand in one launch, v never leaves the chip ---
+ * Same result as shrink followed by expand (fp32 accumulation, summation order
+ * may differ).  workspace_dev may be NULL when mint_lora_apply_workspace_bytes
+ * returns 0 for the pool and T.                                              */
+size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T);
+int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table,
+                              const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
+                              void *y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes,
+                              int32_t *status_dev, mint_stream_t stream);
+
+/* ---- MoE expert LoRA apply -------------------------------------------------
+ * Per-expert LoRA tensors keyed by expert id (paper, "Scale Up", Megatron
+ * placement), in the packed layout.  For pair p = t*K + k with expert e and
+ * slot sigma of token t:
+ *   Y[p, :] += s_sigma * w_p * (X[row(p), :] . A[sigma][e]) . B[sigma][e]
+ * row(p) = x_row_dev[p], or p when x_row_dev is NULL (gate/up projections pass
+ * row(p) = t, the down projection reads the pair's own intermediate row);
+ * w_p = pair_weight_dev[p], or 1 when NULL.  y_dev: bf16 [T*K][ldy].
+ * plan_dev must be a MoE plan (expert_ids given) made with the pool's
+ * num_experts.  x_rows is the number of rows of x_dev (range check).         */
+size_t mint_moe_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K);
+int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table,
+                            const void *plan_dev, int32_t T, int32_t K, const void *x_dev,
+                            int64_t ldx, int64_t x_rows,
+                            const int32_t *x_row_dev, const float *pair_weight_dev, void *y_dev,
+                            int64_t ldy, void *workspace_dev, size_t workspace_bytes,
+                            int32_t *status_dev, mint_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MINT_LORA_H */

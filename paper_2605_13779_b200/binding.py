@@ -1,0 +1,342 @@
+"""Thin Python binding of libmint_lora.so (the C ABI in include/mint_lora.h).
+
+Argument marshalling only: every step of the LoRA apply runs in the CUDA
+library.  PyTorch supplies device memory and the stream.  There is no CPU
+fallback: if the library is missing, importing it here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmint_lora.so")
+
+MINT_OK = 0
+MINT_ERR_INVALID_ARG = -1
+MINT_ERR_NOT_RESIDENT = -2
+MINT_ERR_SHAPE_MISMATCH = -3
+MINT_ERR_RANK_TOO_LARGE = -4
+MINT_ERR_WORKSPACE_TOO_SMALL = -5
+MINT_ERR_MISALIGNED = -6
+MINT_ERR_CUDA = -7
+MINT_ERR_TIMEOUT = -8
+MINT_ERR_UNSUPPORTED = -9
+MINT_ERR_STALE_PLAN = -10
+MINT_ERR_BAD_INDEX = -11
+MINT_STATUS_WORDS = 4
+MINT_LAYOUT_RANK_MAJOR = 0
+MINT_LAYOUT_PACKED_MOE = 1
+
+# Every symbol include/mint_lora.h declares (the CPU test checks the export list).
+EXPORTS = [
+    "mint_last_error_string", "mint_status_name",
+    "mint_pool_create", "mint_pool_destroy", "mint_pool_write_slot",
+    "mint_slot_table_create", "mint_slot_table_bind", "mint_slot_table_bind_many",
+    "mint_slot_table_evict", "mint_slot_table_destroy", "mint_slot_table_generation",
+    "mint_lora_plan_bytes", "mint_lora_plan_layout", "mint_lora_plan", "mint_plan_fetch_summary",
+    "mint_lora_shrink", "mint_lora_expand",
+    "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused",
+    "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
+]
+
+
+class MintError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{status_name(status)} ({status}): {message}")
+        self.status = status
+
+
+class PoolDesc(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int32), ("n", ctypes.c_int32), ("r_max", ctypes.c_int32),
+                ("num_slots", ctypes.c_int32), ("num_experts", ctypes.c_int32),
+                ("layout", ctypes.c_int32), ("A_dev", ctypes.c_void_p), ("B_dev", ctypes.c_void_p)]
+
+
+class PlanLayout(ctypes.Structure):
+    _fields_ = [("total_bytes", ctypes.c_int64), ("header_off", ctypes.c_int64),
+                ("perm_off", ctypes.c_int64), ("seg_start_off", ctypes.c_int64),
+                ("seg_key_off", ctypes.c_int64)]
+
+
+class PlanSummary(ctypes.Structure):
+    _fields_ = [("num_items", ctypes.c_int32), ("num_active", ctypes.c_int32),
+                ("num_segments", ctypes.c_int32), ("max_segment", ctypes.c_int32),
+                ("sum_rank", ctypes.c_int32), ("not_resident", ctypes.c_int32),
+                ("bad_expert", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("generation", ctypes.c_int64)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libmint_lora.so from the package directory.  Raises when it has not
+    been built (python -m paper_2605_13779_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with "
+                          "`python -m paper_2605_13779_b200.build` (there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float, ctypes.c_size_t
+    sig = {
+        "mint_last_error_string": (ctypes.c_char_p, []),
+        "mint_status_name": (ctypes.c_char_p, [i32]),
+        "mint_pool_create": (i32, [ctypes.POINTER(vp), ctypes.POINTER(PoolDesc)]),
+        "mint_pool_destroy": (i32, [vp]),
+        "mint_pool_write_slot": (i32, [vp, i32, i32, vp, vp, i32, i32, vp]),
+        "mint_slot_table_create": (i32, [ctypes.POINTER(vp), i64, i32, vp, vp, vp, vp]),
+        "mint_slot_table_bind": (i32, [vp, i64, i32, i32, f32, vp]),
+        "mint_slot_table_bind_many": (i32, [vp, i64, vp, vp, vp, vp, vp]),
+        "mint_slot_table_evict": (i32, [vp, i64, vp]),
+        "mint_slot_table_destroy": (i32, [vp]),
+        "mint_slot_table_generation": (i64, [vp]),
+        "mint_lora_plan_bytes": (sz, [i32, i32, i32, i32]),
+        "mint_lora_plan_layout": (i32, [i32, i32, i32, i32, ctypes.POINTER(PlanLayout)]),
+        "mint_lora_plan": (i32, [vp, vp, i32, vp, i32, i32, vp, sz, vp, vp]),
+        "mint_plan_fetch_summary": (i32, [vp, ctypes.POINTER(PlanSummary), vp]),
+        "mint_lora_shrink": (i32, [vp, vp, vp, i32, vp, i64, vp, vp, vp]),
+        "mint_lora_expand": (i32, [vp, vp, vp, i32, vp, vp, i64, vp, vp]),
+        "mint_lora_apply_workspace_bytes": (sz, [vp, i32]),
+        "mint_lora_apply_fused": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, sz, vp, vp]),
+        "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
+        "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def status_name(status: int) -> str:
+    return load_library().mint_status_name(int(status)).decode()
+
+
+def last_error() -> str:
+    return load_library().mint_last_error_string().decode()
+
+
+def _check(status: int):
+    if status != MINT_OK:
+        raise MintError(status, last_error())
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_cuda, "device tensor expected"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def bf16_from_bits(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    """uint16 bf16 bit patterns (numpy) -> torch.bfloat16 tensor on the device."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.view(torch.bfloat16).to(device)
+
+
+def bits_from_bf16(t: torch.Tensor) -> np.ndarray:
+    """torch.bfloat16 tensor -> uint16 bit patterns on the host."""
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def new_status(device="cuda") -> torch.Tensor:
+    return torch.zeros(MINT_STATUS_WORDS, dtype=torch.int32, device=device)
+
+
+# --------------------------------------------------------------------------
+# handles
+# --------------------------------------------------------------------------
+class Pool:
+    """Packed weights of one projection over all GPU slots (caller-owned
+    tensors A, B in bf16)."""
+
+    def __init__(self, A: torch.Tensor, B: torch.Tensor, d: int, n: int, r_max: int, num_slots: int,
+                 num_experts: int = 0, layout: Optional[int] = None):
+        lib = load_library()
+        if layout is None:
+            layout = MINT_LAYOUT_PACKED_MOE if num_experts > 0 else MINT_LAYOUT_RANK_MAJOR
+        self.A, self.B = A, B
+        self.d, self.n, self.r_max, self.num_slots, self.num_experts = d, n, r_max, num_slots, num_experts
+        self.layout = layout
+        desc = PoolDesc(d, n, r_max, num_slots, num_experts, layout, _ptr(A), _ptr(B))
+        h = ctypes.c_void_p()
+        _check(lib.mint_pool_create(ctypes.byref(h), ctypes.byref(desc)))
+        self.handle = h
+
+    def write_slot(self, slot: int, A_src, B_src, rank: int, expert: int = -1):
+        """A_src/B_src: torch tensors (device or pinned/pageable host), bf16."""
+        lib = load_library()
+        on_dev = A_src.is_cuda
+        assert B_src.is_cuda == on_dev
+        _check(lib.mint_pool_write_slot(self.handle, slot, expert, A_src.data_ptr(), B_src.data_ptr(),
+                                        rank, 1 if on_dev else 0, _stream()))
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.mint_pool_destroy(self.handle)
+            self.handle = None
+
+
+class SlotTable:
+    """Catalog id -> slot and per-slot (rank, scale); device arrays are torch
+    tensors owned here, the host mirror lives in the library handle."""
+
+    def __init__(self, catalog_size: int, num_slots: int, device="cuda"):
+        lib = load_library()
+        self.catalog_size, self.num_slots = catalog_size, num_slots
+        self.id_to_slot = torch.empty(catalog_size, dtype=torch.int32, device=device)
+        self.slot_rank = torch.empty(num_slots, dtype=torch.int32, device=device)
+        self.slot_scale = torch.empty(num_slots, dtype=torch.float32, device=device)
+        h = ctypes.c_void_p()
+        _check(lib.mint_slot_table_create(ctypes.byref(h), catalog_size, num_slots, _ptr(self.id_to_slot),
+                                          _ptr(self.slot_rank), _ptr(self.slot_scale), _stream()))
+        self.handle = h
+
+    def bind(self, catalog_id: int, slot: int, rank: int, scale: float):
+        _check(load_library().mint_slot_table_bind(self.handle, catalog_id, slot, rank, scale, _stream()))
+
+    def bind_many(self, ids, slots, ranks, scales):
+        ids = np.ascontiguousarray(ids, dtype=np.int64)
+        slots = np.ascontiguousarray(slots, dtype=np.int32)
+        ranks = np.ascontiguousarray(ranks, dtype=np.int32)
+        scales = np.ascontiguousarray(scales, dtype=np.float32)
+        assert ids.shape == slots.shape == ranks.shape == scales.shape
+        _check(load_library().mint_slot_table_bind_many(
+            self.handle, ids.shape[0], ids.ctypes.data, slots.ctypes.data, ranks.ctypes.data,
+            scales.ctypes.data, _stream()))
+
+    def evict(self, catalog_id: int):
+        _check(load_library().mint_slot_table_evict(self.handle, catalog_id, _stream()))
+
+    @property
+    def generation(self) -> int:
+        return int(load_library().mint_slot_table_generation(self.handle))
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.mint_slot_table_destroy(self.handle)
+            self.handle = None
+
+
+class Plan:
+    """The opaque device plan blob plus the shape it was made for."""
+
+    def __init__(self, T: int, K: int, num_slots: int, num_experts: int, device="cuda"):
+        lib = load_library()
+        self.T, self.K, self.num_slots, self.num_experts = T, K, num_slots, num_experts
+        self.layout = PlanLayout()
+        _check(lib.mint_lora_plan_layout(T, K, num_slots, num_experts, ctypes.byref(self.layout)))
+        self.nbytes = int(lib.mint_lora_plan_bytes(T, K, num_slots, num_experts))
+        assert self.nbytes == self.layout.total_bytes
+        self.blob = torch.empty(self.nbytes, dtype=torch.uint8, device=device)
+
+    def summary(self) -> PlanSummary:
+        s = PlanSummary()
+        _check(load_library().mint_plan_fetch_summary(_ptr(self.blob), ctypes.byref(s), _stream()))
+        return s
+
+    def arrays(self) -> dict:
+        """Canonical plan arrays on the host (synchronises): perm, seg_start, seg_key."""
+        s = self.summary()
+        host = self.blob.cpu().numpy()
+
+        def take(off, count):
+            return host[off:off + 4 * count].view(np.int32).copy()
+        return {
+            "perm": take(self.layout.perm_off, s.num_active),
+            "seg_start": take(self.layout.seg_start_off, s.num_segments + 1),
+            "seg_key": take(self.layout.seg_key_off, s.num_segments),
+            "S": s.num_segments,
+            "n_active": s.num_active,
+            "n_not_resident": s.not_resident,
+            "n_bad_expert": s.bad_expert,
+            "max_segment": s.max_segment,
+            "sum_rank": s.sum_rank,
+        }
+
+
+# --------------------------------------------------------------------------
+# calls (same names as the C ABI)
+# --------------------------------------------------------------------------
+def mint_lora_plan(table: SlotTable, ids: torch.Tensor, status: torch.Tensor,
+                   expert_ids: Optional[torch.Tensor] = None, num_experts: int = 0,
+                   plan: Optional[Plan] = None) -> Plan:
+    assert ids.dtype == torch.int64 and ids.is_contiguous()
+    T = ids.shape[0]
+    K = 1
+    if expert_ids is not None:
+        assert expert_ids.dtype == torch.int32 and expert_ids.is_contiguous()
+        K = expert_ids.shape[1] if expert_ids.dim() == 2 else 1
+    if plan is None:
+        plan = Plan(T, K, table.num_slots, num_experts, device=ids.device)
+    _check(load_library().mint_lora_plan(table.handle, _ptr(ids) if T else None, T, _ptr(expert_ids), K,
+                                         num_experts, _ptr(plan.blob), plan.nbytes, _ptr(status), _stream()))
+    return plan
+
+
+def mint_lora_shrink(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, status: torch.Tensor,
+                     v: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if v is None:
+        v = torch.empty(plan.T, pool.r_max, dtype=torch.float32, device=x.device)
+    assert v.dtype == torch.float32 and v.is_contiguous()
+    _check(load_library().mint_lora_shrink(pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x),
+                                           x.stride(0) if x.dim() == 2 and x.shape[0] > 0 else pool.d,
+                                           _ptr(v), _ptr(status), _stream()))
+    return v
+
+
+def mint_lora_expand(pool: Pool, table: SlotTable, plan: Plan, v: torch.Tensor, y: torch.Tensor,
+                     status: torch.Tensor) -> torch.Tensor:
+    _check(load_library().mint_lora_expand(pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(v),
+                                           _ptr(y), y.stride(0) if y.dim() == 2 and y.shape[0] > 0 else pool.n,
+                                           _ptr(status), _stream()))
+    return y
+
+
+def mint_lora_apply_workspace_bytes(pool: Pool, T: int) -> int:
+    return int(load_library().mint_lora_apply_workspace_bytes(pool.handle, T))
+
+
+def mint_lora_apply_fused(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
+                          status: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _check(load_library().mint_lora_apply_fused(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x),
+        x.stride(0) if x.dim() == 2 and x.shape[0] > 0 else pool.d, _ptr(y),
+        y.stride(0) if y.dim() == 2 and y.shape[0] > 0 else pool.n,
+        _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+        _ptr(status), _stream()))
+    return y
+
+
+def mint_moe_lora_apply_workspace_bytes(pool: Pool, T: int, K: int) -> int:
+    return int(load_library().mint_moe_lora_apply_workspace_bytes(pool.handle, T, K))
+
+
+def mint_moe_lora_apply(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
+                        status: torch.Tensor, x_row: Optional[torch.Tensor] = None,
+                        pair_weight: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if x_row is not None:
+        assert x_row.dtype == torch.int32 and x_row.is_contiguous()
+    if pair_weight is not None:
+        assert pair_weight.dtype == torch.float32 and pair_weight.is_contiguous()
+    _check(load_library().mint_moe_lora_apply(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, plan.K, _ptr(x), x.stride(0), x.shape[0],
+        _ptr(x_row), _ptr(pair_weight), _ptr(y), y.stride(0),
+        _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+        _ptr(status), _stream()))
+    return y

@@ -1,0 +1,556 @@
+// Host side of the C ABI: argument validation, the pool and slot-table
+// handles, and the launch of each kernel on the caller's stream.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "mint_device.cuh"
+
+// ---------------------------------------------------------------------------
+// errors
+// ---------------------------------------------------------------------------
+static thread_local char g_err[512] = "";
+
+int32_t mint_fail(int32_t code, const char *fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof g_err, fmt, ap);
+  va_end(ap);
+  return code;
+}
+
+int32_t mint_check_cuda(cudaError_t e, const char *what) {
+  if (e == cudaSuccess) return MINT_OK;
+  return mint_fail(MINT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+extern "C" const char *mint_last_error_string(void) { return g_err; }
+
+extern "C" const char *mint_status_name(int32_t s) {
+  switch (s) {
+    case MINT_OK: return "MINT_OK";
+    case MINT_ERR_INVALID_ARG: return "MINT_ERR_INVALID_ARG";
+    case MINT_ERR_NOT_RESIDENT: return "MINT_ERR_NOT_RESIDENT";
+    case MINT_ERR_SHAPE_MISMATCH: return "MINT_ERR_SHAPE_MISMATCH";
+    case MINT_ERR_RANK_TOO_LARGE: return "MINT_ERR_RANK_TOO_LARGE";
+    case MINT_ERR_WORKSPACE_TOO_SMALL: return "MINT_ERR_WORKSPACE_TOO_SMALL";
+    case MINT_ERR_MISALIGNED: return "MINT_ERR_MISALIGNED";
+    case MINT_ERR_CUDA: return "MINT_ERR_CUDA";
+    case MINT_ERR_TIMEOUT: return "MINT_ERR_TIMEOUT";
+    case MINT_ERR_UNSUPPORTED: return "MINT_ERR_UNSUPPORTED";
+    case MINT_ERR_STALE_PLAN: return "MINT_ERR_STALE_PLAN";
+    case MINT_ERR_BAD_INDEX: return "MINT_ERR_BAD_INDEX";
+    default: return "MINT_ERR_UNKNOWN";
+  }
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static const int64_t kMaxItems = 1ll << 24;
+
+// ---------------------------------------------------------------------------
+// small device kernels for the slot table
+// ---------------------------------------------------------------------------
+namespace {
+
+__global__ void table_init_kernel(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
+                                  float *slot_scale, int32_t num_slots) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < catalog_size; i += stride)
+    id_to_slot[i] = -1;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < num_slots; i += stride) {
+    slot_rank[i] = 0;
+    slot_scale[i] = 0.f;
+  }
+}
+
+// Entries are applied in order by one thread: later entries of a batch may
+// rebind a slot an earlier one emptied.
+__global__ void bind_kernel(int32_t *id_to_slot, int32_t *slot_rank, float *slot_scale,
+                            const BindBatch b) {
+  if (blockIdx.x != 0 || threadIdx.x != 0) return;
+  for (int i = 0; i < b.count; ++i) {
+    if (b.slot[i] < 0) {
+      id_to_slot[b.id[i]] = -1;
+      slot_rank[b.old_slot[i]] = 0;
+      slot_scale[b.old_slot[i]] = 0.f;
+    } else {
+      id_to_slot[b.id[i]] = b.slot[i];
+      slot_rank[b.slot[i]] = b.rank[i];
+      slot_scale[b.slot[i]] = b.scale[i];
+    }
+  }
+}
+
+}  // namespace
+
+int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
+                               float *slot_scale, int32_t num_slots, cudaStream_t s) {
+  int64_t blocks = (catalog_size + 255) / 256;
+  if (blocks > 1184) blocks = 1184;
+  if (blocks < 1) blocks = 1;
+  table_init_kernel<<<(unsigned)blocks, 256, 0, s>>>(id_to_slot, catalog_size, slot_rank, slot_scale,
+                                                      num_slots);
+  return mint_check_cuda(cudaGetLastError(), "slot table init launch");
+}
+
+int32_t mint_launch_bind(int32_t *id_to_slot, int32_t *slot_rank, float *slot_scale,
+                         const BindBatch &batch, cudaStream_t s) {
+  bind_kernel<<<1, 32, 0, s>>>(id_to_slot, slot_rank, slot_scale, batch);
+  return mint_check_cuda(cudaGetLastError(), "slot table bind launch");
+}
+
+// ---------------------------------------------------------------------------
+// pool
+// ---------------------------------------------------------------------------
+extern "C" int32_t mint_pool_create(mint_pool **out, const mint_pool_desc *desc) {
+  if (!out || !desc) return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: null argument");
+  *out = nullptr;
+  if (desc->d <= 0 || desc->n <= 0 || desc->r_max <= 0 || desc->num_slots <= 0 || desc->num_experts < 0)
+    return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: non-positive dimension");
+  if ((desc->d & 7) || (desc->n & 7))
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "pool_create: d=%d and n=%d must be multiples of 8",
+                     desc->d, desc->n);
+  if (desc->r_max > mint::kRankCapHost)
+    return mint_fail(MINT_ERR_RANK_TOO_LARGE, "pool_create: r_max=%d exceeds the supported %d",
+                     desc->r_max, mint::kRankCapHost);
+  if (desc->layout == MINT_LAYOUT_RANK_MAJOR) {
+    if (desc->num_experts != 0)
+      return mint_fail(MINT_ERR_UNSUPPORTED, "pool_create: rank-major layout is for dense pools (num_experts=0)");
+  } else if (desc->layout == MINT_LAYOUT_PACKED_MOE) {
+    if (desc->num_experts < 1)
+      return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: packed MoE layout needs num_experts >= 1");
+  } else {
+    return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: unknown layout %d", desc->layout);
+  }
+  if (!desc->A_dev || !desc->B_dev) return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: null storage");
+  if (!aligned16(desc->A_dev) || !aligned16(desc->B_dev))
+    return mint_fail(MINT_ERR_MISALIGNED, "pool_create: A_dev/B_dev must be 16-byte aligned");
+  mint_pool *p = new (std::nothrow) mint_pool;
+  if (!p) return mint_fail(MINT_ERR_INVALID_ARG, "pool_create: out of host memory");
+  p->desc = *desc;
+  *out = p;
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_pool_destroy(mint_pool *pool) {
+  delete pool;
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_pool_write_slot(mint_pool *pool, int32_t slot, int32_t expert, const void *A_src,
+                                        const void *B_src, int32_t rank, int32_t src_is_device,
+                                        mint_stream_t stream) {
+  if (!pool || !A_src || !B_src) return mint_fail(MINT_ERR_INVALID_ARG, "write_slot: null argument");
+  const mint_pool_desc &p = pool->desc;
+  if (slot < 0 || slot >= p.num_slots) return mint_fail(MINT_ERR_INVALID_ARG, "write_slot: slot %d out of range", slot);
+  if (rank < 1) return mint_fail(MINT_ERR_INVALID_ARG, "write_slot: rank %d", rank);
+  if (rank > p.r_max) return mint_fail(MINT_ERR_RANK_TOO_LARGE, "write_slot: rank %d > r_max %d", rank, p.r_max);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const cudaMemcpyKind kind = src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+  uint16_t *A = static_cast<uint16_t *>(p.A_dev);
+  uint16_t *B = static_cast<uint16_t *>(p.B_dev);
+  if (p.layout == MINT_LAYOUT_RANK_MAJOR) {
+    int32_t st = mint_check_cuda(cudaMemcpyAsync(A + (int64_t)slot * p.r_max * p.d, A_src,
+                                                 (size_t)rank * p.d * 2, kind, s), "write_slot A");
+    if (st) return st;
+    return mint_check_cuda(cudaMemcpyAsync(B + (int64_t)slot * p.r_max * p.n, B_src,
+                                           (size_t)rank * p.n * 2, kind, s), "write_slot B");
+  }
+  if (expert < 0 || expert >= p.num_experts)
+    return mint_fail(MINT_ERR_INVALID_ARG, "write_slot: expert %d out of range", expert);
+  const int64_t se = (int64_t)slot * p.num_experts + expert;
+  int32_t st = mint_check_cuda(cudaMemcpy2DAsync(A + se * p.d * p.r_max, (size_t)p.r_max * 2, A_src,
+                                                 (size_t)rank * 2, (size_t)rank * 2, (size_t)p.d, kind, s),
+                               "write_slot A");
+  if (st) return st;
+  return mint_check_cuda(cudaMemcpyAsync(B + se * p.r_max * p.n, B_src, (size_t)rank * p.n * 2, kind, s),
+                         "write_slot B");
+}
+
+// ---------------------------------------------------------------------------
+// slot table
+// ---------------------------------------------------------------------------
+extern "C" int32_t mint_slot_table_create(mint_slot_table **out, int64_t catalog_size, int32_t num_slots,
+                                          int32_t *id_to_slot_dev, int32_t *slot_rank_dev,
+                                          float *slot_scale_dev, mint_stream_t stream) {
+  if (!out) return mint_fail(MINT_ERR_INVALID_ARG, "slot_table_create: null out");
+  *out = nullptr;
+  if (catalog_size <= 0 || num_slots <= 0 || catalog_size > (1ll << 31) - 1)
+    return mint_fail(MINT_ERR_INVALID_ARG, "slot_table_create: catalog_size=%lld num_slots=%d",
+                     (long long)catalog_size, num_slots);
+  if (!id_to_slot_dev || !slot_rank_dev || !slot_scale_dev)
+    return mint_fail(MINT_ERR_INVALID_ARG, "slot_table_create: null device array");
+  mint_slot_table *t = new (std::nothrow) mint_slot_table;
+  if (!t) return mint_fail(MINT_ERR_INVALID_ARG, "slot_table_create: out of host memory");
+  t->catalog_size = catalog_size;
+  t->num_slots = num_slots;
+  t->id_to_slot_dev = id_to_slot_dev;
+  t->slot_rank_dev = slot_rank_dev;
+  t->slot_scale_dev = slot_scale_dev;
+  t->generation = 1;
+  t->max_rank = 0;
+  t->id_to_slot_host = static_cast<int32_t *>(malloc(sizeof(int32_t) * (size_t)catalog_size));
+  t->slots_host = static_cast<SlotBinding *>(malloc(sizeof(SlotBinding) * (size_t)num_slots));
+  if (!t->id_to_slot_host || !t->slots_host) {
+    free(t->id_to_slot_host);
+    free(t->slots_host);
+    delete t;
+    return mint_fail(MINT_ERR_INVALID_ARG, "slot_table_create: out of host memory");
+  }
+  for (int64_t i = 0; i < catalog_size; ++i) t->id_to_slot_host[i] = -1;
+  for (int32_t i = 0; i < num_slots; ++i) t->slots_host[i] = SlotBinding{-1, 0, 0.f};
+  int32_t st = mint_launch_table_init(id_to_slot_dev, catalog_size, slot_rank_dev, slot_scale_dev, num_slots,
+                                      static_cast<cudaStream_t>(stream));
+  if (st) {
+    free(t->id_to_slot_host);
+    free(t->slots_host);
+    delete t;
+    return st;
+  }
+  *out = t;
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_slot_table_destroy(mint_slot_table *t) {
+  if (t) {
+    free(t->id_to_slot_host);
+    free(t->slots_host);
+    delete t;
+  }
+  return MINT_OK;
+}
+
+extern "C" int64_t mint_slot_table_generation(const mint_slot_table *t) { return t ? t->generation : -1; }
+
+static int32_t validate_bind(const mint_slot_table *t, int64_t id, int32_t slot, int32_t rank) {
+  if (id < 0 || id >= t->catalog_size)
+    return mint_fail(MINT_ERR_INVALID_ARG, "bind: catalog id %lld outside [0, %lld)", (long long)id,
+                     (long long)t->catalog_size);
+  if (slot < 0 || slot >= t->num_slots) return mint_fail(MINT_ERR_INVALID_ARG, "bind: slot %d out of range", slot);
+  if (rank < 1) return mint_fail(MINT_ERR_INVALID_ARG, "bind: rank %d", rank);
+  if (rank > mint::kRankCapHost) return mint_fail(MINT_ERR_RANK_TOO_LARGE, "bind: rank %d exceeds %d", rank, mint::kRankCapHost);
+  if (t->id_to_slot_host[id] >= 0)
+    return mint_fail(MINT_ERR_INVALID_ARG, "bind: id %lld is already resident in slot %d", (long long)id,
+                     t->id_to_slot_host[id]);
+  if (t->slots_host[slot].catalog_id >= 0)
+    return mint_fail(MINT_ERR_INVALID_ARG, "bind: slot %d is occupied by id %lld", slot,
+                     (long long)t->slots_host[slot].catalog_id);
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_slot_table_bind_many(mint_slot_table *t, int64_t count, const int64_t *ids,
+                                             const int32_t *slots, const int32_t *ranks, const float *scales,
+                                             mint_stream_t stream) {
+  if (!t || count < 0 || (count > 0 && (!ids || !slots || !ranks || !scales)))
+    return mint_fail(MINT_ERR_INVALID_ARG, "bind_many: null argument");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  BindBatch b;
+  b.count = 0;
+  int32_t result = MINT_OK;
+  auto flush = [&]() -> int32_t {
+    if (b.count == 0) return MINT_OK;
+    int32_t st = mint_launch_bind(t->id_to_slot_dev, t->slot_rank_dev, t->slot_scale_dev, b, s);
+    b.count = 0;
+    return st;
+  };
+  for (int64_t i = 0; i < count; ++i) {
+    result = validate_bind(t, ids[i], slots[i], ranks[i]);
+    if (result) break;
+    t->id_to_slot_host[ids[i]] = slots[i];
+    t->slots_host[slots[i]] = SlotBinding{ids[i], ranks[i], scales[i]};
+    if (ranks[i] > t->max_rank) t->max_rank = ranks[i];
+    ++t->generation;
+    const int k = b.count++;
+    b.id[k] = ids[i];
+    b.slot[k] = slots[i];
+    b.old_slot[k] = -1;
+    b.rank[k] = ranks[i];
+    b.scale[k] = scales[i];
+    if (b.count == BindBatch::kMax) {
+      int32_t st = flush();
+      if (st) return st;
+    }
+  }
+  int32_t st = flush();
+  return result ? result : st;
+}
+
+extern "C" int32_t mint_slot_table_bind(mint_slot_table *t, int64_t id, int32_t slot, int32_t rank, float scale,
+                                        mint_stream_t stream) {
+  return mint_slot_table_bind_many(t, 1, &id, &slot, &rank, &scale, stream);
+}
+
+extern "C" int32_t mint_slot_table_evict(mint_slot_table *t, int64_t id, mint_stream_t stream) {
+  if (!t) return mint_fail(MINT_ERR_INVALID_ARG, "evict: null table");
+  if (id < 0 || id >= t->catalog_size)
+    return mint_fail(MINT_ERR_INVALID_ARG, "evict: catalog id %lld outside the catalog", (long long)id);
+  const int32_t slot = t->id_to_slot_host[id];
+  if (slot < 0) return mint_fail(MINT_ERR_NOT_RESIDENT, "evict: id %lld is not resident", (long long)id);
+  t->id_to_slot_host[id] = -1;
+  t->slots_host[slot] = SlotBinding{-1, 0, 0.f};
+  ++t->generation;
+  int32_t mr = 0;
+  for (int32_t i = 0; i < t->num_slots; ++i)
+    if (t->slots_host[i].catalog_id >= 0 && t->slots_host[i].rank > mr) mr = t->slots_host[i].rank;
+  t->max_rank = mr;
+  BindBatch b;
+  b.count = 1;
+  b.id[0] = id;
+  b.slot[0] = -1;
+  b.old_slot[0] = slot;
+  b.rank[0] = 0;
+  b.scale[0] = 0.f;
+  return mint_launch_bind(t->id_to_slot_dev, t->slot_rank_dev, t->slot_scale_dev, b,
+                          static_cast<cudaStream_t>(stream));
+}
+
+static TableDev table_dev(const mint_slot_table *t) {
+  TableDev d;
+  d.id_to_slot = t->id_to_slot_dev;
+  d.slot_rank = t->slot_rank_dev;
+  d.slot_scale = t->slot_scale_dev;
+  d.catalog_size = t->catalog_size;
+  d.num_slots = t->num_slots;
+  d.gen_lo = (int32_t)(t->generation & 0xffffffffll);
+  d.gen_hi = (int32_t)(t->generation >> 32);
+  return d;
+}
+
+// ---------------------------------------------------------------------------
+// plan
+// ---------------------------------------------------------------------------
+static int32_t check_plan_shape(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts, const char *who) {
+  if (T < 0 || K < 1 || num_slots < 1 || num_experts < 0)
+    return mint_fail(MINT_ERR_INVALID_ARG, "%s: T=%d K=%d num_slots=%d num_experts=%d", who, T, K, num_slots,
+                     num_experts);
+  if ((int64_t)T * K > kMaxItems)
+    return mint_fail(MINT_ERR_UNSUPPORTED, "%s: T*K=%lld exceeds %lld items", who, (long long)T * K,
+                     (long long)kMaxItems);
+  if ((int64_t)num_slots * (num_experts > 0 ? num_experts : 1) > (1ll << 30))
+    return mint_fail(MINT_ERR_UNSUPPORTED, "%s: key space too large", who);
+  return MINT_OK;
+}
+
+extern "C" size_t mint_lora_plan_bytes(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts) {
+  if (check_plan_shape(T, K, num_slots, num_experts, "plan_bytes")) return 0;
+  return (size_t)mint_plan_offsets((int64_t)T * K).total;
+}
+
+extern "C" int32_t mint_lora_plan_layout(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts,
+                                         mint_plan_layout *out) {
+  if (!out) return mint_fail(MINT_ERR_INVALID_ARG, "plan_layout: null out");
+  int32_t st = check_plan_shape(T, K, num_slots, num_experts, "plan_layout");
+  if (st) return st;
+  const PlanOffsets o = mint_plan_offsets((int64_t)T * K);
+  out->total_bytes = o.total;
+  out->header_off = o.header;
+  out->perm_off = o.perm;
+  out->seg_start_off = o.seg_start;
+  out->seg_key_off = o.seg_key;
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_lora_plan(const mint_slot_table *table, const int64_t *ids_dev, int32_t T,
+                                  const int32_t *expert_ids_dev, int32_t K, int32_t num_experts,
+                                  void *plan_dev, size_t plan_bytes, int32_t *status_dev,
+                                  mint_stream_t stream) {
+  if (!table || !plan_dev || !status_dev || (T > 0 && !ids_dev))
+    return mint_fail(MINT_ERR_INVALID_ARG, "plan: null argument");
+  int32_t st = check_plan_shape(T, K, table->num_slots, num_experts, "plan");
+  if (st) return st;
+  if (expert_ids_dev == nullptr && (K != 1 || num_experts != 0))
+    return mint_fail(MINT_ERR_INVALID_ARG, "plan: a dense plan has K=1 and num_experts=0");
+  if (expert_ids_dev != nullptr && num_experts < 1)
+    return mint_fail(MINT_ERR_INVALID_ARG, "plan: a MoE plan needs num_experts >= 1");
+  if (!aligned16(plan_dev)) return mint_fail(MINT_ERR_MISALIGNED, "plan: plan_dev must be 16-byte aligned");
+  const size_t need = (size_t)mint_plan_offsets((int64_t)T * K).total;
+  if (plan_bytes < need)
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "plan: plan_bytes=%zu < %zu", plan_bytes, need);
+  return mint_launch_plan(table_dev(table), ids_dev, T, expert_ids_dev, K, num_experts, plan_dev, status_dev,
+                          static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t mint_plan_fetch_summary(const void *plan_dev, mint_plan_summary *out, mint_stream_t stream) {
+  if (!plan_dev || !out) return mint_fail(MINT_ERR_INVALID_ARG, "fetch_summary: null argument");
+  int32_t h[PH_WORDS];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t st = mint_check_cuda(cudaMemcpyAsync(h, plan_dev, sizeof h, cudaMemcpyDeviceToHost, s), "fetch_summary copy");
+  if (st) return st;
+  st = mint_check_cuda(cudaStreamSynchronize(s), "fetch_summary sync");
+  if (st) return st;
+  if (h[PH_MAGIC] != MINT_PLAN_MAGIC) return mint_fail(MINT_ERR_INVALID_ARG, "fetch_summary: not a plan");
+  out->num_items = h[PH_NUM_ITEMS];
+  out->num_active = h[PH_NUM_ACTIVE];
+  out->num_segments = h[PH_NUM_SEGMENTS];
+  out->max_segment = h[PH_MAX_SEGMENT];
+  out->sum_rank = h[PH_SUM_RANK];
+  out->not_resident = h[PH_NOT_RESIDENT];
+  out->bad_expert = h[PH_BAD_EXPERT];
+  out->reserved = 0;
+  out->generation = ((int64_t)(uint32_t)h[PH_GEN_HI] << 32) | (uint32_t)h[PH_GEN_LO];
+  return MINT_OK;
+}
+
+// ---------------------------------------------------------------------------
+// dense shrink / expand / fused
+// ---------------------------------------------------------------------------
+static int32_t check_dense(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev, int32_t T,
+                           const char *who) {
+  if (!pool || !table || !plan_dev) return mint_fail(MINT_ERR_INVALID_ARG, "%s: null argument", who);
+  if (T < 0 || T > kMaxItems) return mint_fail(MINT_ERR_INVALID_ARG, "%s: T=%d", who, T);
+  if (pool->desc.layout != MINT_LAYOUT_RANK_MAJOR || pool->desc.num_experts != 0)
+    return mint_fail(MINT_ERR_UNSUPPORTED, "%s: needs a dense rank-major pool", who);
+  if (pool->desc.num_slots != table->num_slots)
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "%s: pool has %d slots, table has %d", who, pool->desc.num_slots,
+                     table->num_slots);
+  if (table->max_rank > pool->desc.r_max)
+    return mint_fail(MINT_ERR_RANK_TOO_LARGE, "%s: a bound adapter has rank %d > pool r_max %d", who,
+                     table->max_rank, pool->desc.r_max);
+  return MINT_OK;
+}
+
+static int32_t check_act(const void *p, int64_t ld, int32_t width, const char *name, const char *who) {
+  if (!p) return mint_fail(MINT_ERR_INVALID_ARG, "%s: null %s", who, name);
+  if (!aligned16(p)) return mint_fail(MINT_ERR_MISALIGNED, "%s: %s must be 16-byte aligned", who, name);
+  if (ld < width) return mint_fail(MINT_ERR_SHAPE_MISMATCH, "%s: row stride of %s (%lld) < width %d", who, name, (long long)ld, width);
+  if (ld & 7) return mint_fail(MINT_ERR_MISALIGNED, "%s: row stride of %s (%lld) must be a multiple of 8", who, name, (long long)ld);
+  return MINT_OK;
+}
+
+static DenseArgs dense_args(const mint_pool *pool, int32_t T) {
+  DenseArgs a = {};
+  a.A = static_cast<const uint16_t *>(pool->desc.A_dev);
+  a.B = static_cast<const uint16_t *>(pool->desc.B_dev);
+  a.d = pool->desc.d;
+  a.n = pool->desc.n;
+  a.r_max = pool->desc.r_max;
+  a.num_slots = pool->desc.num_slots;
+  a.T = T;
+  return a;
+}
+
+extern "C" int32_t mint_lora_shrink(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                    int32_t T, const void *x_dev, int64_t ldx, float *v_dev, int32_t *status_dev,
+                                    mint_stream_t stream) {
+  int32_t st = check_dense(pool, table, plan_dev, T, "shrink");
+  if (st) return st;
+  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "shrink: null status_dev");
+  if (T == 0) return MINT_OK;
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "shrink"))) return st;
+  if (!v_dev) return mint_fail(MINT_ERR_INVALID_ARG, "shrink: null v_dev");
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = mint_check_cuda(cudaMemsetAsync(v_dev, 0, (size_t)T * pool->desc.r_max * sizeof(float), s), "shrink: clear v");
+  if (st) return st;
+  DenseArgs a = dense_args(pool, T);
+  a.x = static_cast<const uint16_t *>(x_dev);
+  a.ldx = ldx;
+  a.v = v_dev;
+  a.status = status_dev;
+  return mint_launch_shrink(a, table_dev(table), plan_dev, s);
+}
+
+extern "C" int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                    int32_t T, const float *v_dev, void *y_dev, int64_t ldy, int32_t *status_dev,
+                                    mint_stream_t stream) {
+  int32_t st = check_dense(pool, table, plan_dev, T, "expand");
+  if (st) return st;
+  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "expand: null status_dev");
+  if (T == 0) return MINT_OK;
+  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", "expand"))) return st;
+  if (!v_dev) return mint_fail(MINT_ERR_INVALID_ARG, "expand: null v_dev");
+  DenseArgs a = dense_args(pool, T);
+  a.y = static_cast<uint16_t *>(y_dev);
+  a.ldy = ldy;
+  a.v = const_cast<float *>(v_dev);
+  a.status = status_dev;
+  return mint_launch_expand(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T) {
+  (void)pool;
+  (void)T;
+  return 0;
+}
+
+extern "C" int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                         int32_t T, const void *x_dev, int64_t ldx, void *y_dev, int64_t ldy,
+                                         void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                                         mint_stream_t stream) {
+  int32_t st = check_dense(pool, table, plan_dev, T, "apply_fused");
+  if (st) return st;
+  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "apply_fused: null status_dev");
+  if (T == 0) return MINT_OK;
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "apply_fused"))) return st;
+  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", "apply_fused"))) return st;
+  const size_t need = mint_lora_apply_workspace_bytes(pool, T);
+  if (need > 0 && (!workspace_dev || workspace_bytes < need))
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "apply_fused: workspace %zu < %zu", workspace_bytes, need);
+  DenseArgs a = dense_args(pool, T);
+  a.x = static_cast<const uint16_t *>(x_dev);
+  a.ldx = ldx;
+  a.y = static_cast<uint16_t *>(y_dev);
+  a.ldy = ldy;
+  a.status = status_dev;
+  return mint_launch_fused(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
+}
+
+// ---------------------------------------------------------------------------
+// MoE
+// ---------------------------------------------------------------------------
+extern "C" size_t mint_moe_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K) {
+  (void)pool;
+  (void)T;
+  (void)K;
+  return 0;
+}
+
+extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                       int32_t T, int32_t K, const void *x_dev, int64_t ldx, int64_t x_rows,
+                                       const int32_t *x_row_dev, const float *pair_weight_dev, void *y_dev,
+                                       int64_t ldy, void *workspace_dev, size_t workspace_bytes,
+                                       int32_t *status_dev, mint_stream_t stream) {
+  if (!pool || !table || !plan_dev || !status_dev)
+    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: null argument");
+  if (T < 0 || K < 1 || (int64_t)T * K > kMaxItems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: T=%d K=%d", T, K);
+  if (pool->desc.layout != MINT_LAYOUT_PACKED_MOE || pool->desc.num_experts < 1)
+    return mint_fail(MINT_ERR_UNSUPPORTED, "moe_apply: needs a packed MoE pool");
+  if (pool->desc.num_slots != table->num_slots)
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "moe_apply: pool has %d slots, table has %d", pool->desc.num_slots,
+                     table->num_slots);
+  if (table->max_rank > pool->desc.r_max)
+    return mint_fail(MINT_ERR_RANK_TOO_LARGE, "moe_apply: a bound adapter has rank %d > pool r_max %d",
+                     table->max_rank, pool->desc.r_max);
+  if (T == 0) return MINT_OK;
+  int32_t st;
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "moe_apply"))) return st;
+  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", "moe_apply"))) return st;
+  if (x_rows < 1) return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: x_rows=%lld", (long long)x_rows);
+  if (!x_row_dev && x_rows < (int64_t)T * K)
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "moe_apply: identity rows need x_rows >= T*K");
+  const size_t need = mint_moe_lora_apply_workspace_bytes(pool, T, K);
+  if (need > 0 && (!workspace_dev || workspace_bytes < need))
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "moe_apply: workspace %zu < %zu", workspace_bytes, need);
+  MoEArgs a = {};
+  a.A = static_cast<const uint16_t *>(pool->desc.A_dev);
+  a.B = static_cast<const uint16_t *>(pool->desc.B_dev);
+  a.d = pool->desc.d;
+  a.n = pool->desc.n;
+  a.r_max = pool->desc.r_max;
+  a.num_slots = pool->desc.num_slots;
+  a.num_experts = pool->desc.num_experts;
+  a.T = T;
+  a.K = K;
+  a.x = static_cast<const uint16_t *>(x_dev);
+  a.ldx = ldx;
+  a.x_rows = x_rows;
+  a.x_row = x_row_dev;
+  a.pair_weight = pair_weight_dev;
+  a.y = static_cast<uint16_t *>(y_dev);
+  a.ldy = ldy;
+  a.status = status_dev;
+  return mint_launch_moe(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
+}

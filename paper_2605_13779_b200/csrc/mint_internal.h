@@ -1,0 +1,154 @@
+// Internal declarations shared by the translation units of libmint_lora.so.
+// Nothing here is part of the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mint_lora.h"
+
+namespace mint {
+constexpr int kRankCapHost = 128;  // largest slot rank any kernel here handles
+}
+
+// ---- plan blob ------------------------------------------------------------
+// Header words (int32) at the start of the plan blob.
+enum {
+  PH_MAGIC = 0,
+  PH_T,
+  PH_K,
+  PH_NUM_ITEMS,
+  PH_NUM_SLOTS,
+  PH_NUM_EXPERTS,
+  PH_NUM_ACTIVE,
+  PH_NUM_SEGMENTS,
+  PH_MAX_SEGMENT,
+  PH_SUM_RANK,
+  PH_NOT_RESIDENT,
+  PH_BAD_EXPERT,
+  PH_GEN_LO,
+  PH_GEN_HI,
+  PH_NCHUNK0,   // number of tiles in list g (MINT_NUM_TILE_LISTS entries)
+  PH_NCHUNK1,
+  PH_NCHUNK2,
+  PH_WORDS = 32
+};
+#define MINT_PLAN_MAGIC 0x4D4C5031  // "MLP1"
+#define MINT_NUM_TILE_LISTS 3
+// Tile list g cuts every segment into runs of at most kTileTokens[g] items.
+__host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : (g == 1 ? 32 : 128); }
+
+// Byte offsets of every array inside the plan blob (host-computed, passed by value).
+struct PlanOffsets {
+  int64_t header;      // int32[PH_WORDS]
+  int64_t perm;        // int32[P]        item indices grouped by key (inactive items after the active ones)
+  int64_t seg_start;   // int32[P+1]
+  int64_t seg_key;     // int32[P]
+  int64_t seg_slot;    // int32[P]
+  int64_t seg_expert;  // int32[P]
+  int64_t tile_seg[MINT_NUM_TILE_LISTS];  // int32[P]  segment of tile c
+  int64_t tile_off[MINT_NUM_TILE_LISTS];  // int32[P]  first position (in perm) of tile c
+  int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
+  int64_t total;
+};
+PlanOffsets mint_plan_offsets(int64_t P);
+// Upper bound on the number of tiles of list g, computable without reading the plan.
+int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space);
+
+// Device view of a plan: typed pointers into the blob.
+struct PlanView {
+  const int32_t *header;
+  const int32_t *perm;
+  const int32_t *seg_start;
+  const int32_t *seg_key;
+  const int32_t *seg_slot;
+  const int32_t *seg_expert;
+  const int32_t *tile_seg[MINT_NUM_TILE_LISTS];
+  const int32_t *tile_off[MINT_NUM_TILE_LISTS];
+};
+PlanView mint_plan_view(const void *plan_dev, int64_t P);
+
+// ---- host handles ----------------------------------------------------------
+struct mint_pool {
+  mint_pool_desc desc;
+};
+
+struct SlotBinding {
+  int64_t catalog_id;  // -1 = empty
+  int32_t rank;
+  float scale;
+};
+
+struct mint_slot_table {
+  int64_t catalog_size;
+  int32_t num_slots;
+  int32_t *id_to_slot_dev;
+  int32_t *slot_rank_dev;
+  float *slot_scale_dev;
+  int64_t generation;
+  int32_t max_rank;          // largest rank currently bound
+  int32_t *id_to_slot_host;  // mirror [catalog_size]
+  SlotBinding *slots_host;   // mirror [num_slots]
+};
+
+// ---- error reporting --------------------------------------------------------
+int32_t mint_fail(int32_t code, const char *fmt, ...);
+int32_t mint_check_cuda(cudaError_t e, const char *what);
+
+// ---- kernel launchers (each returns MINT_OK or MINT_ERR_CUDA) ---------------
+struct TableDev {
+  const int32_t *id_to_slot;
+  const int32_t *slot_rank;
+  const float *slot_scale;
+  int64_t catalog_size;
+  int32_t num_slots;
+  int32_t gen_lo, gen_hi;
+};
+
+int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, const int32_t *expert_ids,
+                         int32_t K, int32_t num_experts, void *plan_dev, int32_t *status,
+                         cudaStream_t stream);
+
+struct DenseArgs {
+  const uint16_t *A;   // [slot][r_max][d]
+  const uint16_t *B;   // [slot][r_max][n]
+  int32_t d, n, r_max, num_slots;
+  int32_t T;
+  const uint16_t *x;
+  int64_t ldx;
+  uint16_t *y;
+  int64_t ldy;
+  float *v;            // [T][r_max] (unfused calls)
+  int32_t *status;
+};
+int32_t mint_launch_shrink(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
+int32_t mint_launch_expand(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
+int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
+
+struct MoEArgs {
+  const uint16_t *A;   // [slot][E][d][r_max]
+  const uint16_t *B;   // [slot][E][r_max][n]
+  int32_t d, n, r_max, num_slots, num_experts;
+  int32_t T, K;
+  const uint16_t *x;
+  int64_t ldx, x_rows;
+  const int32_t *x_row;
+  const float *pair_weight;
+  uint16_t *y;
+  int64_t ldy;
+  int32_t *status;
+};
+int32_t mint_launch_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
+
+int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
+                               float *slot_scale, int32_t num_slots, cudaStream_t s);
+struct BindBatch {
+  static constexpr int kMax = 128;
+  int32_t count;
+  int64_t id[kMax];
+  int32_t slot[kMax];   // -1 = evict (id unbound; slot in old_slot emptied)
+  int32_t old_slot[kMax];
+  int32_t rank[kMax];
+  float scale[kMax];
+};
+int32_t mint_launch_bind(int32_t *id_to_slot, int32_t *slot_rank, float *slot_scale,
+                         const BindBatch &batch, cudaStream_t s);

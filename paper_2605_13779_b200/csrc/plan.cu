@@ -1,0 +1,364 @@
+// Segment planner: token -> adapter segmentation of one batch.
+//
+// The paper's serving engine runs a batch that holds several adapters at once
+// (at most 64 distinct adapters in the GPU-batch tier, section "Scale Out:
+// Policy-Population Serving"); grouping the batch by adapter is the engine's
+// job.  This kernel produces the canonical stable grouping: work items (tokens,
+// or (token, k) pairs for MoE) ordered by key = slot (dense) or
+// expert*num_slots + slot (MoE), ties by item index; one segment per key.
+//
+// One CTA of 1024 threads.  The order is produced by a least-significant-digit
+// radix sort over the key bits with digits of at most 8 bits.  Every pass is
+// stable by construction and free of scheduling-dependent choices:
+//   - warp w owns the contiguous item range [w*R, (w+1)*R) and walks it in
+//     order, 32 items per step;
+//   - count walk: per-warp digit histogram (match_any groups equal digits, the
+//     group's lowest lane adds the group size);
+//   - the histogram is scanned bin-major, warp-minor: items of a smaller digit
+//     first, and inside one digit the items of a lower warp first;
+//   - scatter walk: position = bin base + warp offset + rank inside the step.
+// Items without an adapter get key = key_space (sorted last), so the active
+// items form a prefix.  Segment boundaries and the derived tile lists are then
+// found with block-wide prefix sums over contiguous runs per thread.
+#include "mint_device.cuh"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = 32;
+
+struct PlanParams {
+  TableDev tab;
+  const int64_t *ids;
+  const int32_t *expert_ids;
+  int32_t T, K, E;
+  int32_t P;
+  int32_t key_space;   // num_slots * max(E, 1); also the key of inactive items
+  int32_t npass;
+  int32_t digit_bits;
+  PlanOffsets off;
+  char *blob;
+  int32_t *status;
+};
+
+// Exclusive prefix sum of one int per thread over the block; returns the total.
+__device__ int block_exclusive_scan(int val, int *warp_tot /*[kWarps + 1]*/, int &total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = val;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int nb = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += nb;
+  }
+  __syncthreads();  // warp_tot may still be read from a previous call
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_tot[lane];
+    int winc = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int nb = __shfl_up_sync(0xffffffffu, winc, o);
+      if (lane >= o) winc += nb;
+    }
+    warp_tot[lane] = winc - w;
+    if (lane == 31) warp_tot[kWarps] = winc;
+  }
+  __syncthreads();
+  total = warp_tot[kWarps];
+  return warp_tot[warp] + inc - val;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
+  __shared__ int32_t hist[kWarps][256];
+  __shared__ int32_t bin_base[256];
+  __shared__ int warp_tot[kWarps + 1];
+  __shared__ int32_t counters[8];  // 0 inactive, 1 not resident, 2 first missing token, 3 bad expert,
+                                   // 4 first bad item, 5 max segment, 6 sum rank
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = p.P;
+  int32_t *hdr = reinterpret_cast<int32_t *>(p.blob + p.off.header);
+  int32_t *perm = reinterpret_cast<int32_t *>(p.blob + p.off.perm);
+  int32_t *seg_start = reinterpret_cast<int32_t *>(p.blob + p.off.seg_start);
+  int32_t *seg_key = reinterpret_cast<int32_t *>(p.blob + p.off.seg_key);
+  int32_t *seg_slot = reinterpret_cast<int32_t *>(p.blob + p.off.seg_slot);
+  int32_t *seg_expert = reinterpret_cast<int32_t *>(p.blob + p.off.seg_expert);
+  int32_t *key_a = reinterpret_cast<int32_t *>(p.blob + p.off.key_a);
+  int32_t *key_b = reinterpret_cast<int32_t *>(p.blob + p.off.key_b);
+  int32_t *idx_a = reinterpret_cast<int32_t *>(p.blob + p.off.idx_a);
+  int32_t *idx_b = reinterpret_cast<int32_t *>(p.blob + p.off.idx_b);
+
+  if (tid < 8) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff : 0;
+  __syncthreads();
+
+  // ---- keys: id -> slot through the table, (expert, slot) -> key ----------
+  for (int i = tid; i < P; i += kThreads) {
+    const int t = i / p.K;
+    const int64_t id = p.ids[t];
+    int32_t key = p.key_space;
+    if (id != -1) {
+      int32_t slot = -1;
+      if (id >= 0 && id < p.tab.catalog_size) slot = p.tab.id_to_slot[id];
+      if (slot < 0 || slot >= p.tab.num_slots) {
+        if (i == t * p.K) {
+          atomicAdd(&counters[1], 1);
+          atomicMin(&counters[2], t);
+        }
+      } else if (p.expert_ids != nullptr) {
+        const int32_t e = p.expert_ids[i];
+        if (e < 0 || e >= p.E) {
+          atomicAdd(&counters[3], 1);
+          atomicMin(&counters[4], i);
+        } else {
+          key = e * p.tab.num_slots + slot;
+        }
+      } else {
+        key = slot;
+      }
+    }
+    if (key == p.key_space) atomicAdd(&counters[0], 1);
+    key_a[i] = key;
+  }
+  __syncthreads();
+
+  // ---- stable LSD radix sort of (key, item index) ---------------------------
+  const int R = (((P + kWarps - 1) / kWarps + 31) / 32) * 32;  // items per warp, multiple of 32
+  const int w_begin = min(P, warp * R), w_end = min(P, (warp + 1) * R);
+  const int nbins = 1 << p.digit_bits;
+  for (int pass = 0; pass < p.npass; ++pass) {
+    const int32_t *kin = (pass & 1) ? key_b : key_a;
+    int32_t *kout = (pass & 1) ? key_a : key_b;
+    const int32_t *iin = (pass & 1) ? idx_b : idx_a;  // unused in pass 0 (index = position)
+    int32_t *iout = (pass == p.npass - 1) ? perm : ((pass & 1) ? idx_a : idx_b);
+    const int shift = pass * p.digit_bits;
+    const uint32_t mask = (uint32_t)nbins - 1u;
+
+    for (int i = tid; i < kWarps * 256; i += kThreads) (&hist[0][0])[i] = 0;
+    __syncthreads();
+    for (int base = w_begin; base < w_end; base += 32) {
+      const int i = base + lane;
+      const uint32_t dig = (i < w_end) ? (((uint32_t)kin[i] >> shift) & mask) : 0xFFFFFFFFu;
+      const uint32_t grp = __match_any_sync(0xffffffffu, dig);
+      if (i < w_end && lane == (__ffs(grp) - 1)) hist[warp][dig] += __popc(grp);
+      __syncwarp();
+    }
+    __syncthreads();
+    if (tid < nbins) {
+      int run = 0;
+      for (int w = 0; w < kWarps; ++w) {
+        const int c = hist[w][tid];
+        hist[w][tid] = run;
+        run += c;
+      }
+      bin_base[tid] = run;
+    }
+    __syncthreads();
+    if (warp == 0) {  // exclusive scan of the (up to 256) bin totals
+      int v[8], s = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int b = lane * 8 + q;
+        v[q] = (b < nbins) ? bin_base[b] : 0;
+        s += v[q];
+      }
+      int inc = s;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int nb = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += nb;
+      }
+      int run = inc - s;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const int b = lane * 8 + q;
+        if (b < nbins) bin_base[b] = run;
+        run += v[q];
+      }
+    }
+    __syncthreads();
+    for (int base = w_begin; base < w_end; base += 32) {
+      const int i = base + lane;
+      const bool live = i < w_end;
+      const int32_t key = live ? kin[i] : 0;
+      const uint32_t dig = live ? (((uint32_t)key >> shift) & mask) : 0xFFFFFFFFu;
+      const uint32_t grp = __match_any_sync(0xffffffffu, dig);
+      if (live) {
+        const int rank = __popc(grp & ((1u << lane) - 1u));
+        const int pos = bin_base[dig] + hist[warp][dig] + rank;
+        kout[pos] = key;
+        iout[pos] = (pass == 0) ? i : iin[i];
+      }
+      __syncwarp();
+      if (live && lane == (__ffs(grp) - 1)) hist[warp][dig] += __popc(grp);
+      __syncwarp();
+    }
+    __syncthreads();
+  }
+  const int32_t *skey = (p.npass & 1) ? key_b : key_a;  // keys in sorted order
+  const int n_active = P - counters[0];
+
+  // ---- segments: one per distinct key among the active prefix ----------------
+  const int run_len = (P + kThreads - 1) / kThreads;
+  const int r_begin = min(n_active, tid * run_len), r_end = min(n_active, (tid + 1) * run_len);
+  int heads = 0;
+  for (int i = r_begin; i < r_end; ++i) heads += (i == 0 || skey[i] != skey[i - 1]);
+  int S;
+  int seg = block_exclusive_scan(heads, warp_tot, S);
+  for (int i = r_begin; i < r_end; ++i) {
+    const int32_t k = skey[i];
+    if (i == 0 || k != skey[i - 1]) {
+      seg_start[seg] = i;
+      seg_key[seg] = k;
+      seg_slot[seg] = k % p.tab.num_slots;
+      seg_expert[seg] = k / p.tab.num_slots;
+      ++seg;
+    }
+  }
+  if (tid == 0) seg_start[S] = n_active;
+  __syncthreads();
+
+  for (int s = tid; s < S; s += kThreads) {
+    atomicMax(&counters[5], seg_start[s + 1] - seg_start[s]);
+    atomicAdd(&counters[6], p.tab.slot_rank[seg_slot[s]]);
+  }
+
+  // ---- derived tile lists: every segment cut into runs of at most G items ----
+  // Position i starts a tile of list g when (i - start of its segment) % G == 0.
+  int s0 = 0;
+  if (r_begin < r_end) {  // segment containing r_begin: last s with seg_start[s] <= r_begin
+    int lo = 0, hi = S - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (seg_start[mid] <= r_begin) lo = mid; else hi = mid - 1;
+    }
+    s0 = lo;
+  }
+  int tile_total[MINT_NUM_TILE_LISTS];
+#pragma unroll
+  for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
+    const int G = mint_tile_tokens(g);
+    int cnt = 0, s = s0;
+    for (int i = r_begin; i < r_end; ++i) {
+      while (i >= seg_start[s + 1]) ++s;
+      cnt += ((i - seg_start[s]) % G) == 0;
+    }
+    int pos = block_exclusive_scan(cnt, warp_tot, tile_total[g]);
+    int32_t *tseg = reinterpret_cast<int32_t *>(p.blob + p.off.tile_seg[g]);
+    int32_t *toff = reinterpret_cast<int32_t *>(p.blob + p.off.tile_off[g]);
+    s = s0;
+    for (int i = r_begin; i < r_end; ++i) {
+      while (i >= seg_start[s + 1]) ++s;
+      if (((i - seg_start[s]) % G) == 0) {
+        tseg[pos] = s;
+        toff[pos] = i;
+        ++pos;
+      }
+    }
+  }
+  __syncthreads();
+
+  if (tid == 0) {
+    hdr[PH_MAGIC] = MINT_PLAN_MAGIC;
+    hdr[PH_T] = p.T;
+    hdr[PH_K] = p.K;
+    hdr[PH_NUM_ITEMS] = P;
+    hdr[PH_NUM_SLOTS] = p.tab.num_slots;
+    hdr[PH_NUM_EXPERTS] = p.E;
+    hdr[PH_NUM_ACTIVE] = n_active;
+    hdr[PH_NUM_SEGMENTS] = S;
+    hdr[PH_MAX_SEGMENT] = counters[5];
+    hdr[PH_SUM_RANK] = counters[6];
+    hdr[PH_NOT_RESIDENT] = counters[1];
+    hdr[PH_BAD_EXPERT] = counters[3];
+    hdr[PH_GEN_LO] = p.tab.gen_lo;
+    hdr[PH_GEN_HI] = p.tab.gen_hi;
+    hdr[PH_NCHUNK0] = tile_total[0];
+    hdr[PH_NCHUNK1] = tile_total[1];
+    hdr[PH_NCHUNK2] = tile_total[2];
+    for (int w = PH_NCHUNK2 + 1; w < PH_WORDS; ++w) hdr[w] = 0;
+    if (counters[1] > 0) {
+      mint::report(p.status, MINT_ERR_NOT_RESIDENT, counters[2]);
+      if (p.status) atomicAdd(&p.status[1], counters[1]);
+    }
+    if (counters[3] > 0) mint::report(p.status, MINT_ERR_BAD_INDEX, counters[4]);
+  }
+}
+
+int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+PlanOffsets mint_plan_offsets(int64_t P) {
+  PlanOffsets o;
+  const int64_t n = (P > 0 ? P : 1);
+  int64_t cur = 0;
+  auto take = [&](int64_t count) {
+    int64_t at = cur;
+    cur = align_up(cur + count * 4, 256);
+    return at;
+  };
+  o.header = take(PH_WORDS);
+  o.perm = take(n);
+  o.seg_start = take(n + 1);
+  o.seg_key = take(n);
+  o.seg_slot = take(n);
+  o.seg_expert = take(n);
+  for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
+    o.tile_seg[g] = take(n);
+    o.tile_off[g] = take(n);
+  }
+  o.key_a = take(n);
+  o.key_b = take(n);
+  o.idx_a = take(n);
+  o.idx_b = take(n);
+  o.total = cur;
+  return o;
+}
+
+int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space) {
+  const int64_t G = mint_tile_tokens(g);
+  const int64_t max_segments = key_space < P ? key_space : P;
+  int64_t ub = P / G + max_segments;
+  return ub < P ? ub : P;
+}
+
+PlanView mint_plan_view(const void *plan_dev, int64_t P) {
+  const PlanOffsets o = mint_plan_offsets(P);
+  const char *b = static_cast<const char *>(plan_dev);
+  PlanView v;
+  v.header = reinterpret_cast<const int32_t *>(b + o.header);
+  v.perm = reinterpret_cast<const int32_t *>(b + o.perm);
+  v.seg_start = reinterpret_cast<const int32_t *>(b + o.seg_start);
+  v.seg_key = reinterpret_cast<const int32_t *>(b + o.seg_key);
+  v.seg_slot = reinterpret_cast<const int32_t *>(b + o.seg_slot);
+  v.seg_expert = reinterpret_cast<const int32_t *>(b + o.seg_expert);
+  for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
+    v.tile_seg[g] = reinterpret_cast<const int32_t *>(b + o.tile_seg[g]);
+    v.tile_off[g] = reinterpret_cast<const int32_t *>(b + o.tile_off[g]);
+  }
+  return v;
+}
+
+int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, const int32_t *expert_ids,
+                         int32_t K, int32_t num_experts, void *plan_dev, int32_t *status,
+                         cudaStream_t stream) {
+  PlanParams p;
+  p.tab = tab;
+  p.ids = ids;
+  p.expert_ids = expert_ids;
+  p.T = T;
+  p.K = K;
+  p.E = num_experts;
+  p.P = T * K;
+  p.key_space = tab.num_slots * (num_experts > 0 ? num_experts : 1);
+  int nbits = 1;
+  while ((1ll << nbits) <= (long long)p.key_space) ++nbits;  // key_space itself must fit
+  p.npass = (nbits + 7) / 8;
+  p.digit_bits = (nbits + p.npass - 1) / p.npass;
+  p.off = mint_plan_offsets(p.P);
+  p.blob = static_cast<char *>(plan_dev);
+  p.status = status;
+  plan_kernel<<<1, kThreads, 0, stream>>>(p);
+  return mint_check_cuda(cudaGetLastError(), "plan kernel launch");
+}

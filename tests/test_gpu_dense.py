@@ -1,0 +1,164 @@
+"""Dense shrink / expand / fused apply on the GPU against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_13779_b200 import synth
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def run_fused(case, y0_bits=None):
+    from paper_2605_13779_b200 import binding as mb, harness
+    dev = harness.upload_dense(case)
+    if y0_bits is not None:
+        dev.y = mb.bf16_from_bits(y0_bits)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    mb.mint_lora_apply_fused(dev.pool, dev.table, plan, dev.x, dev.y, dev.status)
+    torch.cuda.synchronize()
+    return harness.y_to_f64(dev.y), dev.status.cpu().numpy(), dev
+
+
+def run_unfused(case):
+    from paper_2605_13779_b200 import binding as mb, harness
+    dev = harness.upload_dense(case)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    v = torch.full((case.T, case.r_max), float("nan"), dtype=torch.float32, device="cuda")
+    mb.mint_lora_shrink(dev.pool, dev.table, plan, dev.x, dev.status, v=v)
+    mb.mint_lora_expand(dev.pool, dev.table, plan, v, dev.y, dev.status)
+    torch.cuda.synchronize()
+    return harness.y_to_f64(dev.y), v.cpu().numpy().astype(np.float64), dev.status.cpu().numpy()
+
+
+def check_case(case, what):
+    y_ref, v_ref, missing = parity.oracle_dense(case, want_v=True)
+    y_f, status, _ = run_fused(case)
+    assert status[0] == 0, status
+    parity.assert_close(y_f, y_ref, what + " fused")
+    y_u, v_u, status = run_unfused(case)
+    assert status[0] == 0, status
+    parity.assert_close(y_u, y_ref, what + " shrink+expand")
+    # shrink output is fully defined: zeros beyond the rank and for tokens without adapter
+    np.testing.assert_allclose(v_u, v_ref, rtol=2e-4, atol=2e-4 * max(1.0, np.abs(v_ref).max()))
+    assert (v_u[v_ref == 0] == 0).all()
+    # rows of tokens without an adapter are untouched bit for bit
+    none = case.ids < 0
+    if none.any():
+        np.testing.assert_array_equal(y_f[none], synth.bf16_bits_to_f64(case.y0)[none])
+    # the delta itself: same case with y0 = 0, where the 5e-3 bound bites on the update
+    zero = np.zeros_like(case.y0)
+    y_ref0, _, _ = parity.oracle_dense(case, y0=zero)
+    y_f0, _, _ = run_fused(case, y0_bits=zero)
+    parity.assert_close(y_f0, y_ref0, what + " fused, y0=0")
+
+
+def test_config1():
+    check_case(synth.config1(), "config1")
+
+
+@pytest.mark.parametrize("proj", list(synth.QWEN3_4B_PROJECTIONS))
+def test_config2_projection(proj):
+    batch = synth.config2_batch()
+    check_case(synth.config2_projection(batch, proj), f"config2/{proj}")
+
+
+def test_config3_reduced_lengths():
+    """Prefill segments at one eighth of the lengths (16..128 tokens per request)."""
+    batch = synth.config3_batch(len_lo=16, len_hi=128, tag="config3/small")
+    check_case(synth.config3_projection(batch, 5120, 5120, tag="config3/small"), "config3/small")
+
+
+def test_config3_non_contiguous_requests():
+    batch = synth.config3_batch(num_requests=12, len_lo=5, len_hi=70, rank=64, bijection=False,
+                                tag="config3/iid")
+    check_case(synth.config3_projection(batch, 1024, 2048, tag="config3/iid"), "config3/iid")
+
+
+def test_config5_full_size():
+    check_case(synth.config5(), "config5")
+
+
+@pytest.mark.parametrize("T,d,n,num_slots,ranks,r_max,p_none", [
+    (1, 64, 64, 1, [1], 1, 0.0),
+    (3, 8, 8, 2, [2, 1], 2, 0.0),
+    (37, 264, 520, 6, [1, 2, 3, 5, 7, 12], 12, 0.2),
+    (130, 1032, 776, 9, [1, 4, 8, 9, 16, 17, 31, 32, 3], 32, 0.1),
+    (64, 2048, 1024, 3, [64, 100, 128], 128, 0.0),
+    (300, 512, 512, 2, [4, 24], 24, 0.05),
+    (20, 4096, 72, 20, [8] * 20, 16, 0.0),
+])
+def test_ragged_shapes_and_ranks(T, d, n, num_slots, ranks, r_max, p_none):
+    case = synth.random_dense_case(f"gpu/ragged/{T}/{d}/{n}", T, d, n, num_slots, ranks, r_max, p_none=p_none)
+    check_case(case, f"ragged T={T} d={d} n={n}")
+
+
+def test_empty_batch_and_all_none():
+    from paper_2605_13779_b200 import binding as mb, harness
+    case = synth.random_dense_case("gpu/empty", 0, 64, 64, 2, [2, 2], 2)
+    y, status, _ = run_fused(case)
+    assert y.shape == (0, 64) and status[0] == 0
+    case = synth.random_dense_case("gpu/allnone", 19, 64, 64, 2, [2, 2], 2, p_none=1.0)
+    y, status, _ = run_fused(case)
+    np.testing.assert_array_equal(y, synth.bf16_bits_to_f64(case.y0))
+    assert status[0] == 0
+
+
+def test_rank_padding_is_never_read():
+    """Rank-r adapters in an r_max-wide slot with NaN padding equal the same
+    adapters in exact-size slots."""
+    wide = synth.random_dense_case("gpu/pad", 40, 256, 256, 3, [2, 3, 1], 8, p_none=0.0)
+    y_wide, status, _ = run_fused(wide)
+    assert status[0] == 0 and np.isfinite(y_wide).all()
+    tight = synth.DenseCase("gpu/pad/tight", wide.T, wide.d, wide.n, 3, wide.table, wide.ids,
+                            wide.A[:, :3].copy(), wide.B[:, :3].copy(), wide.x, wide.y0)
+    y_tight, _, _ = run_fused(tight)
+    np.testing.assert_array_equal(y_wide, y_tight)
+
+
+def test_mixed_batch_rows_equal_isolated_rows():
+    case = synth.config1()
+    y_mixed, _, _ = run_fused(case)
+    for a in range(4):
+        sel = np.nonzero(case.ids == a)[0]
+        iso = synth.DenseCase("iso", sel.size, case.d, case.n, case.r_max, case.table, case.ids[sel],
+                              case.A, case.B, case.x[sel], case.y0[sel])
+        y_iso, _, _ = run_fused(iso)
+        # same tokens, possibly tiled differently: equal to within one bf16 rounding of the sum
+        assert np.abs(y_iso - y_mixed[sel]).max() <= 2.0 ** -6
+
+
+def test_fused_is_deterministic():
+    case = synth.config2_projection(synth.config2_batch(), "o")
+    y1, _, _ = run_fused(case)
+    y2, _, _ = run_fused(case)
+    np.testing.assert_array_equal(y1, y2)
+
+
+def test_non_resident_tokens_are_left_untouched():
+    from paper_2605_13779_b200 import binding as mb
+    case = synth.config5(T=128, d=256, n=256, leave_unbound=2)
+    y_ref, _, missing = parity.oracle_dense(case)
+    y, status, _ = run_fused(case)
+    assert missing > 0 and status[0] == mb.MINT_ERR_NOT_RESIDENT and status[1] == missing
+    parity.assert_close(y, y_ref, "config5 with unbound ids")
+    gone = case.table.id_to_slot[case.ids] < 0
+    np.testing.assert_array_equal(y[gone], synth.bf16_bits_to_f64(case.y0)[gone])
+
+
+def test_strided_activations():
+    """x and y as column slices of wider buffers (row stride > width)."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    case = synth.random_dense_case("gpu/strided", 21, 128, 192, 3, [4, 4, 2], 4, p_none=0.1)
+    dev = harness.upload_dense(case)
+    xw = torch.zeros(case.T, 128 + 64, dtype=torch.bfloat16, device="cuda")
+    yw = torch.zeros(case.T, 192 + 8, dtype=torch.bfloat16, device="cuda")
+    xw[:, :128] = dev.x
+    yw[:, :192] = dev.y
+    yw[:, 192:] = 5.0
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    mb.mint_lora_apply_fused(dev.pool, dev.table, plan, xw[:, :128], yw[:, :192], dev.status)
+    torch.cuda.synchronize()
+    y_ref, _, _ = parity.oracle_dense(case)
+    parity.assert_close(harness.y_to_f64(yw[:, :192]), y_ref, "strided")
+    assert (yw[:, 192:] == 5.0).all()

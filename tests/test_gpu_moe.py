@@ -1,0 +1,102 @@
+"""MoE expert LoRA apply on the GPU against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_13779_b200 import synth
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def run_moe(case, weighted=False, y0_bits=None):
+    from paper_2605_13779_b200 import binding as mb, harness
+    dev = harness.upload_moe(case)
+    if y0_bits is not None:
+        dev.y = mb.bf16_from_bits(y0_bits)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status, expert_ids=dev.expert_ids, num_experts=case.E)
+    mb.mint_moe_lora_apply(dev.pool, dev.table, plan, dev.x, dev.y, dev.status, x_row=dev.x_row,
+                           pair_weight=dev.pair_weight if weighted else None)
+    torch.cuda.synchronize()
+    return harness.y_to_f64(dev.y), dev.status.cpu().numpy()
+
+
+def check_case(case, what):
+    for weighted in (False, True):
+        y_ref, _ = parity.oracle_moe(case, weighted=weighted)
+        y, status = run_moe(case, weighted=weighted)
+        assert status[0] == 0, status
+        parity.assert_close(y, y_ref, f"{what} weighted={weighted}")
+    zero = np.zeros_like(case.y0)
+    y_ref0, _ = parity.oracle_moe(case, y0=zero)
+    y0, _ = run_moe(case, y0_bits=zero)
+    parity.assert_close(y0, y_ref0, what + " y0=0")
+    none = np.repeat(case.ids < 0, case.K)
+    if none.any():
+        y, _ = run_moe(case)
+        np.testing.assert_array_equal(y[none], synth.bf16_bits_to_f64(case.y0)[none])
+
+
+@pytest.mark.parametrize("proj", ["gate", "down"])
+def test_config4_reduced_tokens(proj):
+    """30B-A3B shapes (hidden 2048, 128 experts, top-8, expert width 768, 16 rank-16
+    adapters) at T=512 tokens: 4096 pairs in about 1750 (expert, adapter) groups."""
+    batch = synth.config4_batch(T=512)
+    check_case(synth.config4_projection(batch, proj), f"config4/{proj}/T512")
+
+
+def test_config4_contiguous_requests_fewer_experts():
+    """Fewer experts and contiguous requests give long (expert, adapter) groups."""
+    batch = synth.config4_batch(T=768, E=8, K=2, num_slots=4, rank=16, contiguous_requests=True,
+                                tag="config4/long")
+    check_case(synth.config4_projection(batch, "gate", tag="config4/long"), "config4/long")
+
+
+@pytest.mark.parametrize("T,K,E,d,n,num_slots,rank,p_none", [
+    (1, 1, 1, 8, 8, 1, 1, 0.0),
+    (9, 2, 3, 72, 40, 2, 3, 0.2),
+    (65, 4, 16, 520, 264, 5, 8, 0.1),
+    (33, 8, 32, 256, 1024, 3, 24, 0.0),
+    (40, 2, 4, 768, 2048, 2, 1, 0.0),
+])
+def test_ragged_moe(T, K, E, d, n, num_slots, rank, p_none):
+    tag = f"gpu/moe/{T}/{K}/{E}"
+    batch = synth.config4_batch(T=T, E=E, K=K, num_slots=num_slots, rank=rank, p_none=p_none, tag=tag)
+    check_case(synth.config4_projection(batch, "gate", d=d, n=n, tag=tag), tag + "/gate")
+    check_case(synth.config4_projection(batch, "down", d=d, n=n, tag=tag), tag + "/down")
+
+
+def test_one_expert_top1_equals_dense_apply():
+    from paper_2605_13779_b200 import binding as mb, harness
+    batch = synth.config4_batch(T=50, E=1, K=1, num_slots=3, rank=8, tag="gpu/moe1")
+    case = synth.config4_projection(batch, "gate", d=256, n=128, tag="gpu/moe1")
+    y_moe, status = run_moe(case)
+    assert status[0] == 0
+    A_rd = np.ascontiguousarray(case.A[:, 0].transpose(0, 2, 1))      # [slot][r][d]
+    dense = synth.DenseCase("dense", case.T, case.d, case.n, case.r_max, case.table, case.ids, A_rd,
+                            np.ascontiguousarray(case.B[:, 0]), case.x, case.y0)
+    dev = harness.upload_dense(dense)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    mb.mint_lora_apply_fused(dev.pool, dev.table, plan, dev.x, dev.y, dev.status)
+    y_dense = harness.y_to_f64(dev.y)
+    assert np.abs(y_moe - y_dense).max() <= 2.0 ** -6
+
+
+def test_bad_row_index_is_reported_and_skipped():
+    from paper_2605_13779_b200 import binding as mb, harness
+    batch = synth.config4_batch(T=8, E=2, K=2, num_slots=2, rank=2, tag="gpu/moebad")
+    case = synth.config4_projection(batch, "gate", d=64, n=64, tag="gpu/moebad")
+    dev = harness.upload_moe(case)
+    rows = case.x_row.copy()
+    rows[5] = 10_000
+    x_row = torch.from_numpy(rows).cuda()
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status, expert_ids=dev.expert_ids, num_experts=case.E)
+    mb.mint_moe_lora_apply(dev.pool, dev.table, plan, dev.x, dev.y, dev.status, x_row=x_row)
+    torch.cuda.synchronize()
+    status = dev.status.cpu().numpy()
+    assert status[0] == mb.MINT_ERR_BAD_INDEX and status[2] == 5
+    y = harness.y_to_f64(dev.y)
+    np.testing.assert_array_equal(y[5], synth.bf16_bits_to_f64(case.y0)[5])
+    y_ref, _ = parity.oracle_moe(case)
+    keep = np.arange(16) != 5
+    parity.assert_close(y[keep], y_ref[keep], "other pairs")
