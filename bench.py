@@ -96,7 +96,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -156,7 +156,7 @@ def oracle_layer_seconds(wl, max_seconds: float = 12.0):
                 oracle.lora_apply(c.ids, t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B, c.x, c.y0)
         t_total += time.perf_counter() - t0
         n_layers += 1
-        if t_total >= max_seconds or n_layers >= 8:
+        if t_total >= max_seconds or n_layers >= 2000:
             break
     per_layer = t_total / n_layers
     return wl["T"] / per_layer, threads, f"{n_layers} layer(s) of the workload ({len(wl['cases'])} projections each, all {wl['T']} tokens), {t_total:.1f} s"
@@ -234,15 +234,37 @@ def run_gpu(args):
     def enqueue_plan():
         mb.mint_lora_plan(table, ids, status, expert_ids=expert_ids, num_experts=E, plan=plan)
 
-    def enqueue_applies():
+    # call grouping: "none" = one fused call per projection; "stage" = projections that can run at the
+    # same point of a transformer layer share a call (q,k,v | o | gate,up | down); "layer" = one call per layer
+    ncase = len(wl["cases"])
+    if moe or args.grouping == "none" or ncase == 1:
+        groups_idx = [[i] for i in range(ncase)]
+    elif args.grouping == "layer":
+        groups_idx = [list(range(ncase))]
+    else:
+        groups_idx = [[0, 1, 2], [3], [4, 5], [6]] if ncase == 7 else [[i] for i in range(ncase)]
+    workspaces = None if moe else [mb.new_workspace(dv.pool, T) for dv in base]
+    groups = []
+    if not moe:
         for row in layers:
-            for ci, (pool, x, y) in enumerate(row):
-                if moe:
-                    mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row)
-                else:
-                    mb.mint_lora_apply_fused(pool, table, plan, x, y, status)
+            groups.append([mb.ApplyGroup([(row[i][0], row[i][1], row[i][2], workspaces[i]) for i in g])
+                           for g in groups_idx])
 
-    launches_per_step = 1 + L * len(wl["cases"])
+    def enqueue_layer(li):
+        if moe:
+            for ci, (pool, x, y) in enumerate(layers[li]):
+                mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row)
+        else:
+            for grp in groups[li]:
+                mb.mint_lora_apply_fused_grouped(grp, table, plan, status)
+
+    def enqueue_applies():
+        for li in range(L):
+            enqueue_layer(li)
+
+    kernels_per_call = 1 if moe else 2          # the dense fused call is a shrink and an expand launch
+    calls_per_layer = len(groups_idx)
+    launches_per_step = 1 + L * calls_per_layer * kernels_per_call
 
     # warm-up outside any graph (first launches load the module), then capture
     enqueue_plan()
@@ -291,6 +313,14 @@ def run_gpu(args):
     ms_step = ms_total / args.steps
     value = world * T * L / (ms_step * 1e-3)
 
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_run": True, "workload": wl["name"], "layers": L, "ms_per_step": ms_step,
+                              "us_per_layer": ms_step * 1e3 / L, "grouping": args.grouping,
+                              "layer_GBps": layer_bytes / (ms_step * 1e-3 / L) / 1e9,
+                              "avg_apply_call_us": ms_apply * 1e3 / args.steps / (L * calls_per_layer)}))
+        return
+
     # ---- end to end through the C ABI with host buffers --------------------------
     # Per step: ids, every x and every y0 come from pinned host memory, the plan and
     # all applies run, and every updated y goes back to pinned host memory.
@@ -310,11 +340,8 @@ def run_gpu(args):
                 y.copy_(host_y[li][ci], non_blocking=True)
         enqueue_plan()
         for li in range(e2e_layers):
+            enqueue_layer(li)
             for ci, (pool, x, y) in enumerate(layers[li]):
-                if moe:
-                    mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row)
-                else:
-                    mb.mint_lora_apply_fused(pool, table, plan, x, y, status)
                 host_y[li][ci].copy_(y, non_blocking=True)
 
     with torch.cuda.stream(stream):
@@ -345,11 +372,13 @@ def run_gpu(args):
         peak, peak_src = json.load(open(peaks_path))["hbm_gbs"], "measured (MEASURED_PEAKS.json hbm_gbs)"
     else:
         peak, peak_src = 6650.0, "fallback"
-    n_apply = L * len(wl["cases"])
+    # the apply is a shrink launch and an expand launch that overlap (programmatic dependent launch),
+    # so the roofline unit is the pair: bytes of one call / time of one call
+    n_apply = L * calls_per_layer
     avg_launch_s = ms_apply * 1e-3 / args.steps / n_apply
-    avg_launch_bytes = layer_bytes / len(wl["cases"])
+    avg_launch_bytes = layer_bytes / calls_per_layer
     achieved = avg_launch_bytes / avg_launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "moe_kernel" if moe else "fused_kernel",
+    roofline = {"bound": "hbm", "kernel": "moe_kernel" if moe else "shrink_stream_kernel+expand_stream_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_8TBps": achieved / 8000.0, "peak_source": peak_src,
                 "bytes_per_launch": avg_launch_bytes, "avg_launch_us": avg_launch_s * 1e6,
@@ -365,6 +394,7 @@ def run_gpu(args):
         "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic (seeded)",
         "config": {"workload": wl["name"], "layers_per_step": L, "tokens": T,
                    "l2": f"inputs larger than L2: every layer has its own pool/x/y, {layer_bytes * L / 1e6:.0f} MB algorithmic bytes per step",
+                   "grouping": args.grouping, "calls_per_layer": calls_per_layer,
                    "timing": "CUDA graph of plan + all applies, CUDA events on the launching stream"},
         "us_per_layer": ms_step * 1e3 / L,
         "layer_bytes": layer_bytes,
@@ -384,11 +414,15 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--layers", type=int, default=0, help="layers per step (0 = the workload's own)")
+    ap.add_argument("--grouping", default="stage", choices=["none", "stage", "layer"],
+                    help="how the projections of a layer are grouped into fused calls")
+    ap.add_argument("--profile", action="store_true",
+                    help="device-timed part only (no end-to-end leg, no CPU oracle): the command profilers wrap")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

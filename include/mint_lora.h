@@ -196,15 +196,39 @@ int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table *table, co
                          int32_t T, const float *v_dev, void *y_dev, int64_t ldy,
                          int32_t *status_dev, mint_stream_t stream);
 
-/* ---- fused apply: shrink + expand in one launch, v never leaves the chip ---
+/* ---- fused apply: shrink + expand in one call -----------------------------------
  * Same result as shrink followed by expand (fp32 accumulation, summation order
- * may differ).  workspace_dev may be NULL when mint_lora_apply_workspace_bytes
- * returns 0 for the pool and T.                                              */
+ * may differ).  The shrink result never goes to HBM as a tensor of its own: it
+ * crosses from the shrink stage to the expand stage through workspace_dev, a
+ * few KB per tile that stay in L2.  workspace_dev: at least
+ * mint_lora_apply_workspace_bytes(pool, T) bytes, 256-byte aligned, ZERO-FILLED
+ * by the caller before its first use; every call leaves it ready for the next
+ * one.  Calls that share a workspace must be ordered on one stream.           */
 size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T);
 int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table,
                               const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
                               void *y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes,
                               int32_t *status_dev, mint_stream_t stream);
+
+/* Grouped form: the fused apply of up to MINT_MAX_GROUP projections that share
+ * one plan (for instance q, k and v, which read the same x; or gate and up), in
+ * one pair of launches.  An adapter's target modules come as a set (the paper's
+ * policy record lists rank and target modules), so one step applies the same
+ * batch plan to every targeted projection.  Each item has its own pool, x, y
+ * and workspace (rules as above); items must not alias each other's y.        */
+#define MINT_MAX_GROUP 8
+typedef struct {
+  const mint_pool *pool;
+  const void *x_dev;
+  int64_t ldx;
+  void *y_dev;
+  int64_t ldy;
+  void *workspace_dev;
+  size_t workspace_bytes;
+} mint_apply_item;
+int32_t mint_lora_apply_fused_grouped(const mint_apply_item *items, int32_t count,
+                                      const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                      int32_t *status_dev, mint_stream_t stream);
 
 /* ---- MoE expert LoRA apply -------------------------------------------------
  * Per-expert LoRA tensors keyed by expert id (paper, "Scale Up", Megatron

@@ -40,7 +40,7 @@ EXPORTS = [
     "mint_slot_table_evict", "mint_slot_table_destroy", "mint_slot_table_generation",
     "mint_lora_plan_bytes", "mint_lora_plan_layout", "mint_lora_plan", "mint_plan_fetch_summary",
     "mint_lora_shrink", "mint_lora_expand",
-    "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused",
+    "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
 ]
 
@@ -55,6 +55,15 @@ class PoolDesc(ctypes.Structure):
     _fields_ = [("d", ctypes.c_int32), ("n", ctypes.c_int32), ("r_max", ctypes.c_int32),
                 ("num_slots", ctypes.c_int32), ("num_experts", ctypes.c_int32),
                 ("layout", ctypes.c_int32), ("A_dev", ctypes.c_void_p), ("B_dev", ctypes.c_void_p)]
+
+
+class ApplyItem(ctypes.Structure):
+    _fields_ = [("pool", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("y_dev", ctypes.c_void_p), ("ldy", ctypes.c_int64), ("workspace_dev", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+MINT_MAX_GROUP = 8
 
 
 class PlanLayout(ctypes.Structure):
@@ -105,6 +114,7 @@ def load_library() -> ctypes.CDLL:
         "mint_lora_expand": (i32, [vp, vp, vp, i32, vp, vp, i64, vp, vp]),
         "mint_lora_apply_workspace_bytes": (sz, [vp, i32]),
         "mint_lora_apply_fused": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, sz, vp, vp]),
+        "mint_lora_apply_fused_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
     }
@@ -311,15 +321,44 @@ def mint_lora_apply_workspace_bytes(pool: Pool, T: int) -> int:
     return int(load_library().mint_lora_apply_workspace_bytes(pool.handle, T))
 
 
+def new_workspace(pool: Pool, T: int, device="cuda") -> torch.Tensor:
+    """Zero-filled workspace of the fused apply for one projection (the library
+    keeps it zero where it must be between calls)."""
+    nbytes = max(256, mint_lora_apply_workspace_bytes(pool, T))
+    return torch.zeros(nbytes, dtype=torch.uint8, device=device)
+
+
+def _ld(t: torch.Tensor, width: int) -> int:
+    return t.stride(0) if t.dim() == 2 and t.shape[0] > 0 else width
+
+
 def mint_lora_apply_fused(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
                           status: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    if workspace is None:
+        workspace = new_workspace(pool, plan.T, x.device)
     _check(load_library().mint_lora_apply_fused(
-        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x),
-        x.stride(0) if x.dim() == 2 and x.shape[0] > 0 else pool.d, _ptr(y),
-        y.stride(0) if y.dim() == 2 and y.shape[0] > 0 else pool.n,
-        _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
-        _ptr(status), _stream()))
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(y), _ld(y, pool.n),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
     return y
+
+
+class ApplyGroup:
+    """Up to MINT_MAX_GROUP (pool, x, y, workspace) items sharing one plan, marshalled once."""
+
+    def __init__(self, items):
+        assert 1 <= len(items) <= MINT_MAX_GROUP
+        self.keep = items
+        arr = (ApplyItem * len(items))()
+        for i, (pool, x, y, ws) in enumerate(items):
+            arr[i] = ApplyItem(pool.handle, _ptr(x), _ld(x, pool.d), _ptr(y), _ld(y, pool.n), _ptr(ws),
+                               ws.numel() * ws.element_size())
+        self.array = arr
+        self.count = len(items)
+
+
+def mint_lora_apply_fused_grouped(group: ApplyGroup, table: SlotTable, plan: Plan, status: torch.Tensor):
+    _check(load_library().mint_lora_apply_fused_grouped(group.array, group.count, table.handle,
+                                                        _ptr(plan.blob), plan.T, _ptr(status), _stream()))
 
 
 def mint_moe_lora_apply_workspace_bytes(pool: Pool, T: int, K: int) -> int:

@@ -470,31 +470,76 @@ extern "C" int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table
 }
 
 extern "C" size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T) {
-  (void)pool;
-  (void)T;
-  return 0;
+  if (!pool || T < 0) return 0;
+  return mint_stream_workspace_bytes(T, pool->desc.num_slots, pool->desc.r_max);
+}
+
+static int32_t fill_item(const mint_apply_item &it, const mint_slot_table *table, const void *plan_dev, int32_t T,
+                         int32_t *status_dev, bool need_ws, DenseArgs &a, const char *who) {
+  int32_t st = check_dense(it.pool, table, plan_dev, T, who);
+  if (st) return st;
+  if ((st = check_act(it.x_dev, it.ldx, it.pool->desc.d, "x_dev", who))) return st;
+  if ((st = check_act(it.y_dev, it.ldy, it.pool->desc.n, "y_dev", who))) return st;
+  if (need_ws) {
+    const size_t need = mint_lora_apply_workspace_bytes(it.pool, T);
+    if (!it.workspace_dev || it.workspace_bytes < need)
+      return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu", who, it.workspace_bytes, need);
+    if (reinterpret_cast<uintptr_t>(it.workspace_dev) & 255u)
+      return mint_fail(MINT_ERR_MISALIGNED, "%s: workspace must be 256-byte aligned", who);
+  }
+  a = dense_args(it.pool, T);
+  a.x = static_cast<const uint16_t *>(it.x_dev);
+  a.ldx = it.ldx;
+  a.y = static_cast<uint16_t *>(it.y_dev);
+  a.ldy = it.ldy;
+  a.status = status_dev;
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_lora_apply_fused_grouped(const mint_apply_item *items, int32_t count,
+                                                 const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                                 int32_t *status_dev, mint_stream_t stream) {
+  if (!items || count < 1 || count > MINT_MAX_GROUP)
+    return mint_fail(MINT_ERR_INVALID_ARG, "apply_fused_grouped: count=%d (1..%d)", count, MINT_MAX_GROUP);
+  if (!table || !status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "apply_fused_grouped: null argument");
+  if (T == 0) {
+    for (int i = 0; i < count; ++i) {
+      int32_t st = check_dense(items[i].pool, table, plan_dev, T, "apply_fused_grouped");
+      if (st) return st;
+    }
+    return MINT_OK;
+  }
+  const bool stream_path = mint_stream_supported(table->max_rank);
+  DenseArgs args[MINT_MAX_GROUP];
+  void *ws[MINT_MAX_GROUP];
+  for (int i = 0; i < count; ++i) {
+    int32_t st = fill_item(items[i], table, plan_dev, T, status_dev, stream_path, args[i], "apply_fused_grouped");
+    if (st) return st;
+    ws[i] = items[i].workspace_dev;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (stream_path) return mint_launch_stream(args, count, table_dev(table), plan_dev, ws, s);
+  // ranks above the streamed path's limit: one cluster kernel per projection
+  for (int i = 0; i < count; ++i) {
+    int32_t st = mint_launch_fused(args[i], table_dev(table), plan_dev, s);
+    if (st) return st;
+  }
+  return MINT_OK;
 }
 
 extern "C" int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
                                          int32_t T, const void *x_dev, int64_t ldx, void *y_dev, int64_t ldy,
                                          void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
                                          mint_stream_t stream) {
-  int32_t st = check_dense(pool, table, plan_dev, T, "apply_fused");
-  if (st) return st;
-  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "apply_fused: null status_dev");
-  if (T == 0) return MINT_OK;
-  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "apply_fused"))) return st;
-  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", "apply_fused"))) return st;
-  const size_t need = mint_lora_apply_workspace_bytes(pool, T);
-  if (need > 0 && (!workspace_dev || workspace_bytes < need))
-    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "apply_fused: workspace %zu < %zu", workspace_bytes, need);
-  DenseArgs a = dense_args(pool, T);
-  a.x = static_cast<const uint16_t *>(x_dev);
-  a.ldx = ldx;
-  a.y = static_cast<uint16_t *>(y_dev);
-  a.ldy = ldy;
-  a.status = status_dev;
-  return mint_launch_fused(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
+  mint_apply_item it;
+  it.pool = pool;
+  it.x_dev = x_dev;
+  it.ldx = ldx;
+  it.y_dev = y_dev;
+  it.ldy = ldy;
+  it.workspace_dev = workspace_dev;
+  it.workspace_bytes = workspace_bytes;
+  return mint_lora_apply_fused_grouped(&it, 1, table, plan_dev, T, status_dev, stream);
 }
 
 // ---------------------------------------------------------------------------

@@ -124,6 +124,13 @@ int32_t mint_launch_shrink(const DenseArgs &a, const TableDev &tab, const void *
 int32_t mint_launch_expand(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
 int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
 
+// Streamed fused path (bulk-copy pipelines + warp MMA) for ranks up to 64: one
+// shrink and one expand launch cover up to 8 projections that share a plan.
+bool mint_stream_supported(int32_t max_bound_rank);
+size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);
+int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                           void *const *workspaces, cudaStream_t s);
+
 struct MoEArgs {
   const uint16_t *A;   // [slot][E][d][r_max]
   const uint16_t *B;   // [slot][E][r_max][n]

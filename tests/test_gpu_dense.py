@@ -162,3 +162,34 @@ def test_strided_activations():
     y_ref, _, _ = parity.oracle_dense(case)
     parity.assert_close(harness.y_to_f64(yw[:, :192]), y_ref, "strided")
     assert (yw[:, 192:] == 5.0).all()
+
+
+def test_grouped_call_equals_separate_calls():
+    """q, k and v read the same x: one grouped call gives the same bits as three calls."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    batch = synth.config2_batch()
+    cases = [synth.config2_projection(batch, p) for p in ("q", "k", "v")]
+    devs = [harness.upload_dense(c) for c in cases]
+    table, status = devs[0].table, devs[0].status
+    plan = mb.mint_lora_plan(table, devs[0].ids, status)
+    x = devs[0].x
+    sep = []
+    for dv in devs:
+        y = dv.y.clone()
+        mb.mint_lora_apply_fused(dv.pool, table, plan, x, y, status)
+        sep.append(y)
+    ws = [mb.new_workspace(dv.pool, batch.T) for dv in devs]
+    group = mb.ApplyGroup([(dv.pool, x, dv.y, w) for dv, w in zip(devs, ws)])
+    mb.mint_lora_apply_fused_grouped(group, table, plan, status)
+    mb.mint_lora_apply_fused_grouped(group, table, plan, status)     # workspaces are reusable as they are
+    torch.cuda.synchronize()
+    assert status[0].item() == 0
+    for dv, c, y1 in zip(devs, cases, sep):
+        once = harness.y_to_f64(y1)
+        c2 = synth.DenseCase(c.name, c.T, c.d, c.n, c.r_max, c.table, c.ids, c.A, c.B, cases[0].x, c.y0)
+        y_ref, _, _ = parity.oracle_dense(c2)
+        parity.assert_close(once, y_ref, c.name)
+        # second application on top of the first: y0 + 2 delta within two roundings
+        twice = harness.y_to_f64(dv.y)
+        delta = y_ref - synth.bf16_bits_to_f64(c.y0)
+        assert np.abs(twice - (y_ref + delta)).max() <= 6e-2
