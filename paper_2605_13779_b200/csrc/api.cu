@@ -27,6 +27,23 @@ int32_t mint_check_cuda(cudaError_t e, const char *what) {
   return mint_fail(MINT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+int32_t mint_device_lanes(int32_t *lanes_out) {
+  static int cached[64] = {0};
+  int dev = 0;
+  int32_t st = mint_check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (st) return st;
+  if (dev < 0 || dev >= 64) return mint_fail(MINT_ERR_UNSUPPORTED, "device ordinal %d", dev);
+  if (cached[dev] == 0) {
+    int sms = 0;
+    st = mint_check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
+    if (st) return st;
+    if (sms < 1) return mint_fail(MINT_ERR_CUDA, "device reports %d SMs", sms);
+    cached[dev] = sms > MINT_MAX_LANES ? MINT_MAX_LANES : sms;
+  }
+  *lanes_out = cached[dev];
+  return MINT_OK;
+}
+
 extern "C" const char *mint_last_error_string(void) { return g_err; }
 
 extern "C" const char *mint_status_name(int32_t s) {
@@ -336,7 +353,7 @@ static int32_t check_plan_shape(int32_t T, int32_t K, int32_t num_slots, int32_t
 
 extern "C" size_t mint_lora_plan_bytes(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts) {
   if (check_plan_shape(T, K, num_slots, num_experts, "plan_bytes")) return 0;
-  return (size_t)mint_plan_offsets((int64_t)T * K).total;
+  return (size_t)mint_plan_offsets((int64_t)T * K, (int64_t)num_slots * (num_experts > 0 ? num_experts : 1)).total;
 }
 
 extern "C" int32_t mint_lora_plan_layout(int32_t T, int32_t K, int32_t num_slots, int32_t num_experts,
@@ -344,7 +361,7 @@ extern "C" int32_t mint_lora_plan_layout(int32_t T, int32_t K, int32_t num_slots
   if (!out) return mint_fail(MINT_ERR_INVALID_ARG, "plan_layout: null out");
   int32_t st = check_plan_shape(T, K, num_slots, num_experts, "plan_layout");
   if (st) return st;
-  const PlanOffsets o = mint_plan_offsets((int64_t)T * K);
+  const PlanOffsets o = mint_plan_offsets((int64_t)T * K, (int64_t)num_slots * (num_experts > 0 ? num_experts : 1));
   out->total_bytes = o.total;
   out->header_off = o.header;
   out->perm_off = o.perm;
@@ -366,11 +383,13 @@ extern "C" int32_t mint_lora_plan(const mint_slot_table *table, const int64_t *i
   if (expert_ids_dev != nullptr && num_experts < 1)
     return mint_fail(MINT_ERR_INVALID_ARG, "plan: a MoE plan needs num_experts >= 1");
   if (!aligned16(plan_dev)) return mint_fail(MINT_ERR_MISALIGNED, "plan: plan_dev must be 16-byte aligned");
-  const size_t need = (size_t)mint_plan_offsets((int64_t)T * K).total;
+  const size_t need = (size_t)mint_plan_offsets((int64_t)T * K, (int64_t)table->num_slots * (num_experts > 0 ? num_experts : 1)).total;
   if (plan_bytes < need)
     return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "plan: plan_bytes=%zu < %zu", plan_bytes, need);
-  return mint_launch_plan(table_dev(table), ids_dev, T, expert_ids_dev, K, num_experts, plan_dev, status_dev,
-                          static_cast<cudaStream_t>(stream));
+  int32_t lanes = 0;
+  if ((st = mint_device_lanes(&lanes))) return st;
+  return mint_launch_plan(table_dev(table), ids_dev, T, expert_ids_dev, K, num_experts, lanes, plan_dev,
+                          status_dev, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int32_t mint_plan_fetch_summary(const void *plan_dev, mint_plan_summary *out, mint_stream_t stream) {

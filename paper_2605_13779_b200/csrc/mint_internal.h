@@ -29,13 +29,33 @@ enum {
   PH_GEN_HI,
   PH_NCHUNK0,   // number of tiles in list g (MINT_NUM_TILE_LISTS entries)
   PH_NCHUNK1,
-  PH_NCHUNK2,
+  PH_LANES,     // number of cost lanes G the lane tables were cut for
+  PH_ROWS_SHRINK,  // sum over list-1 tiles of (rank + len)
+  PH_ROWS_EXPAND,  // sum over list-1 tiles of (rank + 2 len)
   PH_WORDS = 32
 };
-#define MINT_PLAN_MAGIC 0x4D4C5031  // "MLP1"
-#define MINT_NUM_TILE_LISTS 3
-// Tile list g cuts every segment into runs of at most kTileTokens[g] items.
-__host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : (g == 1 ? 32 : 128); }
+#define MINT_PLAN_MAGIC 0x4D4C5032  // "MLP2"
+#define MINT_NUM_TILE_LISTS 2
+#define MINT_MAX_LANES 256
+// Tile list g cuts every segment into runs of at most mint_tile_tokens(g) items.
+__host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 32; }
+
+// One tile of list 1 with everything a streaming kernel needs to start on it:
+// no dependent lookups through segment or slot arrays.  rank and scale are the
+// slot's values when the plan was made (the plan's generation guards them).
+// rows_shrink / rows_expand are the exclusive prefix sums, over tiles, of
+// (rank + len) and (rank + 2 len): the row counts whose product with a
+// projection's width gives the bytes the shrink and the expand stream.
+struct __align__(16) TileDesc {
+  int32_t off;     // first position of the tile in perm
+  int32_t len;     // 1..32 items
+  int32_t slot;
+  int32_t expert;  // 0 for dense plans
+  int32_t rank;
+  float scale;
+  int32_t rows_shrink;
+  int32_t rows_expand;
+};
 
 // Byte offsets of every array inside the plan blob (host-computed, passed by value).
 struct PlanOffsets {
@@ -47,10 +67,13 @@ struct PlanOffsets {
   int64_t seg_expert;  // int32[P]
   int64_t tile_seg[MINT_NUM_TILE_LISTS];  // int32[P]  segment of tile c
   int64_t tile_off[MINT_NUM_TILE_LISTS];  // int32[P]  first position (in perm) of tile c
+  int64_t tile_desc;   // TileDesc[tile upper bound of list 1]
+  int64_t lane_shrink; // int32[MINT_MAX_LANES + 1]  tile holding the start of cost lane j (shrink rows)
+  int64_t lane_expand; // int32[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
   int64_t total;
 };
-PlanOffsets mint_plan_offsets(int64_t P);
+PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space);
 // Upper bound on the number of tiles of list g, computable without reading the plan.
 int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space);
 
@@ -64,8 +87,13 @@ struct PlanView {
   const int32_t *seg_expert;
   const int32_t *tile_seg[MINT_NUM_TILE_LISTS];
   const int32_t *tile_off[MINT_NUM_TILE_LISTS];
+  const TileDesc *tile_desc;
+  const int32_t *lane_shrink;
+  const int32_t *lane_expand;
 };
-PlanView mint_plan_view(const void *plan_dev, int64_t P);
+PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space);
+// Number of cost lanes plans are cut for on the current device (its SM count).
+int32_t mint_device_lanes(int32_t *lanes_out);
 
 // ---- host handles ----------------------------------------------------------
 struct mint_pool {
@@ -105,7 +133,7 @@ struct TableDev {
 };
 
 int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, const int32_t *expert_ids,
-                         int32_t K, int32_t num_experts, void *plan_dev, int32_t *status,
+                         int32_t K, int32_t num_experts, int32_t lanes, void *plan_dev, int32_t *status,
                          cudaStream_t stream);
 
 struct DenseArgs {

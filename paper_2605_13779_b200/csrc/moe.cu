@@ -73,6 +73,6 @@ int32_t mint_launch_moe(const MoEArgs &a, const TableDev &tab, const void *plan_
   const int64_t P = (int64_t)a.T * a.K;
   const int64_t ub = mint_tile_upper_bound(0, P, (int64_t)tab.num_slots * a.num_experts);
   if (ub == 0) return MINT_OK;
-  moe_kernel<<<(unsigned)ub, kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, P));
+  moe_kernel<<<(unsigned)ub, kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, P, (int64_t)tab.num_slots * a.num_experts));
   return mint_check_cuda(cudaGetLastError(), "moe kernel launch");
 }

@@ -36,6 +36,7 @@ struct PlanParams {
   int32_t key_space;   // num_slots * max(E, 1); also the key of inactive items
   int32_t npass;
   int32_t digit_bits;
+  int32_t lanes;       // cost lanes G of the lane tables
   PlanOffsets off;
   char *blob;
   int32_t *status;
@@ -258,6 +259,66 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   }
   __syncthreads();
 
+  // ---- list-1 tile descriptors, their row prefix sums and the lane tables ----
+  // A streaming kernel splits the rows x columns area of its work evenly over
+  // G lanes; lane j starts inside the tile t with rows[t]*G <= j*rows_total,
+  // which does not depend on the projection's width, so it is tabulated here.
+  TileDesc *desc = reinterpret_cast<TileDesc *>(p.blob + p.off.tile_desc);
+  int32_t *lane_tab[2] = {reinterpret_cast<int32_t *>(p.blob + p.off.lane_shrink),
+                          reinterpret_cast<int32_t *>(p.blob + p.off.lane_expand)};
+  int rows_total[2];
+  {
+    const int32_t *tseg = reinterpret_cast<const int32_t *>(p.blob + p.off.tile_seg[1]);
+    const int32_t *toff = reinterpret_cast<const int32_t *>(p.blob + p.off.tile_off[1]);
+    const int ntile = tile_total[1];
+    const int per = (ntile + kThreads - 1) / kThreads;
+    const int c_begin = min(ntile, tid * per), c_end = min(ntile, (tid + 1) * per);
+    int sum_s = 0, sum_e = 0;
+    for (int c = c_begin; c < c_end; ++c) {
+      const int sg = tseg[c];
+      const int len = min(mint_tile_tokens(1), seg_start[sg + 1] - toff[c]);
+      const int r = p.tab.slot_rank[seg_slot[sg]];
+      sum_s += r + len;
+      sum_e += r + 2 * len;
+    }
+    int run_s = block_exclusive_scan(sum_s, warp_tot, rows_total[0]);
+    int run_e = block_exclusive_scan(sum_e, warp_tot, rows_total[1]);
+    for (int c = c_begin; c < c_end; ++c) {
+      const int sg = tseg[c];
+      const int slot = seg_slot[sg];
+      TileDesc dsc;
+      dsc.off = toff[c];
+      dsc.len = min(mint_tile_tokens(1), seg_start[sg + 1] - toff[c]);
+      dsc.slot = slot;
+      dsc.expert = seg_expert[sg];
+      dsc.rank = p.tab.slot_rank[slot];
+      dsc.scale = p.tab.slot_scale[slot];
+      dsc.rows_shrink = run_s;
+      dsc.rows_expand = run_e;
+      desc[c] = dsc;
+      // lanes whose start falls inside this tile: rows[c]*G <= j*total < rows[c+1]*G
+      const int64_t G = p.lanes;
+      const int begin[2] = {run_s, run_e};
+      const int end[2] = {run_s + dsc.rank + dsc.len, run_e + dsc.rank + 2 * dsc.len};
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int64_t tot = rows_total[q];
+        const int64_t j_lo = (begin[q] * G + tot - 1) / tot;
+        const int64_t j_hi = (end[q] * G + tot - 1) / tot;   // exclusive
+        for (int64_t j = j_lo; j < j_hi && j < G; ++j) lane_tab[q][j] = c;
+      }
+      run_s = end[0];
+      run_e = end[1];
+    }
+    if (tid == 0) {
+      lane_tab[0][p.lanes] = ntile;
+      lane_tab[1][p.lanes] = ntile;
+    }
+    if (ntile == 0)
+      for (int j = tid; j < p.lanes; j += kThreads) lane_tab[0][j] = lane_tab[1][j] = 0;
+  }
+  __syncthreads();
+
   if (tid == 0) {
     hdr[PH_MAGIC] = MINT_PLAN_MAGIC;
     hdr[PH_T] = p.T;
@@ -275,8 +336,10 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     hdr[PH_GEN_HI] = p.tab.gen_hi;
     hdr[PH_NCHUNK0] = tile_total[0];
     hdr[PH_NCHUNK1] = tile_total[1];
-    hdr[PH_NCHUNK2] = tile_total[2];
-    for (int w = PH_NCHUNK2 + 1; w < PH_WORDS; ++w) hdr[w] = 0;
+    hdr[PH_LANES] = p.lanes;
+    hdr[PH_ROWS_SHRINK] = rows_total[0];
+    hdr[PH_ROWS_EXPAND] = rows_total[1];
+    for (int w = PH_ROWS_EXPAND + 1; w < PH_WORDS; ++w) hdr[w] = 0;
     if (counters[1] > 0) {
       mint::report(p.status, MINT_ERR_NOT_RESIDENT, counters[2]);
       if (p.status) atomicAdd(&p.status[1], counters[1]);
@@ -289,7 +352,7 @@ int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 
 }  // namespace
 
-PlanOffsets mint_plan_offsets(int64_t P) {
+PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
   PlanOffsets o;
   const int64_t n = (P > 0 ? P : 1);
   int64_t cur = 0;
@@ -308,6 +371,9 @@ PlanOffsets mint_plan_offsets(int64_t P) {
     o.tile_seg[g] = take(n);
     o.tile_off[g] = take(n);
   }
+  o.tile_desc = take((mint_tile_upper_bound(1, P, key_space) + 1) * (int64_t)(sizeof(TileDesc) / 4));
+  o.lane_shrink = take(MINT_MAX_LANES + 1);
+  o.lane_expand = take(MINT_MAX_LANES + 1);
   o.key_a = take(n);
   o.key_b = take(n);
   o.idx_a = take(n);
@@ -323,8 +389,8 @@ int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space) {
   return ub < P ? ub : P;
 }
 
-PlanView mint_plan_view(const void *plan_dev, int64_t P) {
-  const PlanOffsets o = mint_plan_offsets(P);
+PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space) {
+  const PlanOffsets o = mint_plan_offsets(P, key_space);
   const char *b = static_cast<const char *>(plan_dev);
   PlanView v;
   v.header = reinterpret_cast<const int32_t *>(b + o.header);
@@ -337,13 +403,17 @@ PlanView mint_plan_view(const void *plan_dev, int64_t P) {
     v.tile_seg[g] = reinterpret_cast<const int32_t *>(b + o.tile_seg[g]);
     v.tile_off[g] = reinterpret_cast<const int32_t *>(b + o.tile_off[g]);
   }
+  v.tile_desc = reinterpret_cast<const TileDesc *>(b + o.tile_desc);
+  v.lane_shrink = reinterpret_cast<const int32_t *>(b + o.lane_shrink);
+  v.lane_expand = reinterpret_cast<const int32_t *>(b + o.lane_expand);
   return v;
 }
 
 int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, const int32_t *expert_ids,
-                         int32_t K, int32_t num_experts, void *plan_dev, int32_t *status,
+                         int32_t K, int32_t num_experts, int32_t lanes, void *plan_dev, int32_t *status,
                          cudaStream_t stream) {
   PlanParams p;
+  p.lanes = lanes;
   p.tab = tab;
   p.ids = ids;
   p.expert_ids = expert_ids;
@@ -356,7 +426,7 @@ int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, con
   while ((1ll << nbits) <= (long long)p.key_space) ++nbits;  // key_space itself must fit
   p.npass = (nbits + 7) / 8;
   p.digit_bits = (nbits + p.npass - 1) / p.npass;
-  p.off = mint_plan_offsets(p.P);
+  p.off = mint_plan_offsets(p.P, p.key_space);
   p.blob = static_cast<char *>(plan_dev);
   p.status = status;
   plan_kernel<<<1, kThreads, 0, stream>>>(p);

@@ -159,7 +159,7 @@ int pick_cluster(int64_t tiles_ub) {
 int32_t mint_launch_shrink(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s) {
   const int64_t ub = mint_tile_upper_bound(0, a.T, tab.num_slots);
   if (ub == 0) return MINT_OK;
-  shrink_kernel<<<(unsigned)ub, kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, a.T));
+  shrink_kernel<<<(unsigned)ub, kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, a.T, tab.num_slots));
   return mint_check_cuda(cudaGetLastError(), "shrink kernel launch");
 }
 
@@ -168,7 +168,7 @@ int32_t mint_launch_expand(const DenseArgs &a, const TableDev &tab, const void *
   if (ub == 0) return MINT_OK;
   int ny = 1;
   while (ub * ny < 592 && ny < 16 && (a.n >> 3) / (ny * 2) >= 32) ny *= 2;
-  expand_kernel<<<dim3((unsigned)ub, ny), kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, a.T));
+  expand_kernel<<<dim3((unsigned)ub, ny), kTileThreads, 0, s>>>(a, tab, mint_plan_view(plan_dev, a.T, tab.num_slots));
   return mint_check_cuda(cudaGetLastError(), "expand kernel launch");
 }
 
@@ -189,6 +189,6 @@ int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *p
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const PlanView pv = mint_plan_view(plan_dev, a.T);
+  const PlanView pv = mint_plan_view(plan_dev, a.T, tab.num_slots);
   return mint_check_cuda(cudaLaunchKernelEx(&cfg, fused_kernel, a, tab, pv), "fused kernel launch");
 }
