@@ -36,7 +36,7 @@ enum {
 };
 #define MINT_PLAN_MAGIC 0x4D4C5032  // "MLP2"
 #define MINT_NUM_TILE_LISTS 2
-#define MINT_MAX_LANES 256
+#define MINT_MAX_LANES 1024
 // Tile list g cuts every segment into runs of at most mint_tile_tokens(g) items.
 __host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 32; }
 
@@ -92,7 +92,7 @@ struct PlanView {
   const int32_t *lane_expand;
 };
 PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space);
-// Number of cost lanes plans are cut for on the current device (its SM count).
+// Number of cost lanes plans are cut for on the current device (four per SM).
 int32_t mint_device_lanes(int32_t *lanes_out);
 
 // ---- host handles ----------------------------------------------------------
