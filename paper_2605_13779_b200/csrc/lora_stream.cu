@@ -40,10 +40,11 @@
 // before the dependency wait of a launch, by prefetching the weights.
 //
 // v travels from the shrink to the expand through a small L2-resident
-// workspace.  A tile whose columns are shared by several lanes gets one partial
-// sum per lane; the lane that completes the tile (a ticket counted in column
-// blocks) adds the partials in lane order, so the result does not depend on
-// scheduling.
+// workspace: every shrink lane writes the sum over its own columns of a tile
+// (slot tile + lane, so no two writers meet), and the expand, which knows the
+// shrink's split from the same arithmetic, adds the lanes of a tile in lane
+// order while it builds its operand fragments.  No atomics, no fences, and the
+// result does not depend on scheduling.
 //
 // Launch overlap: both kernels let their successor become resident at once
 // (griddepcontrol.launch_dependents first thing) and are launched with
@@ -81,9 +82,7 @@ struct StreamProblem {
   int64_t ldx, ldy;
   int32_t d, n, r_max;
   int32_t cb0_shrink, cb0_expand;  // first virtual column block of this problem
-  float *ws_v;         // [tiles_ub][32 * r_max]          complete shrink result of a tile, [len][rank] packed
-  float *ws_part;      // [tiles_ub + lanes][32 * r_max]  partial sums of tiles shared by several lanes
-  int32_t *ws_ticket;  // [tiles_ub], zero between launches
+  float *ws_part;      // [tiles_ub + lanes][32 * r_max]  slot (tile + lane): that lane's sum, [len][rank] packed
 };
 
 struct StreamParams {
@@ -166,10 +165,9 @@ struct CtaRange {
 struct CtaShared {
   TileDesc desc[kBatchTiles];
   int32_t rows[kBatchItems];
-  int32_t contrib[MINT_MAX_LANES];   // lanes holding a partial of the tile being completed
-  int32_t range[5];
+  int32_t contrib[MINT_MAX_LANES];   // expand: shrink lanes holding a part of the current tile's v
+  int32_t range[4];
   int32_t ncontrib;
-  int32_t flag;
 };
 
 template <bool kExpand>
@@ -295,32 +293,46 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][b][e] = 0.f;
 
-  for (int blk = pc.lo + warp; blk < pc.hi; blk += kWarps) {
-    const int col = blk * kShrinkBlock;
-    const bool ok = col + t * 8 < pb.d;
-    const int colp = col + kPrefetchAhead * kWarps * kShrinkBlock;
-    if (colp + t * 8 < pb.d && blk + kPrefetchAhead * kWarps < pc.hi) {
+  // U blocks of this warp are loaded together so that enough bytes are in flight
+  constexpr int U = (2 * MT + NT <= 4) ? 4 : 2;
+  for (int blk0 = pc.lo + warp; blk0 < pc.hi; blk0 += kWarps * U) {
+    const int colp = (blk0 + kPrefetchAhead * kWarps * U) * kShrinkBlock;
+    if (colp + t * 8 < pb.d && blk0 + kPrefetchAhead * kWarps * U < pc.hi) {
 #pragma unroll
-      for (int i = 0; i < MT * 2; ++i)
-        if (xr[i]) prefetch_l2(xr[i] + colp);
+      for (int u = 0; u < U; ++u) {
+        const int cu = colp + u * kWarps * kShrinkBlock;
+        if (cu + t * 8 < pb.d && blk0 + (kPrefetchAhead * U + u) * kWarps < pc.hi) {
 #pragma unroll
-      for (int i = 0; i < NT; ++i)
-        if (wr[i]) prefetch_l2(wr[i] + colp);
+          for (int i = 0; i < MT * 2; ++i)
+            if (xr[i]) prefetch_l2(xr[i] + cu);
+#pragma unroll
+          for (int i = 0; i < NT; ++i)
+            if (wr[i]) prefetch_l2(wr[i] + cu);
+        }
+      }
     }
-    uint4 xa[MT * 2], wb[NT];
+    uint4 xa[U][MT * 2], wb[U][NT];
 #pragma unroll
-    for (int i = 0; i < MT * 2; ++i) xa[i] = (ok && xr[i]) ? ld128(xr[i] + col) : zero4();
+    for (int u = 0; u < U; ++u) {
+      const int blk = blk0 + u * kWarps;
+      const int col = blk * kShrinkBlock;
+      const bool ok = blk < pc.hi && col + t * 8 < pb.d;
 #pragma unroll
-    for (int i = 0; i < NT; ++i) wb[i] = (ok && wr[i]) ? ldg128_stream(wr[i] + col) : zero4();
+      for (int i = 0; i < MT * 2; ++i) xa[u][i] = (ok && xr[i]) ? ld128(xr[i] + col) : zero4();
 #pragma unroll
-    for (int ks = 0; ks < 2; ++ks)
+      for (int i = 0; i < NT; ++i) wb[u][i] = (ok && wr[i]) ? ldg128_stream(wr[i] + col) : zero4();
+    }
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt)
+    for (int u = 0; u < U; ++u)
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-          mma_bf16(acc[mt][nt], word(xa[2 * mt], 2 * ks), word(xa[2 * mt + 1], 2 * ks),
-                   word(xa[2 * mt], 2 * ks + 1), word(xa[2 * mt + 1], 2 * ks + 1), word(wb[nt], 2 * ks),
-                   word(wb[nt], 2 * ks + 1));
+      for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt)
+            mma_bf16(acc[mt][nt], word(xa[u][2 * mt], 2 * ks), word(xa[u][2 * mt + 1], 2 * ks),
+                     word(xa[u][2 * mt], 2 * ks + 1), word(xa[u][2 * mt + 1], 2 * ks + 1), word(wb[u][nt], 2 * ks),
+                     word(wb[u][nt], 2 * ks + 1));
   }
   // scratch[warp][mt][nt][lane][4]
 #pragma unroll
@@ -344,24 +356,38 @@ __device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece 
   for (int l = 0; l < L; ++l) acc[l] = 0.f;
   const int c0 = pc.lo * kShrinkBlock, c1 = min(pc.hi * kShrinkBlock, pb.d);
   constexpr int kStep = kWarps * 256;
-  for (int col = c0 + warp * 256 + lane * 8; col < c1; col += kStep) {
-    if (col + kPrefetchAhead * kStep < c1) {
-      prefetch_l2(w + col + kPrefetchAhead * kStep);
+  constexpr int U = L <= 2 ? 4 : 2;
+  for (int col0 = c0 + warp * 256 + lane * 8; col0 < c1; col0 += kStep * U) {
 #pragma unroll
-      for (int l = 0; l < L; ++l)
-        if (l < pc.len) prefetch_l2(xr[l] + col + kPrefetchAhead * kStep);
+    for (int u = 0; u < U; ++u) {
+      const int cp = col0 + (kPrefetchAhead * U + u) * kStep;
+      if (cp < c1) {
+        prefetch_l2(w + cp);
+#pragma unroll
+        for (int l = 0; l < L; ++l)
+          if (l < pc.len) prefetch_l2(xr[l] + cp);
+      }
     }
-    float wf[8];
-    unpack8(ldg128_stream(w + col), wf);
-    uint4 xq[L];
+    uint4 wq[U], xq[U][L];
 #pragma unroll
-    for (int l = 0; l < L; ++l) xq[l] = ld128(xr[l] + col);
+    for (int u = 0; u < U; ++u) {
+      const int col = col0 + u * kStep;
+      const bool ok = col < c1;
+      wq[u] = ok ? ldg128_stream(w + col) : zero4();
 #pragma unroll
-    for (int l = 0; l < L; ++l) {
-      float xf[8];
-      unpack8(xq[l], xf);
+      for (int l = 0; l < L; ++l) xq[u][l] = ok ? ld128(xr[l] + col) : zero4();
+    }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[l] = fmaf(xf[e], wf[e], acc[l]);
+    for (int u = 0; u < U; ++u) {
+      float wf[8];
+      unpack8(wq[u], wf);
+#pragma unroll
+      for (int l = 0; l < L; ++l) {
+        float xf[8];
+        unpack8(xq[u][l], xf);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[l] = fmaf(xf[e], wf[e], acc[l]);
+      }
     }
   }
 #pragma unroll
@@ -376,14 +402,12 @@ struct SmemShrink {
   float scratch[kWarps * 2 * 4 * 128];   // [warp][m-tile][n-tile][lane][4] MMA fragments, or [warp][8] sums
 };
 
-__device__ __forceinline__ void shrink_piece(const StreamParams &P, const Area &area, SmemShrink &S,
-                                             const Piece &pc) {
+__device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &S, const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x;
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
-  const bool whole = pc.hi - pc.lo == pc.blocks;   // this lane covers the whole width: the result is final
-  float *dst = whole ? pb.ws_v + (size_t)pc.t * slot_floats
-                     : pb.ws_part + (size_t)(pc.t + blockIdx.x) * slot_floats;
+  // the sum over this lane's columns; the expand adds the lanes of a tile in lane order
+  float *dst = pb.ws_part + (size_t)(pc.t + blockIdx.x) * slot_floats;
   const bool vec = pc.r == 1 && pc.len <= 8;
   for (int rh = 0; rh < pc.r; rh += 32) {
     const int rr = min(32, pc.r - rh);
@@ -419,52 +443,6 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, const Area &
       dst[l * pc.r + rh + j] = s;
     }
   }
-  if (whole) return;
-  // several lanes share this tile: count the column blocks done; the lane that
-  // completes the tile adds all partials in lane order
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int done = atomicAdd(&pb.ws_ticket[pc.t], pc.hi - pc.lo) + (pc.hi - pc.lo);
-    S.sh.flag = (done == pc.blocks);
-  }
-  __syncthreads();
-  if (!S.sh.flag) return;
-  __threadfence();
-  if (warp == 0) {
-    // lanes whose share meets this tile's columns of this problem, from the area arithmetic alone
-    const TileDesc d = P.pv.tile_desc[pc.t];
-    const int w_t = tile_rows<false>(d.rank, d.len);
-    const int64_t begin = (int64_t)d.rows_shrink * area.CB, end = begin + (int64_t)w_t * area.CB;
-    int count = 0;
-    for (int base = 0; base < area.active; base += 32) {
-      const int c2 = base + lane;
-      bool hit = false;
-      if (c2 < area.active) {
-        const int64_t p0 = lane_pos(area, c2), p1 = lane_pos(area, c2 + 1);
-        if (p0 < end && p1 > begin) {
-          const int va = p0 <= begin ? 0 : (int)((p0 - begin) / w_t);
-          const int vb = p1 >= end ? area.CB : (int)((p1 - begin) / w_t);
-          const int lo = max(va, pb.cb0_shrink), hi = min(vb, pb.cb0_shrink + pc.blocks);
-          hit = lo < hi;
-        }
-      }
-      const unsigned m = __ballot_sync(0xffffffffu, hit);
-      if (hit) S.sh.contrib[count + __popc(m & ((1u << lane) - 1u))] = c2;
-      count += __popc(m);
-    }
-    if (lane == 0) S.sh.ncontrib = count;
-  }
-  __syncthreads();
-  const int ncontrib = S.sh.ncontrib;
-  float *v_tile = pb.ws_v + (size_t)pc.t * slot_floats;
-  for (int i = tid; i < pc.len * pc.r; i += kThreads) {
-    float s = 0.f;
-    for (int k = 0; k < ncontrib; ++k)
-      s += __ldcg(pb.ws_part + (size_t)(pc.t + S.sh.contrib[k]) * slot_floats + i);
-    v_tile[i] = s;
-  }
-  if (tid == 0) pb.ws_ticket[pc.t] = 0;   // leave the tickets zero for the next launch
 }
 
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(const StreamParams P) {
@@ -484,7 +462,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
       pdl_wait();   // activations, v and the tickets belong to earlier kernels until here
       waited = true;
     }
-    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, area, S, pc); });
+    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, S, pc); });
   }
 }
 
@@ -505,23 +483,13 @@ struct SmemExpand {
   float vvec[8];   // rank-1 path: v per token
 };
 
-// 16 output columns of one row: y += scale * acc, acc[j][0] -> column j, acc[j][1] -> column 8 + j
-__device__ __forceinline__ void update_row(uint16_t *yp, bool ok_a, bool ok_b, float scale, const float (&acc)[8][4],
-                                           int h) {
-  if (ok_a) {
-    float f[8];
-    unpack8(ld128(yp), f);
+// 8 output columns of one row: y += scale * acc[j][e] for column j, stored with one 128-bit write
+__device__ __forceinline__ void update8(uint16_t *yp, const uint4 &old, float scale, const float (&acc)[8][4], int e) {
+  float f[8];
+  unpack8(old, f);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] = fmaf(scale, acc[j][2 * h], f[j]);
-    *reinterpret_cast<uint4 *>(yp) = pack8(f);
-  }
-  if (ok_b) {
-    float f[8];
-    unpack8(ld128(yp + 8), f);
-#pragma unroll
-    for (int j = 0; j < 8; ++j) f[j] = fmaf(scale, acc[j][2 * h + 1], f[j]);
-    *reinterpret_cast<uint4 *>(yp + 8) = pack8(f);
-  }
+  for (int j = 0; j < 8; ++j) f[j] = fmaf(scale, acc[j][e], f[j]);
+  *reinterpret_cast<uint4 *>(yp) = pack8(f);
 }
 
 __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, const SmemExpand &S) {
@@ -542,9 +510,15 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
     }
     uint4 bq[2][4];   // B rows 2t, 2t+1, 2t+8, 2t+9 of two k-steps
     for (int mt = 0; mt < MT; ++mt) {
+      // the y segments this lane updates go out first: their latency overlaps the weights and the MMAs
       const int row0 = mt * 16 + g, row1 = row0 + 8;
       uint16_t *y0 = row0 < pc.len ? pb.y + (int64_t)pc.rows[row0] * pb.ldy + n0 + t * 16 : nullptr;
       uint16_t *y1 = row1 < pc.len ? pb.y + (int64_t)pc.rows[row1] * pb.ldy + n0 + t * 16 : nullptr;
+      uint4 yq[4];
+      yq[0] = (y0 && ok_y0) ? ld128(y0) : zero4();
+      yq[1] = (y0 && ok_y1) ? ld128(y0 + 8) : zero4();
+      yq[2] = (y1 && ok_y0) ? ld128(y1) : zero4();
+      yq[3] = (y1 && ok_y1) ? ld128(y1 + 8) : zero4();
       float acc[8][4];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
@@ -577,8 +551,11 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
           }
         }
       }
-      if (y0) update_row(y0, ok_y0, ok_y1, pc.scale, acc, 0);
-      if (y1) update_row(y1, ok_y0, ok_y1, pc.scale, acc, 1);
+      // acc[j][0], [1]: row g, columns 16 t + j and 16 t + 8 + j; acc[j][2], [3]: row g + 8
+      if (y0 && ok_y0) update8(y0, yq[0], pc.scale, acc, 0);
+      if (y0 && ok_y1) update8(y0 + 8, yq[1], pc.scale, acc, 1);
+      if (y1 && ok_y0) update8(y1, yq[2], pc.scale, acc, 2);
+      if (y1 && ok_y1) update8(y1 + 8, yq[3], pc.scale, acc, 3);
     }
   }
 }
@@ -596,39 +573,100 @@ __device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece 
   }
   const int c0 = pc.lo * kExpandBlock, c1 = min(pc.hi * kExpandBlock, pb.n);
   constexpr int kStep = kWarps * 256;
-  for (int col = c0 + warp * 256 + lane * 8; col < c1; col += kStep) {
-    if (col + kPrefetchAhead * kStep < c1) {
-      prefetch_l2(w + col + kPrefetchAhead * kStep);
+  constexpr int U = L <= 2 ? 4 : 2;
+  for (int col0 = c0 + warp * 256 + lane * 8; col0 < c1; col0 += kStep * U) {
 #pragma unroll
-      for (int l = 0; l < L; ++l)
-        if (l < pc.len) prefetch_l2(yr[l] + col + kPrefetchAhead * kStep);
-    }
-    float wf[8];
-    unpack8(ldg128_stream(w + col), wf);
-    uint4 yq[L];
+    for (int u = 0; u < U; ++u) {
+      const int cp = col0 + (kPrefetchAhead * U + u) * kStep;
+      if (cp < c1) {
+        prefetch_l2(w + cp);
 #pragma unroll
-    for (int l = 0; l < L; ++l)
-      if (l < pc.len) yq[l] = ld128(yr[l] + col);
-#pragma unroll
-    for (int l = 0; l < L; ++l)
-      if (l < pc.len) {
-        float yf[8];
-        unpack8(yq[l], yf);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) yf[e] = fmaf(sv[l], wf[e], yf[e]);
-        *reinterpret_cast<uint4 *>(yr[l] + col) = pack8(yf);
+        for (int l = 0; l < L; ++l)
+          if (l < pc.len) prefetch_l2(yr[l] + cp);
       }
+    }
+    uint4 wq[U], yq[U][L];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int col = col0 + u * kStep;
+      const bool ok = col < c1;
+      wq[u] = ok ? ldg128_stream(w + col) : zero4();
+#pragma unroll
+      for (int l = 0; l < L; ++l) yq[u][l] = (ok && l < pc.len) ? ld128(yr[l] + col) : zero4();
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int col = col0 + u * kStep;
+      if (col < c1) {
+        float wf[8];
+        unpack8(wq[u], wf);
+#pragma unroll
+        for (int l = 0; l < L; ++l)
+          if (l < pc.len) {
+            float yf[8];
+            unpack8(yq[u][l], yf);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) yf[e] = fmaf(sv[l], wf[e], yf[e]);
+            *reinterpret_cast<uint4 *>(yr[l] + col) = pack8(yf);
+          }
+      }
+    }
   }
 }
 
-__device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &S, const Piece &pc) {
+// The shrink lanes whose share met the columns of problem p in tile t, in lane
+// order, from the area arithmetic of the shrink kernel alone (warp 0).
+__device__ __forceinline__ void shrink_contributors(const StreamParams &P, const Area &sa, CtaShared &sh,
+                                                    const Piece &pc) {
+  const int lane = threadIdx.x & 31;
+  const StreamProblem &pb = P.prob[pc.p];
+  const TileDesc d = P.pv.tile_desc[pc.t];
+  const int w_t = tile_rows<false>(d.rank, d.len);
+  const int blocks = (pb.d + kShrinkBlock - 1) / kShrinkBlock;
+  const int64_t begin = (int64_t)d.rows_shrink * sa.CB, end = begin + (int64_t)w_t * sa.CB;
+  const int64_t lo_pos = begin + (int64_t)pb.cb0_shrink * w_t;
+  const int64_t hi_pos = begin + (int64_t)(pb.cb0_shrink + blocks) * w_t - 1;
+  const int64_t total = sa.W * sa.CB;
+  // largest table index j with pos(j) <= P, then the largest active lane starting at or before j
+  const int64_t j_a = ((lo_pos + 1) * sa.G - 1) / total, j_b = ((hi_pos + 1) * sa.G - 1) / total;
+  const int c_a = (int)(((j_a + 1) * sa.active - 1) / sa.G), c_b = (int)(((j_b + 1) * sa.active - 1) / sa.G);
+  int count = 0;
+  for (int base = c_a; base <= c_b; base += 32) {
+    const int c2 = base + lane;
+    bool hit = false;
+    if (c2 <= c_b) {
+      const int64_t p0 = lane_pos(sa, c2), p1 = lane_pos(sa, c2 + 1);
+      if (p0 < end && p1 > begin) {
+        const int va = p0 <= begin ? 0 : (int)((p0 - begin) / w_t);
+        const int vb = p1 >= end ? sa.CB : (int)((p1 - begin) / w_t);
+        hit = max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks);
+      }
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, hit);
+    if (hit) sh.contrib[count + __popc(m & ((1u << lane) - 1u))] = c2;
+    count += __popc(m);
+  }
+  if (lane == 0) sh.ncontrib = count;
+}
+
+// v[row][k] of the current tile: the sum, in lane order, of the shrink lanes' parts
+__device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, const CtaShared &sh, int t, int idx) {
+  float s = 0.f;
+  for (int k = 0; k < sh.ncontrib; ++k) s += __ldcg(part + (size_t)(t + sh.contrib[k]) * slot_floats + idx);
+  return s;
+}
+
+__device__ __forceinline__ void expand_piece(const StreamParams &P, const Area &shrink_area, SmemExpand &S,
+                                             const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
   const int tid = threadIdx.x;
-  const float *v_tile = pb.ws_v + (size_t)pc.t * kTileRowsMax * pb.r_max;
+  const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   const bool vec = pc.r == 1 && pc.len <= 8;
   __syncthreads();   // the previous piece no longer reads the fragments
+  if (tid < 32) shrink_contributors(P, shrink_area, S.sh, pc);
+  __syncthreads();
   if (vec) {
-    if (tid < 8) S.vvec[tid] = tid < pc.len ? __ldcg(v_tile + tid) : 0.f;
+    if (tid < 8) S.vvec[tid] = tid < pc.len ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, tid) : 0.f;
   } else {
     const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
@@ -639,8 +677,9 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int row = mt * 16 + g + (q & 1) * 8, k = ks * 16 + 2 * t + (q >> 1) * 8;
-        const float a = (row < pc.len && k < pc.r) ? __ldcg(v_tile + row * pc.r + k) : 0.f;
-        const float b = (row < pc.len && k + 1 < pc.r) ? __ldcg(v_tile + row * pc.r + k + 1) : 0.f;
+        const float a = (row < pc.len && k < pc.r) ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, row * pc.r + k) : 0.f;
+        const float b =
+            (row < pc.len && k + 1 < pc.r) ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, row * pc.r + k + 1) : 0.f;
         split_pair(a, b, hi[q], lo[q]);
       }
       S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + ln] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
@@ -670,6 +709,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
     pdl_wait();
     return;
   }
+  const Area shrink_area = make_area<false>(P);
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
@@ -688,23 +728,13 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
       pdl_wait();   // the shrink kernel has completed: v is final, y belongs to this kernel
       waited = true;
     }
-    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, S, pc); });
+    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, shrink_area, S, pc); });
   }
 }
 
 // ---- host side -----------------------------------------------------------------
-struct WorkspaceLayout {
-  size_t ticket, v, part, total;
-};
-
-WorkspaceLayout workspace_layout(int64_t tiles, int32_t r_max) {
-  WorkspaceLayout w;
-  const size_t slot_bytes = (size_t)kTileRowsMax * r_max * sizeof(float);
-  w.ticket = 0;
-  w.v = ((size_t)tiles * 4 + 255) / 256 * 256;
-  w.part = w.v + (size_t)tiles * slot_bytes;
-  w.total = w.part + (size_t)(tiles + MINT_MAX_LANES) * slot_bytes + 256;
-  return w;
+size_t workspace_bytes(int64_t tiles, int32_t r_max) {
+  return (size_t)(tiles + MINT_MAX_LANES) * kTileRowsMax * r_max * sizeof(float) + 256;
 }
 
 }  // namespace
@@ -712,7 +742,7 @@ WorkspaceLayout workspace_layout(int64_t tiles, int32_t r_max) {
 bool mint_stream_supported(int32_t r_max_bound) { return r_max_bound <= kStreamRankCap; }
 
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max) {
-  return workspace_layout(mint_tile_upper_bound(1, T, num_slots), r_max).total;
+  return workspace_bytes(mint_tile_upper_bound(1, T, num_slots), r_max);
 }
 
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
@@ -737,11 +767,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
     pb.cb0_expand = cb_e;
     cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
     cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
-    const WorkspaceLayout w = workspace_layout(tiles, a.r_max);
-    uint8_t *base = static_cast<uint8_t *>(workspaces[i]);
-    pb.ws_ticket = reinterpret_cast<int32_t *>(base + w.ticket);
-    pb.ws_v = reinterpret_cast<float *>(base + w.v);
-    pb.ws_part = reinterpret_cast<float *>(base + w.part);
+    pb.ws_part = static_cast<float *>(workspaces[i]);
   }
   P.nprob = nprob;
   P.T = T;
