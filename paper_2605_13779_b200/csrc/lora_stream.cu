@@ -137,6 +137,7 @@ struct Area {
   int CB;        // column blocks of the whole call
   int G;         // lanes the plan's table was cut for (= grid size)
   int active;    // lanes that take work
+  const LaneStart *table;
 };
 
 template <bool kExpand>
@@ -145,16 +146,21 @@ __device__ __forceinline__ Area make_area(const StreamParams &P) {
   a.W = P.pv.header[kExpand ? PH_ROWS_EXPAND : PH_ROWS_SHRINK];
   a.CB = kExpand ? P.cb_expand : P.cb_shrink;
   a.G = P.lanes;
+  a.table = kExpand ? P.pv.lane_expand : P.pv.lane_shrink;
   int64_t g = a.W * a.CB / (kExpand ? kExpandGrain : kShrinkGrain);
   if (g < 1) g = 1;
   if (g > a.G) g = a.G;
   a.active = (int)g;
   return a;
 }
-// Start of active lane c in area positions (c == active: the end of the area).
-__device__ __forceinline__ int64_t lane_pos(const Area &a, int c) {
-  const int64_t j = (int64_t)c * a.G / a.active;
-  return j * a.W * a.CB / a.G;
+// Table index of active lane c (c == active: the end of the area).
+__device__ __forceinline__ int lane_index(const Area &a, int c) {
+  return (int)((unsigned)c * (unsigned)a.G / (unsigned)a.active);
+}
+// Where table lane j starts relative to row `rows` of the area, in (row x column block)
+// units: (q - rows) * CB + r * CB / G.  The caller knows the result is small.
+__device__ __forceinline__ int64_t lane_offset(const Area &a, const LaneStart &ls, int rows) {
+  return (int64_t)(ls.q - rows) * a.CB + (int)((unsigned)ls.r * (unsigned)a.CB / (unsigned)a.G);
 }
 
 struct CtaRange {
@@ -186,17 +192,15 @@ __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, A
   const int c = blockIdx.x;
   if (c >= area.active) return false;
   if (threadIdx.x < 2) {   // thread 0: the cut where this lane starts; thread 1: where it ends
-    const int cc = c + threadIdx.x;
-    const int64_t j = (int64_t)cc * area.G / area.active;
-    const int32_t *table = kExpand ? P.pv.lane_expand : P.pv.lane_shrink;
-    const int tile = table[j];
+    const int j = lane_index(area, c + threadIdx.x);
+    const LaneStart ls = area.table[j];
     int cb = 0;
     if (j < area.G) {
-      const TileDesc d = P.pv.tile_desc[tile];
-      const int64_t base = (int64_t)(kExpand ? d.rows_expand : d.rows_shrink) * area.CB;
-      cb = (int)((lane_pos(area, cc) - base) / tile_rows<kExpand>(d.rank, d.len));
+      const TileDesc d = P.pv.tile_desc[ls.tile];
+      cb = (int)(lane_offset(area, ls, kExpand ? d.rows_expand : d.rows_shrink) /
+                 tile_rows<kExpand>(d.rank, d.len));
     }
-    sh.range[2 * threadIdx.x] = tile;
+    sh.range[2 * threadIdx.x] = ls.tile;
     sh.range[2 * threadIdx.x + 1] = cb;
   }
   __syncthreads();
@@ -213,7 +217,7 @@ __device__ __forceinline__ void load_batch(const StreamParams &P, CtaShared &sh,
   __syncthreads();  // every warp is done with the previous batch
   const int4 *src = reinterpret_cast<const int4 *>(P.pv.tile_desc + tb);
   int4 *dst = reinterpret_cast<int4 *>(sh.desc);
-  for (int i = threadIdx.x; i < ntile * 2; i += kThreads) dst[i] = src[i];
+  for (int i = threadIdx.x; i < ntile * (int)(sizeof(TileDesc) / 16); i += kThreads) dst[i] = src[i];
   __syncthreads();
   const int off0 = sh.desc[0].off;
   const int nitems = sh.desc[ntile - 1].off + sh.desc[ntile - 1].len - off0;
@@ -229,6 +233,7 @@ struct Piece {
   const int32_t *rows;   // the tile's row indices (shared memory)
   int r, len, slot;
   float scale;
+  int lane_lo, lane_hi;   // bounds of the shrink lanes that can meet this tile
 };
 
 // Walks the pieces of one batch of tiles in order; f(piece) is called by all threads.
@@ -247,6 +252,8 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     pc.len = sh.desc[ti].len;
     pc.scale = sh.desc[ti].scale;
     pc.slot = sh.desc[ti].slot;
+    pc.lane_lo = sh.desc[ti].lane_lo;
+    pc.lane_hi = sh.desc[ti].lane_hi;
     pc.rows = sh.rows + (sh.desc[ti].off - sh.desc[0].off);
     for (int p = 0; p < P.nprob; ++p) {
       const StreamProblem &pb = P.prob[p];
@@ -480,7 +487,7 @@ struct SmemExpand {
   CtaShared sh;
   // v of the current tile as MMA A-operand fragments: [m-tile][k-step][head/remainder][lane] x 4 registers
   uint4 vfrag[2 * 4 * 2 * 32];
-  float vvec[8];   // rank-1 path: v per token
+  float vsum[kTileRowsMax * kStreamRankCap];   // v of the current tile, [len][rank] packed
 };
 
 // 8 output columns of one row: y += scale * acc[j][e] for column j, stored with one 128-bit write
@@ -569,7 +576,7 @@ __device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece 
 #pragma unroll
   for (int l = 0; l < L; ++l) {
     yr[l] = pb.y + (int64_t)pc.rows[l < pc.len ? l : 0] * pb.ldy;
-    sv[l] = pc.scale * S.vvec[l];
+    sv[l] = pc.scale * S.vsum[l < pc.len ? l : 0];
   }
   const int c0 = pc.lo * kExpandBlock, c1 = min(pc.hi * kExpandBlock, pb.n);
   constexpr int kStep = kWarps * 256;
@@ -617,28 +624,27 @@ __device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece 
 // The shrink lanes whose share met the columns of problem p in tile t, in lane
 // order, from the area arithmetic of the shrink kernel alone (warp 0).
 __device__ __forceinline__ void shrink_contributors(const StreamParams &P, const Area &sa, CtaShared &sh,
-                                                    const Piece &pc) {
+                                                    const Piece &pc, int lane_lo, int lane_hi) {
   const int lane = threadIdx.x & 31;
   const StreamProblem &pb = P.prob[pc.p];
   const TileDesc d = P.pv.tile_desc[pc.t];
   const int w_t = tile_rows<false>(d.rank, d.len);
   const int blocks = (pb.d + kShrinkBlock - 1) / kShrinkBlock;
-  const int64_t begin = (int64_t)d.rows_shrink * sa.CB, end = begin + (int64_t)w_t * sa.CB;
-  const int64_t lo_pos = begin + (int64_t)pb.cb0_shrink * w_t;
-  const int64_t hi_pos = begin + (int64_t)(pb.cb0_shrink + blocks) * w_t - 1;
-  const int64_t total = sa.W * sa.CB;
-  // largest table index j with pos(j) <= P, then the largest active lane starting at or before j
-  const int64_t j_a = ((lo_pos + 1) * sa.G - 1) / total, j_b = ((hi_pos + 1) * sa.G - 1) / total;
-  const int c_a = (int)(((j_a + 1) * sa.active - 1) / sa.G), c_b = (int)(((j_b + 1) * sa.active - 1) / sa.G);
+  const int span = w_t * sa.CB;   // the tile's extent in area units
+  // active lanes c with table index in [lane_lo, lane_hi]: index(c) = c G / active
+  const int c_a = (int)(((unsigned)(lane_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
+  const int c_b = (int)(((unsigned)(lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
   int count = 0;
   for (int base = c_a; base <= c_b; base += 32) {
     const int c2 = base + lane;
     bool hit = false;
     if (c2 <= c_b) {
-      const int64_t p0 = lane_pos(sa, c2), p1 = lane_pos(sa, c2 + 1);
-      if (p0 < end && p1 > begin) {
-        const int va = p0 <= begin ? 0 : (int)((p0 - begin) / w_t);
-        const int vb = p1 >= end ? sa.CB : (int)((p1 - begin) / w_t);
+      const int j0 = lane_index(sa, c2), j1 = lane_index(sa, c2 + 1);
+      const int64_t p0 = lane_offset(sa, sa.table[j0], d.rows_shrink);
+      const int64_t p1 = lane_offset(sa, sa.table[j1], d.rows_shrink);
+      if (p0 < span && p1 > 0) {
+        const int va = p0 <= 0 ? 0 : (int)p0 / w_t;
+        const int vb = p1 >= span ? sa.CB : (int)p1 / w_t;
         hit = max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks);
       }
     }
@@ -649,10 +655,19 @@ __device__ __forceinline__ void shrink_contributors(const StreamParams &P, const
   if (lane == 0) sh.ncontrib = count;
 }
 
-// v[row][k] of the current tile: the sum, in lane order, of the shrink lanes' parts
+// v[idx] of the current tile: the sum, in lane order, of the shrink lanes' parts.
+// The loads of up to eight parts are issued together.
 __device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, const CtaShared &sh, int t, int idx) {
   float s = 0.f;
-  for (int k = 0; k < sh.ncontrib; ++k) s += __ldcg(part + (size_t)(t + sh.contrib[k]) * slot_floats + idx);
+  const int n = sh.ncontrib;
+  for (int k0 = 0; k0 < n; k0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      v[k] = (k0 + k < n) ? __ldcg(part + (size_t)(t + sh.contrib[min(k0 + k, n - 1)]) * slot_floats + idx) : 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += v[k];
+  }
   return s;
 }
 
@@ -663,11 +678,11 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, const Area &
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   const bool vec = pc.r == 1 && pc.len <= 8;
   __syncthreads();   // the previous piece no longer reads the fragments
-  if (tid < 32) shrink_contributors(P, shrink_area, S.sh, pc);
+  if (tid < 32) shrink_contributors(P, shrink_area, S.sh, pc, pc.lane_lo, pc.lane_hi);
   __syncthreads();
-  if (vec) {
-    if (tid < 8) S.vvec[tid] = tid < pc.len ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, tid) : 0.f;
-  } else {
+  for (int i = tid; i < pc.len * pc.r; i += kThreads) S.vsum[i] = sum_v(pb.ws_part, slot_floats, S.sh, pc.t, i);
+  __syncthreads();
+  if (!vec) {
     const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
     for (int i = tid; i < MT * KS * 32; i += kThreads) {
@@ -677,9 +692,8 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, const Area &
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int row = mt * 16 + g + (q & 1) * 8, k = ks * 16 + 2 * t + (q >> 1) * 8;
-        const float a = (row < pc.len && k < pc.r) ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, row * pc.r + k) : 0.f;
-        const float b =
-            (row < pc.len && k + 1 < pc.r) ? sum_v(pb.ws_part, slot_floats, S.sh, pc.t, row * pc.r + k + 1) : 0.f;
+        const float a = (row < pc.len && k < pc.r) ? S.vsum[row * pc.r + k] : 0.f;
+        const float b = (row < pc.len && k + 1 < pc.r) ? S.vsum[row * pc.r + k + 1] : 0.f;
         split_pair(a, b, hi[q], lo[q]);
       }
       S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + ln] = make_uint4(hi[0], hi[1], hi[2], hi[3]);

@@ -46,6 +46,8 @@ __host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 
 // rows_shrink / rows_expand are the exclusive prefix sums, over tiles, of
 // (rank + len) and (rank + 2 len): the row counts whose product with a
 // projection's width gives the bytes the shrink and the expand stream.
+// lane_lo..lane_hi bound the shrink lanes (of the plan's G) whose share can
+// meet this tile: the lanes j with  rows_shrink - W/G < j W/G < rows_shrink + rank + len.
 struct __align__(16) TileDesc {
   int32_t off;     // first position of the tile in perm
   int32_t len;     // 1..32 items
@@ -55,6 +57,19 @@ struct __align__(16) TileDesc {
   float scale;
   int32_t rows_shrink;
   int32_t rows_expand;
+  int32_t lane_lo;
+  int32_t lane_hi;
+  int32_t pad0, pad1;
+};
+
+// Start of cost lane j in the rows x column-blocks area: the tile that holds it
+// and j * rows_total = q * G + r, so that the position for CB column blocks is
+// q * CB + r * CB / G without any 64-bit division.
+struct __align__(16) LaneStart {
+  int32_t tile;
+  int32_t q;
+  int32_t r;
+  int32_t pad;
 };
 
 // Byte offsets of every array inside the plan blob (host-computed, passed by value).
@@ -68,8 +83,8 @@ struct PlanOffsets {
   int64_t tile_seg[MINT_NUM_TILE_LISTS];  // int32[P]  segment of tile c
   int64_t tile_off[MINT_NUM_TILE_LISTS];  // int32[P]  first position (in perm) of tile c
   int64_t tile_desc;   // TileDesc[tile upper bound of list 1]
-  int64_t lane_shrink; // int32[MINT_MAX_LANES + 1]  tile holding the start of cost lane j (shrink rows)
-  int64_t lane_expand; // int32[MINT_MAX_LANES + 1]  same for the expand rows
+  int64_t lane_shrink; // LaneStart[MINT_MAX_LANES + 1]  start of cost lane j in the shrink rows
+  int64_t lane_expand; // LaneStart[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
   int64_t total;
 };
@@ -88,8 +103,8 @@ struct PlanView {
   const int32_t *tile_seg[MINT_NUM_TILE_LISTS];
   const int32_t *tile_off[MINT_NUM_TILE_LISTS];
   const TileDesc *tile_desc;
-  const int32_t *lane_shrink;
-  const int32_t *lane_expand;
+  const LaneStart *lane_shrink;
+  const LaneStart *lane_expand;
 };
 PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space);
 // Number of cost lanes plans are cut for on the current device (four per SM).

@@ -264,8 +264,8 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   // G lanes; lane j starts inside the tile t with rows[t]*G <= j*rows_total,
   // which does not depend on the projection's width, so it is tabulated here.
   TileDesc *desc = reinterpret_cast<TileDesc *>(p.blob + p.off.tile_desc);
-  int32_t *lane_tab[2] = {reinterpret_cast<int32_t *>(p.blob + p.off.lane_shrink),
-                          reinterpret_cast<int32_t *>(p.blob + p.off.lane_expand)};
+  LaneStart *lane_tab[2] = {reinterpret_cast<LaneStart *>(p.blob + p.off.lane_shrink),
+                            reinterpret_cast<LaneStart *>(p.blob + p.off.lane_expand)};
   int rows_total[2];
   {
     const int32_t *tseg = reinterpret_cast<const int32_t *>(p.blob + p.off.tile_seg[1]);
@@ -283,6 +283,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     }
     int run_s = block_exclusive_scan(sum_s, warp_tot, rows_total[0]);
     int run_e = block_exclusive_scan(sum_e, warp_tot, rows_total[1]);
+    const int64_t G = p.lanes;
     for (int c = c_begin; c < c_end; ++c) {
       const int sg = tseg[c];
       const int slot = seg_slot[sg];
@@ -295,27 +296,35 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       dsc.scale = p.tab.slot_scale[slot];
       dsc.rows_shrink = run_s;
       dsc.rows_expand = run_e;
-      desc[c] = dsc;
-      // lanes whose start falls inside this tile: rows[c]*G <= j*total < rows[c+1]*G
-      const int64_t G = p.lanes;
       const int begin[2] = {run_s, run_e};
       const int end[2] = {run_s + dsc.rank + dsc.len, run_e + dsc.rank + 2 * dsc.len};
+      // shrink lanes that can meet this tile: from the last lane starting at or
+      // before the tile's first row to the last lane starting before its end
+      dsc.lane_lo = (int32_t)(begin[0] * G / rows_total[0]);
+      dsc.lane_hi = (int32_t)min(G - 1, (end[0] * G - 1) / rows_total[0]);
+      dsc.pad0 = dsc.pad1 = 0;
+      desc[c] = dsc;
+      // lanes whose start falls inside this tile: rows[c]*G <= j*total < rows[c+1]*G
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         const int64_t tot = rows_total[q];
         const int64_t j_lo = (begin[q] * G + tot - 1) / tot;
         const int64_t j_hi = (end[q] * G + tot - 1) / tot;   // exclusive
-        for (int64_t j = j_lo; j < j_hi && j < G; ++j) lane_tab[q][j] = c;
+        for (int64_t j = j_lo; j < j_hi && j < G; ++j) lane_tab[q][j].tile = c;
       }
       run_s = end[0];
       run_e = end[1];
     }
-    if (tid == 0) {
-      lane_tab[0][p.lanes] = ntile;
-      lane_tab[1][p.lanes] = ntile;
+    for (int j = tid; j <= p.lanes; j += kThreads) {
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int64_t jw = (int64_t)j * rows_total[q];
+        lane_tab[q][j].q = (int32_t)(jw / G);
+        lane_tab[q][j].r = (int32_t)(jw % G);
+        lane_tab[q][j].pad = 0;
+        if (j == p.lanes || ntile == 0) lane_tab[q][j].tile = (j == p.lanes) ? ntile : 0;
+      }
     }
-    if (ntile == 0)
-      for (int j = tid; j < p.lanes; j += kThreads) lane_tab[0][j] = lane_tab[1][j] = 0;
   }
   __syncthreads();
 
@@ -372,8 +381,8 @@ PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
     o.tile_off[g] = take(n);
   }
   o.tile_desc = take((mint_tile_upper_bound(1, P, key_space) + 1) * (int64_t)(sizeof(TileDesc) / 4));
-  o.lane_shrink = take(MINT_MAX_LANES + 1);
-  o.lane_expand = take(MINT_MAX_LANES + 1);
+  o.lane_shrink = take((MINT_MAX_LANES + 1) * (int64_t)(sizeof(LaneStart) / 4));
+  o.lane_expand = take((MINT_MAX_LANES + 1) * (int64_t)(sizeof(LaneStart) / 4));
   o.key_a = take(n);
   o.key_b = take(n);
   o.idx_a = take(n);
@@ -404,8 +413,8 @@ PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space) {
     v.tile_off[g] = reinterpret_cast<const int32_t *>(b + o.tile_off[g]);
   }
   v.tile_desc = reinterpret_cast<const TileDesc *>(b + o.tile_desc);
-  v.lane_shrink = reinterpret_cast<const int32_t *>(b + o.lane_shrink);
-  v.lane_expand = reinterpret_cast<const int32_t *>(b + o.lane_expand);
+  v.lane_shrink = reinterpret_cast<const LaneStart *>(b + o.lane_shrink);
+  v.lane_expand = reinterpret_cast<const LaneStart *>(b + o.lane_expand);
   return v;
 }
 
