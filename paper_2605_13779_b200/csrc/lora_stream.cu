@@ -72,6 +72,7 @@ constexpr int kExpandBlock = 64;          // elements of n per column block
 constexpr int kShrinkGrain = 128;         // smallest lane share in (row x block) units: 128 x 64 B
 constexpr int kExpandGrain = 64;          //                                           64 x 128 B
 constexpr int kPrefetchAhead = 2;         // a warp prefetches this many of its own blocks ahead
+constexpr int kMaxParts = 8;              // shrink lanes that may share one tile of one projection
 constexpr int kMaxProblems = MINT_MAX_GROUP;
 
 struct StreamProblem {
@@ -91,6 +92,7 @@ struct StreamParams {
   int32_t T;
   int32_t lanes;                      // grid size = the plan's lane count
   int32_t cb_shrink, cb_expand;       // virtual column blocks of the whole call
+  int32_t cb_shrink_widest;           // column blocks of the widest d of the call
   int32_t *status;
   TableDev tab;
   PlanView pv;
@@ -148,6 +150,12 @@ __device__ __forceinline__ Area make_area(const StreamParams &P) {
   a.G = P.lanes;
   a.table = kExpand ? P.pv.lane_expand : P.pv.lane_shrink;
   int64_t g = a.W * a.CB / (kExpand ? kExpandGrain : kShrinkGrain);
+  if (!kExpand) {
+    // The expand adds the parts of every shrink lane that met a tile: keep the
+    // largest tile of the widest projection within kMaxParts lane shares.
+    const int64_t big = (int64_t)P.pv.header[PH_MAX_TILE_ROWS] * P.cb_shrink_widest;
+    if (big > 0) g = min(g, (int64_t)(kMaxParts - 1) * a.W * a.CB / big);
+  }
   if (g < 1) g = 1;
   if (g > a.G) g = a.G;
   a.active = (int)g;
@@ -171,9 +179,9 @@ struct CtaRange {
 struct CtaShared {
   TileDesc desc[kBatchTiles];
   int32_t rows[kBatchItems];
-  int32_t contrib[MINT_MAX_LANES];   // expand: shrink lanes holding a part of the current tile's v
+  int16_t part_first[kBatchTiles * kMaxProblems];   // expand: first shrink lane holding a part of (tile, problem)
+  int16_t part_count[kBatchTiles * kMaxProblems];   //         and how many consecutive lanes do
   int32_t range[4];
-  int32_t ncontrib;
 };
 
 template <bool kExpand>
@@ -234,6 +242,7 @@ struct Piece {
   int r, len, slot;
   float scale;
   int lane_lo, lane_hi;   // bounds of the shrink lanes that can meet this tile
+  int ti;                 // index of the tile in the staged batch
 };
 
 // Walks the pieces of one batch of tiles in order; f(piece) is called by all threads.
@@ -248,6 +257,7 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     if (va >= vb) continue;
     Piece pc;
     pc.t = t;
+    pc.ti = ti;
     pc.r = sh.desc[ti].rank;
     pc.len = sh.desc[ti].len;
     pc.scale = sh.desc[ti].scale;
@@ -267,6 +277,31 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
       pc.hi = hi;
       pc.blocks = count;
       f(pc);
+    }
+  }
+}
+
+// Pulls the rows of a piece into L2 (all threads): the weight rows, which no apply
+// kernel writes, may go before the dependency wait; activations only after it.
+template <bool kExpand>
+__device__ __forceinline__ void prefetch_piece(const StreamProblem &pb, const Piece &pc, bool weights, bool acts) {
+  constexpr int kBlock = kExpand ? kExpandBlock : kShrinkBlock;
+  const int width = kExpand ? pb.n : pb.d;
+  const int c0 = pc.lo * kBlock, c1 = min(pc.hi * kBlock, width);
+  const int lines = ((c1 - c0) * 2 + 127) / 128 + 1;   // one address per 128 bytes, plus the last 16 bytes
+  if (weights) {
+    const uint16_t *w = (kExpand ? pb.B : pb.A) + (int64_t)pc.slot * pb.r_max * width;
+    for (int i = threadIdx.x; i < pc.r * lines; i += kThreads) {
+      const int row = i / lines, ln = i - row * lines;
+      prefetch_l2(w + (int64_t)row * width + min(c0 + ln * 64, c1 - 8));
+    }
+  }
+  if (acts) {
+    const uint16_t *a = kExpand ? pb.y : pb.x;
+    const int64_t ld = kExpand ? pb.ldy : pb.ldx;
+    for (int i = threadIdx.x; i < pc.len * lines; i += kThreads) {
+      const int row = i / lines, ln = i - row * lines;
+      prefetch_l2(a + (int64_t)pc.rows[row] * ld + min(c0 + ln * 64, c1 - 8));
     }
   }
 }
@@ -465,9 +500,14 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
     load_batch(P, S.sh, tb, ntile);
+    // the whole batch goes to L2 at once: A rows right away, x rows once the wait is over
+    walk_batch<false>(P, area, R, S.sh, tb, ntile,
+                      [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, true, waited); });
     if (!waited) {
-      pdl_wait();   // activations, v and the tickets belong to earlier kernels until here
+      pdl_wait();   // activations and the workspace belong to earlier kernels until here
       waited = true;
+      walk_batch<false>(P, area, R, S.sh, tb, ntile,
+                        [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, false, true); });
     }
     walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, S, pc); });
   }
@@ -621,66 +661,60 @@ __device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece 
   }
 }
 
-// The shrink lanes whose share met the columns of problem p in tile t, in lane
-// order, from the area arithmetic of the shrink kernel alone (warp 0).
-__device__ __forceinline__ void shrink_contributors(const StreamParams &P, const Area &sa, CtaShared &sh,
-                                                    const Piece &pc, int lane_lo, int lane_hi) {
-  const int lane = threadIdx.x & 31;
-  const StreamProblem &pb = P.prob[pc.p];
-  const TileDesc d = P.pv.tile_desc[pc.t];
+// The shrink lanes whose share met the columns of problem p in the tile: they
+// are consecutive lanes, found from the area arithmetic of the shrink kernel
+// alone (one thread per piece of the batch).
+__device__ __forceinline__ void shrink_parts(const StreamParams &P, const Area &sa, const TileDesc &d, int p,
+                                             int &first, int &count) {
+  const StreamProblem &pb = P.prob[p];
   const int w_t = tile_rows<false>(d.rank, d.len);
   const int blocks = (pb.d + kShrinkBlock - 1) / kShrinkBlock;
   const int span = w_t * sa.CB;   // the tile's extent in area units
   // active lanes c with table index in [lane_lo, lane_hi]: index(c) = c G / active
-  const int c_a = (int)(((unsigned)(lane_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
-  const int c_b = (int)(((unsigned)(lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
-  int count = 0;
-  for (int base = c_a; base <= c_b; base += 32) {
-    const int c2 = base + lane;
-    bool hit = false;
-    if (c2 <= c_b) {
-      const int j0 = lane_index(sa, c2), j1 = lane_index(sa, c2 + 1);
-      const int64_t p0 = lane_offset(sa, sa.table[j0], d.rows_shrink);
-      const int64_t p1 = lane_offset(sa, sa.table[j1], d.rows_shrink);
-      if (p0 < span && p1 > 0) {
-        const int va = p0 <= 0 ? 0 : (int)p0 / w_t;
-        const int vb = p1 >= span ? sa.CB : (int)p1 / w_t;
-        hit = max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks);
+  const int c_a = (int)(((unsigned)(d.lane_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
+  const int c_b = (int)(((unsigned)(d.lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
+  first = 0;
+  count = 0;
+  int64_t p0 = lane_offset(sa, sa.table[lane_index(sa, c_a)], d.rows_shrink);
+  for (int c2 = c_a; c2 <= c_b; ++c2) {
+    const int64_t p1 = lane_offset(sa, sa.table[lane_index(sa, c2 + 1)], d.rows_shrink);
+    if (p0 < span && p1 > 0) {
+      const int va = p0 <= 0 ? 0 : (int)p0 / w_t;
+      const int vb = p1 >= span ? sa.CB : (int)p1 / w_t;
+      if (max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks)) {
+        if (count == 0) first = c2;
+        ++count;
       }
     }
-    const unsigned m = __ballot_sync(0xffffffffu, hit);
-    if (hit) sh.contrib[count + __popc(m & ((1u << lane) - 1u))] = c2;
-    count += __popc(m);
+    p0 = p1;
   }
-  if (lane == 0) sh.ncontrib = count;
 }
 
 // v[idx] of the current tile: the sum, in lane order, of the shrink lanes' parts.
 // The loads of up to eight parts are issued together.
-__device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, const CtaShared &sh, int t, int idx) {
+__device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, int t, int first, int count, int idx) {
   float s = 0.f;
-  const int n = sh.ncontrib;
-  for (int k0 = 0; k0 < n; k0 += 8) {
+  for (int k0 = 0; k0 < count; k0 += 8) {
     float v[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k)
-      v[k] = (k0 + k < n) ? __ldcg(part + (size_t)(t + sh.contrib[min(k0 + k, n - 1)]) * slot_floats + idx) : 0.f;
+      v[k] = (k0 + k < count) ? __ldcg(part + (size_t)(t + first + k0 + k) * slot_floats + idx) : 0.f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) s += v[k];
   }
   return s;
 }
 
-__device__ __forceinline__ void expand_piece(const StreamParams &P, const Area &shrink_area, SmemExpand &S,
-                                             const Piece &pc) {
+__device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &S, const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
   const int tid = threadIdx.x;
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   const bool vec = pc.r == 1 && pc.len <= 8;
-  __syncthreads();   // the previous piece no longer reads the fragments
-  if (tid < 32) shrink_contributors(P, shrink_area, S.sh, pc, pc.lane_lo, pc.lane_hi);
-  __syncthreads();
-  for (int i = tid; i < pc.len * pc.r; i += kThreads) S.vsum[i] = sum_v(pb.ws_part, slot_floats, S.sh, pc.t, i);
+  const int first = S.sh.part_first[pc.ti * kMaxProblems + pc.p];
+  const int count = S.sh.part_count[pc.ti * kMaxProblems + pc.p];
+  __syncthreads();   // the previous piece no longer reads v or the fragments
+  for (int i = tid; i < pc.len * pc.r; i += kThreads)
+    S.vsum[i] = sum_v(pb.ws_part, slot_floats, pc.t, first, count, i);
   __syncthreads();
   if (!vec) {
     const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
@@ -728,21 +762,26 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
     load_batch(P, S.sh, tb, ntile);
+    // which shrink lanes hold the parts of v of every (tile, projection) of the batch
+    for (int i = threadIdx.x; i < ntile * P.nprob; i += kThreads) {
+      const int ti = i / P.nprob, p = i - ti * P.nprob;
+      int first, count;
+      shrink_parts(P, shrink_area, S.sh.desc[ti], p, first, count);
+      S.sh.part_first[ti * kMaxProblems + p] = (int16_t)first;
+      S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
+    }
+    // the whole batch goes to L2 at once: B rows right away (while the shrink
+    // kernel still runs, for the first batch), y rows once the wait is over
+    walk_batch<true>(P, area, R, S.sh, tb, ntile,
+                     [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, true, waited); });
     if (!waited) {
-      // while the shrink kernel still runs: pull the first weight blocks of every piece into L2
-      walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) {
-        const StreamProblem &pb = P.prob[pc.p];
-        const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
-        const int c0 = pc.lo * kExpandBlock;
-        const int c1 = min(min(pc.hi, pc.lo + kPrefetchAhead * kWarps) * kExpandBlock, pb.n);
-        const int per_row = (c1 - c0 + 63) >> 6;   // 128-byte lines
-        for (int i = threadIdx.x; i < pc.r * per_row; i += kThreads)
-          prefetch_l2(B_slot + (int64_t)(i / per_row) * pb.n + c0 + (i % per_row) * 64);
-      });
       pdl_wait();   // the shrink kernel has completed: v is final, y belongs to this kernel
       waited = true;
+      walk_batch<true>(P, area, R, S.sh, tb, ntile,
+                       [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, false, true); });
     }
-    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, shrink_area, S, pc); });
+    __syncthreads();
+    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, S, pc); });
   }
 }
 
@@ -770,7 +809,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   const int64_t tiles = mint_tile_upper_bound(1, T, tab.num_slots);
   if (tiles == 0) return MINT_OK;
   StreamParams P = {};
-  int cb_s = 0, cb_e = 0;
+  int cb_s = 0, cb_e = 0, cb_widest = 0;
   for (int i = 0; i < nprob; ++i) {
     const DenseArgs &a = args[i];
     StreamProblem &pb = P.prob[i];
@@ -780,6 +819,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
     pb.cb0_shrink = cb_s;
     pb.cb0_expand = cb_e;
     cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
+    cb_widest = std::max(cb_widest, (a.d + kShrinkBlock - 1) / kShrinkBlock);
     cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
     pb.ws_part = static_cast<float *>(workspaces[i]);
   }
@@ -788,6 +828,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   P.lanes = lanes;
   P.cb_shrink = cb_s;
   P.cb_expand = cb_e;
+  P.cb_shrink_widest = cb_widest;
   P.status = args[0].status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);

@@ -32,6 +32,7 @@ enum {
   PH_LANES,     // number of cost lanes G the lane tables were cut for
   PH_ROWS_SHRINK,  // sum over list-1 tiles of (rank + len)
   PH_ROWS_EXPAND,  // sum over list-1 tiles of (rank + 2 len)
+  PH_MAX_TILE_ROWS,  // largest (rank + len) of a list-1 tile
   PH_WORDS = 32
 };
 #define MINT_PLAN_MAGIC 0x4D4C5032  // "MLP2"

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   __shared__ int32_t bin_base[256];
   __shared__ int warp_tot[kWarps + 1];
   __shared__ int32_t counters[8];  // 0 inactive, 1 not resident, 2 first missing token, 3 bad expert,
-                                   // 4 first bad item, 5 max segment, 6 sum rank
+                                   // 4 first bad item, 5 max segment, 6 sum rank, 7 max tile rows
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.P;
@@ -280,6 +280,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       const int r = p.tab.slot_rank[seg_slot[sg]];
       sum_s += r + len;
       sum_e += r + 2 * len;
+      atomicMax(&counters[7], r + len);
     }
     int run_s = block_exclusive_scan(sum_s, warp_tot, rows_total[0]);
     int run_e = block_exclusive_scan(sum_e, warp_tot, rows_total[1]);
@@ -348,7 +349,8 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     hdr[PH_LANES] = p.lanes;
     hdr[PH_ROWS_SHRINK] = rows_total[0];
     hdr[PH_ROWS_EXPAND] = rows_total[1];
-    for (int w = PH_ROWS_EXPAND + 1; w < PH_WORDS; ++w) hdr[w] = 0;
+    hdr[PH_MAX_TILE_ROWS] = counters[7];
+    for (int w = PH_MAX_TILE_ROWS + 1; w < PH_WORDS; ++w) hdr[w] = 0;
     if (counters[1] > 0) {
       mint::report(p.status, MINT_ERR_NOT_RESIDENT, counters[2]);
       if (p.status) atomicAdd(&p.status[1], counters[1]);
