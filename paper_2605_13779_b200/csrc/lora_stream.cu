@@ -62,7 +62,9 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kCtasPerSm = 4;
+constexpr int kCtasPerSm = 3;
+constexpr int kRingSlots = 26;            // 512-byte slots (16 B per lane) of a warp's staging ring
+constexpr int kRingBytes = kRingSlots * 512;
 constexpr int kTileRowsMax = 32;          // plan tile list 1
 constexpr int kStreamRankCap = 64;        // larger ranks take the CUDA-core cluster kernel
 constexpr int kBatchTiles = 16;           // tile descriptors staged in shared memory at a time
@@ -71,7 +73,6 @@ constexpr int kShrinkBlock = 32;          // elements of d per column block
 constexpr int kExpandBlock = 64;          // elements of n per column block
 constexpr int kShrinkGrain = 128;         // smallest lane share in (row x block) units: 128 x 64 B
 constexpr int kExpandGrain = 64;          //                                           64 x 128 B
-constexpr int kPrefetchAhead = 2;         // a warp prefetches this many of its own blocks ahead
 constexpr int kMaxParts = 8;              // shrink lanes that may share one tile of one projection
 constexpr int kMaxProblems = MINT_MAX_GROUP;
 
@@ -106,9 +107,40 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void prefetch_l2(const void *p) {
   asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
-// 128-bit load of data another kernel of this stream produced (y, and x after the wait)
-__device__ __forceinline__ uint4 ld128(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
-__device__ __forceinline__ uint4 zero4() { return make_uint4(0u, 0u, 0u, 0u); }
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+// 16-byte asynchronous copy global -> shared, L2 only; zero-fills when !valid (nothing is read then).
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+  const int bytes = valid ? 16 : 0;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 r;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
+  return r;
+}
+
+// A warp's private staging ring.  Every lane copies the 16-byte segments it will
+// use itself into its own column of the ring (slot s, lane l at byte (s * 32 +
+// l) * 16) and reads them back after cp.async.wait_group: no thread ever reads
+// another thread's copy, so the pipeline needs no barrier, costs no registers
+// for the bytes in flight, and an iteration of N segments runs kRingSlots / N
+// iterations ahead.
+template <int N>
+struct Ring {
+  static constexpr int kDepth = kRingSlots / N;
+  static_assert(kDepth >= 1, "an iteration does not fit the ring");
+  uint32_t base;   // shared-memory address of this lane's column
+  __device__ __forceinline__ uint32_t slot(int it, int i) const {
+    return base + (uint32_t)(((it % kDepth) * N + i) * 512);
+  }
+};
 
 // D(16x8, f32) += A(16x16, bf16, row) * B(16x8, bf16, col)
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -311,21 +343,23 @@ __device__ __forceinline__ void prefetch_piece(const StreamProblem &pb, const Pi
 // ================================================================================
 // Tensor-core body for ranks [rh, rh + 8 NT) of the piece: this warp's blocks.
 template <int MT, int NT>
-__device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece &pc, int rh, float *scratch) {
+__device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece &pc, int rh, uint32_t ring_base,
+                                           float *scratch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
+  constexpr int N = 2 * MT + NT;
+  Ring<N> ring{ring_base};
   const uint16_t *A_slot = pb.A + (int64_t)pc.slot * pb.r_max * pb.d;
-  const uint16_t *xr[MT * 2];
-  const uint16_t *wr[NT];
+  const uint16_t *src[N];   // this lane's row of every operand fragment (nullptr: the row does not exist)
 #pragma unroll
   for (int i = 0; i < MT * 2; ++i) {
     const int row = i * 8 + g;
-    xr[i] = row < pc.len ? pb.x + (int64_t)pc.rows[row] * pb.ldx + t * 8 : nullptr;
+    src[i] = row < pc.len ? pb.x + (int64_t)pc.rows[row] * pb.ldx + t * 8 : nullptr;
   }
 #pragma unroll
   for (int i = 0; i < NT; ++i) {
     const int row = rh + i * 8 + g;
-    wr[i] = row < pc.r ? A_slot + (int64_t)row * pb.d + t * 8 : nullptr;
+    src[2 * MT + i] = row < pc.r ? A_slot + (int64_t)row * pb.d + t * 8 : nullptr;
   }
   float acc[MT][NT][4];
 #pragma unroll
@@ -335,47 +369,39 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[a][b][e] = 0.f;
 
-  // U blocks of this warp are loaded together so that enough bytes are in flight
-  constexpr int U = (2 * MT + NT <= 4) ? 4 : 2;
-  for (int blk0 = pc.lo + warp; blk0 < pc.hi; blk0 += kWarps * U) {
-    const int colp = (blk0 + kPrefetchAhead * kWarps * U) * kShrinkBlock;
-    if (colp + t * 8 < pb.d && blk0 + kPrefetchAhead * kWarps * U < pc.hi) {
+  const int first = pc.lo + warp;
+  const int iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
+  auto issue = [&](int it) {
+    if (it < iters) {
+      const int col = (first + it * kWarps) * kShrinkBlock;
+      const bool ok = col + t * 8 < pb.d;
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int cu = colp + u * kWarps * kShrinkBlock;
-        if (cu + t * 8 < pb.d && blk0 + (kPrefetchAhead * U + u) * kWarps < pc.hi) {
-#pragma unroll
-          for (int i = 0; i < MT * 2; ++i)
-            if (xr[i]) prefetch_l2(xr[i] + cu);
-#pragma unroll
-          for (int i = 0; i < NT; ++i)
-            if (wr[i]) prefetch_l2(wr[i] + cu);
-        }
-      }
+      for (int i = 0; i < N; ++i) cp_async16(ring.slot(it, i), src[i] ? src[i] + col : pb.A, ok && src[i]);
     }
-    uint4 xa[U][MT * 2], wb[U][NT];
+    cp_async_commit();
+  };
+#pragma unroll 1
+  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    issue(it + Ring<N>::kDepth - 1);
+    cp_async_wait<Ring<N>::kDepth - 1>();
+    uint4 xa[MT * 2], wb[NT];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int blk = blk0 + u * kWarps;
-      const int col = blk * kShrinkBlock;
-      const bool ok = blk < pc.hi && col + t * 8 < pb.d;
+    for (int i = 0; i < MT * 2; ++i) xa[i] = lds128(ring.slot(it, i));
 #pragma unroll
-      for (int i = 0; i < MT * 2; ++i) xa[u][i] = (ok && xr[i]) ? ld128(xr[i] + col) : zero4();
+    for (int i = 0; i < NT; ++i) wb[i] = lds128(ring.slot(it, 2 * MT + i));
 #pragma unroll
-      for (int i = 0; i < NT; ++i) wb[u][i] = (ok && wr[i]) ? ldg128_stream(wr[i] + col) : zero4();
-    }
+    for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
-    for (int u = 0; u < U; ++u)
+      for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-      for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-          for (int nt = 0; nt < NT; ++nt)
-            mma_bf16(acc[mt][nt], word(xa[u][2 * mt], 2 * ks), word(xa[u][2 * mt + 1], 2 * ks),
-                     word(xa[u][2 * mt], 2 * ks + 1), word(xa[u][2 * mt + 1], 2 * ks + 1), word(wb[u][nt], 2 * ks),
-                     word(wb[u][nt], 2 * ks + 1));
+        for (int nt = 0; nt < NT; ++nt)
+          mma_bf16(acc[mt][nt], word(xa[2 * mt], 2 * ks), word(xa[2 * mt + 1], 2 * ks),
+                   word(xa[2 * mt], 2 * ks + 1), word(xa[2 * mt + 1], 2 * ks + 1), word(wb[nt], 2 * ks),
+                   word(wb[nt], 2 * ks + 1));
   }
+  cp_async_wait<0>();
   // scratch[warp][mt][nt][lane][4]
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
@@ -387,8 +413,11 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
 
 // rank-1 tiles of at most L tokens: fp32 FMAs over coalesced 512-byte warp loads.
 template <int L>
-__device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece &pc, float *scratch) {
+__device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
+                                           float *scratch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int N = 1 + L;
+  Ring<N> ring{ring_base};
   const uint16_t *w = pb.A + (int64_t)pc.slot * pb.r_max * pb.d;
   const uint16_t *xr[L];
 #pragma unroll
@@ -396,42 +425,36 @@ __device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece 
   float acc[L];
 #pragma unroll
   for (int l = 0; l < L; ++l) acc[l] = 0.f;
-  const int c0 = pc.lo * kShrinkBlock, c1 = min(pc.hi * kShrinkBlock, pb.d);
+  const int c0 = pc.lo * kShrinkBlock + warp * 256 + lane * 8, c1 = min(pc.hi * kShrinkBlock, pb.d);
   constexpr int kStep = kWarps * 256;
-  constexpr int U = L <= 2 ? 4 : 2;
-  for (int col0 = c0 + warp * 256 + lane * 8; col0 < c1; col0 += kStep * U) {
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int cp = col0 + (kPrefetchAhead * U + u) * kStep;
-      if (cp < c1) {
-        prefetch_l2(w + cp);
-#pragma unroll
-        for (int l = 0; l < L; ++l)
-          if (l < pc.len) prefetch_l2(xr[l] + cp);
-      }
-    }
-    uint4 wq[U], xq[U][L];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int col = col0 + u * kStep;
+  const int iters = (c1 - (pc.lo * kShrinkBlock + warp * 256) + kStep - 1) / kStep;   // <= 0: nothing for this warp
+  auto issue = [&](int it) {
+    if (it < iters) {
+      const int col = c0 + it * kStep;
       const bool ok = col < c1;
-      wq[u] = ok ? ldg128_stream(w + col) : zero4();
+      cp_async16(ring.slot(it, 0), ok ? w + col : w, ok);
 #pragma unroll
-      for (int l = 0; l < L; ++l) xq[u][l] = ok ? ld128(xr[l] + col) : zero4();
+      for (int l = 0; l < L; ++l) cp_async16(ring.slot(it, 1 + l), ok ? xr[l] + col : w, ok && l < pc.len);
     }
+    cp_async_commit();
+  };
+#pragma unroll 1
+  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    issue(it + Ring<N>::kDepth - 1);
+    cp_async_wait<Ring<N>::kDepth - 1>();
+    float wf[8];
+    unpack8(lds128(ring.slot(it, 0)), wf);
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      float wf[8];
-      unpack8(wq[u], wf);
+    for (int l = 0; l < L; ++l) {
+      float xf[8];
+      unpack8(lds128(ring.slot(it, 1 + l)), xf);
 #pragma unroll
-      for (int l = 0; l < L; ++l) {
-        float xf[8];
-        unpack8(xq[u][l], xf);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) acc[l] = fmaf(xf[e], wf[e], acc[l]);
-      }
+      for (int e = 0; e < 8; ++e) acc[l] = fmaf(xf[e], wf[e], acc[l]);
     }
   }
+  cp_async_wait<0>();
 #pragma unroll
   for (int l = 0; l < L; ++l) {
     const float s = warp_sum(acc[l]);
@@ -444,7 +467,8 @@ struct SmemShrink {
   float scratch[kWarps * 2 * 4 * 128];   // [warp][m-tile][n-tile][lane][4] MMA fragments, or [warp][8] sums
 };
 
-__device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &S, const Piece &pc) {
+__device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &S, uint32_t ring_base,
+                                             const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
   const int tid = threadIdx.x;
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
@@ -455,18 +479,18 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
     const int rr = min(32, pc.r - rh);
     __syncthreads();   // the scratch is free again
     if (vec) {
-      if (pc.len == 1) shrink_vec<1>(pb, pc, S.scratch);
-      else if (pc.len == 2) shrink_vec<2>(pb, pc, S.scratch);
-      else if (pc.len <= 4) shrink_vec<4>(pb, pc, S.scratch);
-      else shrink_vec<8>(pb, pc, S.scratch);
+      if (pc.len == 1) shrink_vec<1>(pb, pc, ring_base, S.scratch);
+      else if (pc.len == 2) shrink_vec<2>(pb, pc, ring_base, S.scratch);
+      else if (pc.len <= 4) shrink_vec<4>(pb, pc, ring_base, S.scratch);
+      else shrink_vec<8>(pb, pc, ring_base, S.scratch);
     } else if (pc.len <= 16) {
-      if (rr <= 8) shrink_mma<1, 1>(pb, pc, rh, S.scratch);
-      else if (rr <= 16) shrink_mma<1, 2>(pb, pc, rh, S.scratch);
-      else shrink_mma<1, 4>(pb, pc, rh, S.scratch);
+      if (rr <= 8) shrink_mma<1, 1>(pb, pc, rh, ring_base, S.scratch);
+      else if (rr <= 16) shrink_mma<1, 2>(pb, pc, rh, ring_base, S.scratch);
+      else shrink_mma<1, 4>(pb, pc, rh, ring_base, S.scratch);
     } else {
-      if (rr <= 8) shrink_mma<2, 1>(pb, pc, rh, S.scratch);
-      else if (rr <= 16) shrink_mma<2, 2>(pb, pc, rh, S.scratch);
-      else shrink_mma<2, 4>(pb, pc, rh, S.scratch);
+      if (rr <= 8) shrink_mma<2, 1>(pb, pc, rh, ring_base, S.scratch);
+      else if (rr <= 16) shrink_mma<2, 2>(pb, pc, rh, ring_base, S.scratch);
+      else shrink_mma<2, 4>(pb, pc, rh, ring_base, S.scratch);
     }
     __syncthreads();
     // add the four warps' sums in warp order; element (l, rh + j) of the [len][rank] result
@@ -487,7 +511,10 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   }
 }
 
+constexpr size_t kRingsBytes = (size_t)kWarps * kRingBytes;
+
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(const StreamParams P) {
+  extern __shared__ __align__(128) uint8_t dyn_smem[];   // the four warps' rings
   __shared__ SmemShrink S;
   pdl_launch_dependents();
   Area area;
@@ -496,20 +523,20 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
     pdl_wait();
     return;
   }
+  const uint32_t ring_base =
+      smem_addr(dyn_smem) + (uint32_t)((threadIdx.x >> 5) * kRingBytes + (threadIdx.x & 31) * 16);
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
     load_batch(P, S.sh, tb, ntile);
-    // the whole batch goes to L2 at once: A rows right away, x rows once the wait is over
-    walk_batch<false>(P, area, R, S.sh, tb, ntile,
-                      [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, true, waited); });
     if (!waited) {
+      // while the previous kernel still runs: pull this lane's A rows into L2
+      walk_batch<false>(P, area, R, S.sh, tb, ntile,
+                        [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, true, false); });
       pdl_wait();   // activations and the workspace belong to earlier kernels until here
       waited = true;
-      walk_batch<false>(P, area, R, S.sh, tb, ntile,
-                        [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, false, true); });
     }
-    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, S, pc); });
+    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, S, ring_base, pc); });
   }
 }
 
@@ -527,7 +554,7 @@ struct SmemExpand {
   CtaShared sh;
   // v of the current tile as MMA A-operand fragments: [m-tile][k-step][head/remainder][lane] x 4 registers
   uint4 vfrag[2 * 4 * 2 * 32];
-  float vsum[kTileRowsMax * kStreamRankCap];   // v of the current tile, [len][rank] packed
+  float vvec[8];   // rank-1 path: v per token
 };
 
 // 8 output columns of one row: y += scale * acc[j][e] for column j, stored with one 128-bit write
@@ -539,126 +566,142 @@ __device__ __forceinline__ void update8(uint16_t *yp, const uint4 &old, float sc
   *reinterpret_cast<uint4 *>(yp) = pack8(f);
 }
 
-__device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, const SmemExpand &S) {
+template <int MT, int KS>
+__device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
+                                           const SmemExpand &S) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
+  constexpr int N = 4 * KS + 4 * MT;
+  Ring<N> ring{ring_base};
   const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
-  for (int blk = pc.lo + warp; blk < pc.hi; blk += kWarps) {
-    const int n0 = blk * kExpandBlock;
-    const bool ok_b = n0 + g * 8 < pb.n;                       // this lane's 8 columns of B
-    const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;   // its 16 columns of y
-    const int np = n0 + kPrefetchAhead * kWarps * kExpandBlock;
-    if (blk + kPrefetchAhead * kWarps < pc.hi) {
-      if (np + g * 8 < pb.n)
-        for (int k = t; k < pc.r; k += 4) prefetch_l2(B_slot + (int64_t)k * pb.n + np + g * 8);
-      if (np + t * 16 < pb.n)
-        for (int row = g; row < pc.len; row += 8) prefetch_l2(pb.y + (int64_t)pc.rows[row] * pb.ldy + np + t * 16);
+  // this lane's segments of a block: B rows 2t, 2t+1, 2t+8, 2t+9 of every k-step at column 8 g,
+  // then 16 columns of y at column 16 t for rows g, g + 8 of every m-tile
+  const uint16_t *bsrc[4 * KS];
+  uint16_t *ysrc[2 * MT];
+#pragma unroll
+  for (int i = 0; i < 4 * KS; ++i) {
+    const int k = (i >> 2) * 16 + 2 * t + (i & 1) + ((i >> 1) & 1) * 8;
+    bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + g * 8 : nullptr;
+  }
+#pragma unroll
+  for (int i = 0; i < 2 * MT; ++i) {
+    const int row = i * 8 + g;
+    ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 16 : nullptr;
+  }
+  const int first = pc.lo + warp;
+  const int iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
+  auto issue = [&](int it) {
+    if (it < iters) {
+      const int n0 = (first + it * kWarps) * kExpandBlock;
+      const bool ok_b = n0 + g * 8 < pb.n;
+      const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;
+#pragma unroll
+      for (int i = 0; i < 4 * KS; ++i)
+        cp_async16(ring.slot(it, i), bsrc[i] ? bsrc[i] + n0 : pb.B, ok_b && bsrc[i]);
+#pragma unroll
+      for (int i = 0; i < 2 * MT; ++i) {
+        cp_async16(ring.slot(it, 4 * KS + 2 * i), ysrc[i] ? ysrc[i] + n0 : pb.B, ok_y0 && ysrc[i]);
+        cp_async16(ring.slot(it, 4 * KS + 2 * i + 1), ysrc[i] ? ysrc[i] + n0 + 8 : pb.B, ok_y1 && ysrc[i]);
+      }
     }
-    uint4 bq[2][4];   // B rows 2t, 2t+1, 2t+8, 2t+9 of two k-steps
+    cp_async_commit();
+  };
+#pragma unroll 1
+  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    issue(it + Ring<N>::kDepth - 1);
+    cp_async_wait<Ring<N>::kDepth - 1>();
+    const int n0 = (first + it * kWarps) * kExpandBlock;
+    const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;
+#pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      // the y segments this lane updates go out first: their latency overlaps the weights and the MMAs
-      const int row0 = mt * 16 + g, row1 = row0 + 8;
-      uint16_t *y0 = row0 < pc.len ? pb.y + (int64_t)pc.rows[row0] * pb.ldy + n0 + t * 16 : nullptr;
-      uint16_t *y1 = row1 < pc.len ? pb.y + (int64_t)pc.rows[row1] * pb.ldy + n0 + t * 16 : nullptr;
-      uint4 yq[4];
-      yq[0] = (y0 && ok_y0) ? ld128(y0) : zero4();
-      yq[1] = (y0 && ok_y1) ? ld128(y0 + 8) : zero4();
-      yq[2] = (y1 && ok_y0) ? ld128(y1) : zero4();
-      yq[3] = (y1 && ok_y1) ? ld128(y1 + 8) : zero4();
       float acc[8][4];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
-      for (int kk = 0; kk < KS; kk += 2) {
-        if (mt == 0 || KS > 2) {   // with at most two k-steps the weights loaded for m-tile 0 serve m-tile 1
 #pragma unroll
-          for (int q = 0; q < 2; ++q)
+      for (int ks = 0; ks < KS; ++ks) {
+        uint4 bq[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const int k = (kk + q) * 16 + 2 * t + (i & 1) + (i >> 1) * 8;
-              bq[q][i] = (ok_b && k < pc.r) ? ldg128_stream(B_slot + (int64_t)k * pb.n + n0 + g * 8) : zero4();
-            }
-        }
+        for (int i = 0; i < 4; ++i) bq[i] = lds128(ring.slot(it, 4 * ks + i));
+        const uint4 vh = S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + lane];
+        const uint4 vl = S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + lane];
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          if (kk + q < KS) {
-            const uint4 vh = S.vfrag[((mt * 4 + kk + q) * 2 + 0) * 32 + lane];
-            const uint4 vl = S.vfrag[((mt * 4 + kk + q) * 2 + 1) * 32 + lane];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              const uint32_t b0 = (j & 1) ? pair_hi(word(bq[q][0], j >> 1), word(bq[q][1], j >> 1))
-                                          : pair_lo(word(bq[q][0], j >> 1), word(bq[q][1], j >> 1));
-              const uint32_t b1 = (j & 1) ? pair_hi(word(bq[q][2], j >> 1), word(bq[q][3], j >> 1))
-                                          : pair_lo(word(bq[q][2], j >> 1), word(bq[q][3], j >> 1));
-              mma_bf16(acc[j], vh.x, vh.y, vh.z, vh.w, b0, b1);
-              mma_bf16(acc[j], vl.x, vl.y, vl.z, vl.w, b0, b1);
-            }
-          }
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t b0 = (j & 1) ? pair_hi(word(bq[0], j >> 1), word(bq[1], j >> 1))
+                                      : pair_lo(word(bq[0], j >> 1), word(bq[1], j >> 1));
+          const uint32_t b1 = (j & 1) ? pair_hi(word(bq[2], j >> 1), word(bq[3], j >> 1))
+                                      : pair_lo(word(bq[2], j >> 1), word(bq[3], j >> 1));
+          mma_bf16(acc[j], vh.x, vh.y, vh.z, vh.w, b0, b1);
+          mma_bf16(acc[j], vl.x, vl.y, vl.z, vl.w, b0, b1);
         }
       }
       // acc[j][0], [1]: row g, columns 16 t + j and 16 t + 8 + j; acc[j][2], [3]: row g + 8
-      if (y0 && ok_y0) update8(y0, yq[0], pc.scale, acc, 0);
-      if (y0 && ok_y1) update8(y0 + 8, yq[1], pc.scale, acc, 1);
-      if (y1 && ok_y0) update8(y1, yq[2], pc.scale, acc, 2);
-      if (y1 && ok_y1) update8(y1 + 8, yq[3], pc.scale, acc, 3);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint16_t *yr = ysrc[2 * mt + h];
+        if (yr) {
+          if (ok_y0) update8(yr + n0, lds128(ring.slot(it, 4 * KS + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
+          if (ok_y1)
+            update8(yr + n0 + 8, lds128(ring.slot(it, 4 * KS + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
+        }
+      }
     }
   }
+  cp_async_wait<0>();
 }
 
 template <int L>
-__device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece &pc, const SmemExpand &S) {
+__device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
+                                           const SmemExpand &S) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int N = 1 + L;
+  Ring<N> ring{ring_base};
   const uint16_t *w = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
   uint16_t *yr[L];
   float sv[L];
 #pragma unroll
   for (int l = 0; l < L; ++l) {
     yr[l] = pb.y + (int64_t)pc.rows[l < pc.len ? l : 0] * pb.ldy;
-    sv[l] = pc.scale * S.vsum[l < pc.len ? l : 0];
+    sv[l] = pc.scale * S.vvec[l];
   }
-  const int c0 = pc.lo * kExpandBlock, c1 = min(pc.hi * kExpandBlock, pb.n);
+  const int c0 = pc.lo * kExpandBlock + warp * 256 + lane * 8, c1 = min(pc.hi * kExpandBlock, pb.n);
   constexpr int kStep = kWarps * 256;
-  constexpr int U = L <= 2 ? 4 : 2;
-  for (int col0 = c0 + warp * 256 + lane * 8; col0 < c1; col0 += kStep * U) {
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int cp = col0 + (kPrefetchAhead * U + u) * kStep;
-      if (cp < c1) {
-        prefetch_l2(w + cp);
-#pragma unroll
-        for (int l = 0; l < L; ++l)
-          if (l < pc.len) prefetch_l2(yr[l] + cp);
-      }
-    }
-    uint4 wq[U], yq[U][L];
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int col = col0 + u * kStep;
+  const int iters = (c1 - (pc.lo * kExpandBlock + warp * 256) + kStep - 1) / kStep;
+  auto issue = [&](int it) {
+    if (it < iters) {
+      const int col = c0 + it * kStep;
       const bool ok = col < c1;
-      wq[u] = ok ? ldg128_stream(w + col) : zero4();
+      cp_async16(ring.slot(it, 0), ok ? w + col : w, ok);
 #pragma unroll
-      for (int l = 0; l < L; ++l) yq[u][l] = (ok && l < pc.len) ? ld128(yr[l] + col) : zero4();
+      for (int l = 0; l < L; ++l) cp_async16(ring.slot(it, 1 + l), ok ? yr[l] + col : w, ok && l < pc.len);
     }
+    cp_async_commit();
+  };
+#pragma unroll 1
+  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    issue(it + Ring<N>::kDepth - 1);
+    cp_async_wait<Ring<N>::kDepth - 1>();
+    const int col = c0 + it * kStep;
+    if (col < c1) {
+      float wf[8];
+      unpack8(lds128(ring.slot(it, 0)), wf);
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const int col = col0 + u * kStep;
-      if (col < c1) {
-        float wf[8];
-        unpack8(wq[u], wf);
+      for (int l = 0; l < L; ++l)
+        if (l < pc.len) {
+          float yf[8];
+          unpack8(lds128(ring.slot(it, 1 + l)), yf);
 #pragma unroll
-        for (int l = 0; l < L; ++l)
-          if (l < pc.len) {
-            float yf[8];
-            unpack8(yq[u][l], yf);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) yf[e] = fmaf(sv[l], wf[e], yf[e]);
-            *reinterpret_cast<uint4 *>(yr[l] + col) = pack8(yf);
-          }
-      }
+          for (int e = 0; e < 8; ++e) yf[e] = fmaf(sv[l], wf[e], yf[e]);
+          *reinterpret_cast<uint4 *>(yr[l] + col) = pack8(yf);
+        }
     }
   }
+  cp_async_wait<0>();
 }
 
 // The shrink lanes whose share met the columns of problem p in the tile: they
@@ -705,47 +748,60 @@ __device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, in
   return s;
 }
 
-__device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &S, const Piece &pc) {
+__device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &S, uint32_t ring_base,
+                                             const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
   const int tid = threadIdx.x;
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   const bool vec = pc.r == 1 && pc.len <= 8;
   const int first = S.sh.part_first[pc.ti * kMaxProblems + pc.p];
   const int count = S.sh.part_count[pc.ti * kMaxProblems + pc.p];
-  __syncthreads();   // the previous piece no longer reads v or the fragments
-  for (int i = tid; i < pc.len * pc.r; i += kThreads)
-    S.vsum[i] = sum_v(pb.ws_part, slot_floats, pc.t, first, count, i);
-  __syncthreads();
-  if (!vec) {
-    const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
+  const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
+  __syncthreads();   // the previous piece no longer reads v
+  if (vec) {
+    if (tid < 8) S.vvec[tid] = tid < pc.len ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, tid) : 0.f;
+  } else {
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
     for (int i = tid; i < MT * KS * 32; i += kThreads) {
       const int ln = i & 31, ks = (i >> 5) % KS, mt = (i >> 5) / KS;
       const int g = ln >> 2, t = ln & 3;
-      uint32_t hi[4], lo[4];
+      float a[4], b[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int row = mt * 16 + g + (q & 1) * 8, k = ks * 16 + 2 * t + (q >> 1) * 8;
-        const float a = (row < pc.len && k < pc.r) ? S.vsum[row * pc.r + k] : 0.f;
-        const float b = (row < pc.len && k + 1 < pc.r) ? S.vsum[row * pc.r + k + 1] : 0.f;
-        split_pair(a, b, hi[q], lo[q]);
+        a[q] = (row < pc.len && k < pc.r) ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k) : 0.f;
+        b[q] = (row < pc.len && k + 1 < pc.r)
+                   ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k + 1)
+                   : 0.f;
       }
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) split_pair(a[q], b[q], hi[q], lo[q]);
       S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + ln] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
       S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + ln] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
   }
   __syncthreads();
   if (vec) {
-    if (pc.len == 1) expand_vec<1>(pb, pc, S);
-    else if (pc.len == 2) expand_vec<2>(pb, pc, S);
-    else if (pc.len <= 4) expand_vec<4>(pb, pc, S);
-    else expand_vec<8>(pb, pc, S);
+    if (pc.len == 1) expand_vec<1>(pb, pc, ring_base, S);
+    else if (pc.len == 2) expand_vec<2>(pb, pc, ring_base, S);
+    else if (pc.len <= 4) expand_vec<4>(pb, pc, ring_base, S);
+    else expand_vec<8>(pb, pc, ring_base, S);
+  } else if (MT == 1) {
+    if (KS == 1) expand_mma<1, 1>(pb, pc, ring_base, S);
+    else if (KS == 2) expand_mma<1, 2>(pb, pc, ring_base, S);
+    else if (KS == 3) expand_mma<1, 3>(pb, pc, ring_base, S);
+    else expand_mma<1, 4>(pb, pc, ring_base, S);
   } else {
-    expand_mma(pb, pc, S);
+    if (KS == 1) expand_mma<2, 1>(pb, pc, ring_base, S);
+    else if (KS == 2) expand_mma<2, 2>(pb, pc, ring_base, S);
+    else if (KS == 3) expand_mma<2, 3>(pb, pc, ring_base, S);
+    else expand_mma<2, 4>(pb, pc, ring_base, S);
   }
 }
 
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(const StreamParams P) {
+  extern __shared__ __align__(128) uint8_t dyn_smem[];   // the four warps' rings
   __shared__ SmemExpand S;
   pdl_launch_dependents();
   Area area;
@@ -758,6 +814,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
     return;
   }
   const Area shrink_area = make_area<false>(P);
+  const uint32_t ring_base =
+      smem_addr(dyn_smem) + (uint32_t)((threadIdx.x >> 5) * kRingBytes + (threadIdx.x & 31) * 16);
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
@@ -770,18 +828,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
       S.sh.part_first[ti * kMaxProblems + p] = (int16_t)first;
       S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
     }
-    // the whole batch goes to L2 at once: B rows right away (while the shrink
-    // kernel still runs, for the first batch), y rows once the wait is over
-    walk_batch<true>(P, area, R, S.sh, tb, ntile,
-                     [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, true, waited); });
     if (!waited) {
+      // while the shrink kernel still runs: pull this lane's B rows into L2
+      walk_batch<true>(P, area, R, S.sh, tb, ntile,
+                       [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, true, false); });
       pdl_wait();   // the shrink kernel has completed: v is final, y belongs to this kernel
       waited = true;
-      walk_batch<true>(P, area, R, S.sh, tb, ntile,
-                       [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, false, true); });
     }
     __syncthreads();
-    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, S, pc); });
+    walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { expand_piece(P, S, ring_base, pc); });
   }
 }
 
@@ -805,6 +860,16 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   int32_t lanes = 0;
   int32_t st = mint_device_lanes(&lanes);
   if (st) return st;
+  static bool attrs_set = false;
+  if (!attrs_set) {
+    st = mint_check_cuda(cudaFuncSetAttribute(shrink_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kRingsBytes), "shrink_stream shared memory");
+    if (st) return st;
+    st = mint_check_cuda(cudaFuncSetAttribute(expand_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kRingsBytes), "expand_stream shared memory");
+    if (st) return st;
+    attrs_set = true;
+  }
   const int32_t T = args[0].T;
   const int64_t tiles = mint_tile_upper_bound(1, T, tab.num_slots);
   if (tiles == 0) return MINT_OK;
@@ -839,7 +904,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)lanes);
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = kRingsBytes;
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;

@@ -108,7 +108,7 @@ struct PlanView {
   const LaneStart *lane_expand;
 };
 PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space);
-// Number of cost lanes plans are cut for on the current device (four per SM).
+// Number of cost lanes plans are cut for on the current device (three per SM).
 int32_t mint_device_lanes(int32_t *lanes_out);
 
 // ---- host handles ----------------------------------------------------------
