@@ -419,7 +419,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--layers", type=int, default=0, help="layers per step (0 = the workload's own)")
-    ap.add_argument("--grouping", default="stage", choices=["none", "stage", "layer"],
+    ap.add_argument("--grouping", default="layer", choices=["none", "stage", "layer"],
                     help="how the projections of a layer are grouped into fused calls")
     ap.add_argument("--profile", action="store_true",
                     help="device-timed part only (no end-to-end leg, no CPU oracle): the command profilers wrap")
