@@ -210,6 +210,31 @@ int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *tabl
                               void *y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes,
                               int32_t *status_dev, mint_stream_t stream);
 
+/* Fused apply for callers that cannot allocate device memory.  (No counterpart
+ * in the paper: an addition for embedding this library.)  Some hosts of this
+ * code may not call cudaMalloc or any allocator: a plugin running inside an
+ * engine that has already claimed all device memory for its own pools, code on
+ * a path where allocation is forbidden because it would synchronise the device,
+ * or a process whose memory budget was fixed at start-up.  For them the
+ * workspace of mint_lora_apply_fused lives inside the library, in a fixed array
+ * of MINT_STATIC_WORKSPACE_BYTES that every GPU which loads the library holds
+ * until the process exits; the call allocates and frees nothing.  Inputs,
+ * outputs, plan and status word are the caller's, exactly as for
+ * mint_lora_apply_fused, and the result is the same.
+ *  - A batch whose mint_lora_apply_workspace_bytes(pool, T) exceeds
+ *    MINT_STATIC_WORKSPACE_BYTES is refused with MINT_ERR_WORKSPACE_TOO_SMALL
+ *    and nothing is launched.
+ *  - The first call on each device looks up the array's device address (with
+ *    that device current); make that first call before any stream capture.
+ *  - All calls share the one array, which keeps what the last call left there.
+ *    Nothing in it has to start at zero: every call writes each entry before it
+ *    reads it.  Calls that may overlap on the GPU (two streams, or two threads
+ *    on different streams) race on it: order them on one stream.              */
+#define MINT_STATIC_WORKSPACE_BYTES (8u << 20)
+int32_t mint_lora_apply_fused_static(const mint_pool *pool, const mint_slot_table *table,
+                                     const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
+                                     void *y_dev, int64_t ldy, int32_t *status_dev, mint_stream_t stream);
+
 /* Grouped form: the fused apply of up to MINT_MAX_GROUP projections that share
  * one plan (for instance q, k and v, which read the same x; or gate and up), in
  * one pair of launches.  An adapter's target modules come as a set (the paper's

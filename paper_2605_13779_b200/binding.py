@@ -41,6 +41,7 @@ EXPORTS = [
     "mint_lora_plan_bytes", "mint_lora_plan_layout", "mint_lora_plan", "mint_plan_fetch_summary",
     "mint_lora_shrink", "mint_lora_expand",
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
+    "mint_lora_apply_fused_static",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
 ]
 
@@ -115,6 +116,7 @@ def load_library() -> ctypes.CDLL:
         "mint_lora_apply_workspace_bytes": (sz, [vp, i32]),
         "mint_lora_apply_fused": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, sz, vp, vp]),
         "mint_lora_apply_fused_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, vp, vp]),
+        "mint_lora_apply_fused_static": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
     }
@@ -339,6 +341,21 @@ def mint_lora_apply_fused(pool: Pool, table: SlotTable, plan: Plan, x: torch.Ten
     _check(load_library().mint_lora_apply_fused(
         pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(y), _ld(y, pool.n),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
+    return y
+
+
+MINT_STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def mint_lora_apply_fused_static(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
+                                 status: torch.Tensor) -> torch.Tensor:
+    """The fused apply with the library's built-in workspace: no workspace tensor
+    is passed and nothing is allocated.  For callers that cannot allocate device
+    memory; batches that need more than MINT_STATIC_WORKSPACE_BYTES are refused.
+    Calls share the built-in workspace, so keep them ordered on one stream."""
+    _check(load_library().mint_lora_apply_fused_static(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(y), _ld(y, pool.n),
+        _ptr(status), _stream()))
     return y
 
 

@@ -912,3 +912,37 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   if (st) return st;
   return mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
 }
+
+// ---- fused apply without a caller-provided workspace -------------------------------
+// The workspace of the fused apply, held by the library itself so that a caller
+// that cannot allocate device memory needs none: MINT_STATIC_WORKSPACE_BYTES of
+// every GPU that loads this library, until the process exits.
+static __device__ __align__(256) unsigned char g_static_workspace[MINT_STATIC_WORKSPACE_BYTES];
+
+extern "C" int32_t mint_lora_apply_fused_static(const mint_pool *pool, const mint_slot_table *table,
+                                                const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
+                                                void *y_dev, int64_t ldy, int32_t *status_dev,
+                                                mint_stream_t stream) {
+  if (!pool) return mint_fail(MINT_ERR_INVALID_ARG, "apply_fused_static: null pool");
+  const size_t need = mint_lora_apply_workspace_bytes(pool, T);
+  if (need > (size_t)MINT_STATIC_WORKSPACE_BYTES)
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL,
+                     "apply_fused_static: this batch needs %zu workspace bytes, the built-in workspace has %zu; "
+                     "use mint_lora_apply_fused with a workspace of your own",
+                     need, (size_t)MINT_STATIC_WORKSPACE_BYTES);
+  // The array's name is only a handle on the host: its device address is looked
+  // up once per device, with that device current.
+  static void *address[64] = {nullptr};
+  int dev = 0;
+  int32_t st = mint_check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+  if (st) return st;
+  if (dev < 0 || dev >= 64) return mint_fail(MINT_ERR_UNSUPPORTED, "apply_fused_static: device ordinal %d", dev);
+  if (address[dev] == nullptr) {
+    void *ptr = nullptr;
+    st = mint_check_cuda(cudaGetSymbolAddress(&ptr, g_static_workspace), "address of the built-in workspace");
+    if (st) return st;
+    address[dev] = ptr;
+  }
+  return mint_lora_apply_fused(pool, table, plan_dev, T, x_dev, ldx, y_dev, ldy, address[dev],
+                               (size_t)MINT_STATIC_WORKSPACE_BYTES, status_dev, stream);
+}
