@@ -120,6 +120,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
+__device__ __forceinline__ uint4 zero4() { return make_uint4(0u, 0u, 0u, 0u); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 r;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
@@ -342,24 +343,27 @@ __device__ __forceinline__ void prefetch_piece(const StreamProblem &pb, const Pi
 // shrink
 // ================================================================================
 // Tensor-core body for ranks [rh, rh + 8 NT) of the piece: this warp's blocks.
-template <int MT, int NT>
+// XG = groups of 8 token rows, NT = groups of 8 rank rows: only row groups that
+// exist take a slot of the staging ring, so a skinny tile runs deep.
+template <int XG, int NT>
 __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece &pc, int rh, uint32_t ring_base,
                                            float *scratch) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  constexpr int N = 2 * MT + NT;
+  constexpr int N = XG + NT;
+  constexpr int MT = (XG + 1) / 2;
   Ring<N> ring{ring_base};
   const uint16_t *A_slot = pb.A + (int64_t)pc.slot * pb.r_max * pb.d;
   const uint16_t *src[N];   // this lane's row of every operand fragment (nullptr: the row does not exist)
 #pragma unroll
-  for (int i = 0; i < MT * 2; ++i) {
+  for (int i = 0; i < XG; ++i) {
     const int row = i * 8 + g;
     src[i] = row < pc.len ? pb.x + (int64_t)pc.rows[row] * pb.ldx + t * 8 : nullptr;
   }
 #pragma unroll
   for (int i = 0; i < NT; ++i) {
     const int row = rh + i * 8 + g;
-    src[2 * MT + i] = row < pc.r ? A_slot + (int64_t)row * pb.d + t * 8 : nullptr;
+    src[XG + i] = row < pc.r ? A_slot + (int64_t)row * pb.d + t * 8 : nullptr;
   }
   float acc[MT][NT][4];
 #pragma unroll
@@ -386,11 +390,11 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
   for (int it = 0; it < iters; ++it) {
     issue(it + Ring<N>::kDepth - 1);
     cp_async_wait<Ring<N>::kDepth - 1>();
-    uint4 xa[MT * 2], wb[NT];
+    uint4 xa[2 * MT], wb[NT];
 #pragma unroll
-    for (int i = 0; i < MT * 2; ++i) xa[i] = lds128(ring.slot(it, i));
+    for (int i = 0; i < 2 * MT; ++i) xa[i] = i < XG ? lds128(ring.slot(it, i)) : zero4();
 #pragma unroll
-    for (int i = 0; i < NT; ++i) wb[i] = lds128(ring.slot(it, 2 * MT + i));
+    for (int i = 0; i < NT; ++i) wb[i] = lds128(ring.slot(it, XG + i));
 #pragma unroll
     for (int ks = 0; ks < 2; ++ks)
 #pragma unroll
@@ -483,14 +487,16 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
       else if (pc.len == 2) shrink_vec<2>(pb, pc, ring_base, S.scratch);
       else if (pc.len <= 4) shrink_vec<4>(pb, pc, ring_base, S.scratch);
       else shrink_vec<8>(pb, pc, ring_base, S.scratch);
-    } else if (pc.len <= 16) {
-      if (rr <= 8) shrink_mma<1, 1>(pb, pc, rh, ring_base, S.scratch);
-      else if (rr <= 16) shrink_mma<1, 2>(pb, pc, rh, ring_base, S.scratch);
-      else shrink_mma<1, 4>(pb, pc, rh, ring_base, S.scratch);
     } else {
-      if (rr <= 8) shrink_mma<2, 1>(pb, pc, rh, ring_base, S.scratch);
-      else if (rr <= 16) shrink_mma<2, 2>(pb, pc, rh, ring_base, S.scratch);
-      else shrink_mma<2, 4>(pb, pc, rh, ring_base, S.scratch);
+      const int ng = rr <= 8 ? 1 : (rr <= 16 ? 2 : 4);
+#define MINT_SHRINK_CASE(XG)                                                        \
+  if (ng == 1) shrink_mma<XG, 1>(pb, pc, rh, ring_base, S.scratch);                 \
+  else if (ng == 2) shrink_mma<XG, 2>(pb, pc, rh, ring_base, S.scratch);            \
+  else shrink_mma<XG, 4>(pb, pc, rh, ring_base, S.scratch)
+      if (pc.len <= 8) { MINT_SHRINK_CASE(1); }
+      else if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
+      else { MINT_SHRINK_CASE(4); }
+#undef MINT_SHRINK_CASE
     }
     __syncthreads();
     // add the four warps' sums in warp order; element (l, rh + j) of the [len][rank] result
@@ -566,25 +572,27 @@ __device__ __forceinline__ void update8(uint16_t *yp, const uint4 &old, float sc
   *reinterpret_cast<uint4 *>(yp) = pack8(f);
 }
 
-template <int MT, int KS>
+// YG = groups of 8 token rows (two 16-byte segments of y each), KG = groups of 8
+// rank rows of B (rows 8 kg + 2t and 8 kg + 2t + 1): only groups that exist take
+// slots of the staging ring.
+template <int YG, int KG>
 __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
                                            const SmemExpand &S) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  constexpr int N = 4 * KS + 4 * MT;
+  constexpr int N = 2 * KG + 2 * YG;
+  constexpr int MT = (YG + 1) / 2, KS = (KG + 1) / 2;
   Ring<N> ring{ring_base};
   const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
-  // this lane's segments of a block: B rows 2t, 2t+1, 2t+8, 2t+9 of every k-step at column 8 g,
-  // then 16 columns of y at column 16 t for rows g, g + 8 of every m-tile
-  const uint16_t *bsrc[4 * KS];
-  uint16_t *ysrc[2 * MT];
+  const uint16_t *bsrc[2 * KG];
+  uint16_t *ysrc[YG];
 #pragma unroll
-  for (int i = 0; i < 4 * KS; ++i) {
-    const int k = (i >> 2) * 16 + 2 * t + (i & 1) + ((i >> 1) & 1) * 8;
+  for (int i = 0; i < 2 * KG; ++i) {
+    const int k = (i >> 1) * 8 + 2 * t + (i & 1);
     bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + g * 8 : nullptr;
   }
 #pragma unroll
-  for (int i = 0; i < 2 * MT; ++i) {
+  for (int i = 0; i < YG; ++i) {
     const int row = i * 8 + g;
     ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 16 : nullptr;
   }
@@ -596,12 +604,12 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
       const bool ok_b = n0 + g * 8 < pb.n;
       const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;
 #pragma unroll
-      for (int i = 0; i < 4 * KS; ++i)
+      for (int i = 0; i < 2 * KG; ++i)
         cp_async16(ring.slot(it, i), bsrc[i] ? bsrc[i] + n0 : pb.B, ok_b && bsrc[i]);
 #pragma unroll
-      for (int i = 0; i < 2 * MT; ++i) {
-        cp_async16(ring.slot(it, 4 * KS + 2 * i), ysrc[i] ? ysrc[i] + n0 : pb.B, ok_y0 && ysrc[i]);
-        cp_async16(ring.slot(it, 4 * KS + 2 * i + 1), ysrc[i] ? ysrc[i] + n0 + 8 : pb.B, ok_y1 && ysrc[i]);
+      for (int i = 0; i < YG; ++i) {
+        cp_async16(ring.slot(it, 2 * KG + 2 * i), ysrc[i] ? ysrc[i] + n0 : pb.B, ok_y0 && ysrc[i]);
+        cp_async16(ring.slot(it, 2 * KG + 2 * i + 1), ysrc[i] ? ysrc[i] + n0 + 8 : pb.B, ok_y1 && ysrc[i]);
       }
     }
     cp_async_commit();
@@ -623,9 +631,11 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
         for (int e = 0; e < 4; ++e) acc[j][e] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < KS; ++ks) {
+        // B rows 2t, 2t+1 (group 2 ks) and 2t+8, 2t+9 (group 2 ks + 1) of this k-step
         uint4 bq[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) bq[i] = lds128(ring.slot(it, 4 * ks + i));
+        for (int i = 0; i < 4; ++i)
+          bq[i] = (2 * ks + (i >> 1) < KG) ? lds128(ring.slot(it, 2 * (2 * ks + (i >> 1)) + (i & 1))) : zero4();
         const uint4 vh = S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + lane];
         const uint4 vl = S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + lane];
 #pragma unroll
@@ -641,11 +651,13 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
       // acc[j][0], [1]: row g, columns 16 t + j and 16 t + 8 + j; acc[j][2], [3]: row g + 8
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
-        uint16_t *yr = ysrc[2 * mt + h];
-        if (yr) {
-          if (ok_y0) update8(yr + n0, lds128(ring.slot(it, 4 * KS + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
-          if (ok_y1)
-            update8(yr + n0 + 8, lds128(ring.slot(it, 4 * KS + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
+        if (2 * mt + h < YG) {
+          uint16_t *yr = ysrc[2 * mt + h];
+          if (yr) {
+            if (ok_y0) update8(yr + n0, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
+            if (ok_y1)
+              update8(yr + n0 + 8, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
+          }
         }
       }
     }
@@ -756,7 +768,10 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   const bool vec = pc.r == 1 && pc.len <= 8;
   const int first = S.sh.part_first[pc.ti * kMaxProblems + pc.p];
   const int count = S.sh.part_count[pc.ti * kMaxProblems + pc.p];
-  const int MT = (pc.len + 15) >> 4, KS = (pc.r + 15) >> 4;
+  // row groups as the tensor-core body is instantiated: 1, 2 or 4 groups of 8 tokens; 1, 2, 4 or 8 of 8 ranks
+  const int yg = pc.len <= 8 ? 1 : (pc.len <= 16 ? 2 : 4);
+  const int kg = pc.r <= 8 ? 1 : (pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8));
+  const int MT = (yg + 1) >> 1, KS = (kg + 1) >> 1;
   __syncthreads();   // the previous piece no longer reads v
   if (vec) {
     if (tid < 8) S.vvec[tid] = tid < pc.len ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, tid) : 0.f;
@@ -787,16 +802,16 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
     else if (pc.len == 2) expand_vec<2>(pb, pc, ring_base, S);
     else if (pc.len <= 4) expand_vec<4>(pb, pc, ring_base, S);
     else expand_vec<8>(pb, pc, ring_base, S);
-  } else if (MT == 1) {
-    if (KS == 1) expand_mma<1, 1>(pb, pc, ring_base, S);
-    else if (KS == 2) expand_mma<1, 2>(pb, pc, ring_base, S);
-    else if (KS == 3) expand_mma<1, 3>(pb, pc, ring_base, S);
-    else expand_mma<1, 4>(pb, pc, ring_base, S);
   } else {
-    if (KS == 1) expand_mma<2, 1>(pb, pc, ring_base, S);
-    else if (KS == 2) expand_mma<2, 2>(pb, pc, ring_base, S);
-    else if (KS == 3) expand_mma<2, 3>(pb, pc, ring_base, S);
-    else expand_mma<2, 4>(pb, pc, ring_base, S);
+#define MINT_EXPAND_CASE(YG)                                        \
+  if (kg == 1) expand_mma<YG, 1>(pb, pc, ring_base, S);             \
+  else if (kg == 2) expand_mma<YG, 2>(pb, pc, ring_base, S);        \
+  else if (kg == 4) expand_mma<YG, 4>(pb, pc, ring_base, S);        \
+  else expand_mma<YG, 8>(pb, pc, ring_base, S)
+    if (yg == 1) { MINT_EXPAND_CASE(1); }
+    else if (yg == 2) { MINT_EXPAND_CASE(2); }
+    else { MINT_EXPAND_CASE(4); }
+#undef MINT_EXPAND_CASE
   }
 }
 
