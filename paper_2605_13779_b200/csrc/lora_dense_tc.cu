@@ -1,0 +1,328 @@
+// Tensor-core shrink for dense segments:  v[128-row tile] = X[tile rows, :] . A_slot^T   (d -> r).
+//
+// A segmented-prefill batch holds runs of hundreds of tokens of one adapter; for
+// those the d -> r contraction is a genuinely dense [128 x d] . [d x r] product
+// per 128-token tile, and it runs on the fifth-generation tensor cores:
+// tcgen05.mma (M = 128, N = the rank rounded up to 16, K = 16 per instruction,
+// bf16 operands, fp32 accumulators in tensor memory), issued by one thread of
+// the CTA.  Both operands have the reduction index contiguous in memory (rows
+// of x, rows of A[slot][rank][d]), the K-major case of the MMA.
+//
+// One CTA per 128-row tile walks d in chunks of 64 columns.  A chunk of the token
+// rows (128 x 128 bytes) and of the rank rows (N x 128 bytes) is copied into a
+// shared-memory stage with 16-byte asynchronous copies, eight consecutive
+// threads per row, in the 128-byte-swizzled layout the MMA's shared-memory
+// descriptors name (16-byte chunk c of row i at chunk c ^ (i & 7) of its row,
+// rows in groups of 8 x 128 bytes).  Four stages are in flight; a stage is
+// refilled once the MMAs that read it have signalled an mbarrier
+// (tcgen05.commit).  After the last chunk every warp reads its 32 accumulator
+// rows out of tensor memory (tcgen05.ld) and writes them, fp32, to the slots of
+// the workspace from which the expand kernel takes v: a region of slots of its
+// own, one per 32-token sub-tile (the streamed shrink skips these tiles).
+//
+// Every wait on an mbarrier is bounded; a wait that runs out records
+// MINT_ERR_TIMEOUT, and the CTA still frees its tensor memory before it returns.
+#include "mint_device.cuh"
+
+using namespace mint;
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kTileRows = 128;          // M of the MMA
+constexpr int kChunk = 64;              // columns of d per stage: one 128-byte swizzle atom per row
+constexpr int kStages = 4;
+constexpr int kMaxRank = 64;            // N <= 64
+constexpr int kXStageBytes = kTileRows * 128;
+constexpr int kAStageBytes = kMaxRank * 128;
+constexpr int kStageBytes = kXStageBytes + kAStageBytes;   // 24 KB
+constexpr int kTmemCols = 64;
+constexpr size_t kDynSmem = (size_t)kStages * kStageBytes + 1024;   // + alignment slack
+constexpr int kMaxProblems = MINT_MAX_GROUP;
+
+struct DenseProblem {
+  const uint16_t *A;   // [slot][r_max][d]
+  const uint16_t *x;
+  int64_t ldx;
+  int32_t d, r_max;
+  float *ws_part;      // slots of 32 * r_max floats, [len][rank] packed fp32
+};
+
+struct DenseParams {
+  DenseProblem prob[kMaxProblems];
+  int32_t T;
+  int32_t lanes;
+  int32_t dense_slot0;   // the v of dense tile t goes to workspace slot dense_slot0 + t
+  int32_t *status;
+  TableDev tab;
+  PlanView pv;
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid) {
+  const int bytes = valid ? 16 : 0;   // 0: nothing is read, the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait for the phase with the given parity; false after about a second.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  const uint32_t a = smem_addr(bar);
+  uint64_t t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(a), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if ((it & 63u) == 63u) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {   // one whole warp
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(dst_smem)), "r"(cols)
+               : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {     // one whole warp
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 in, fp32 accumulate; one thread issues
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          bool accumulate) {
+  const uint32_t acc = accumulate ? 1u : 0u;
+  const uint32_t zero = 0u;   // no output lane is disabled
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc), "r"(zero)
+      : "memory");
+}
+// the mbarrier gets one arrival when all MMAs issued so far by this thread have completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_addr(bar))
+               : "memory");
+}
+// 16 consecutive fp32 columns of this thread's accumulator row
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand tile in the
+// 128-byte-swizzled layout: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFFu);        // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                        // leading byte offset (not used by swizzled K-major layouts)
+  d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                        // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                        // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DenseParams P) {
+  extern __shared__ uint8_t dyn_raw[];
+  __shared__ uint64_t mma_done[kStages];
+  __shared__ uint64_t all_done;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int32_t rows[kTileRows];
+  __shared__ int32_t failed;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const DenseProblem &pb = P.prob[blockIdx.y];
+
+  pdl_launch_dependents();
+  // The plan and the pool weights were complete before this call's kernels
+  // started; activations and the workspace are touched only after the wait.
+  const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
+                  P.pv.header[PH_LANES] == P.lanes;
+  const int m = blockIdx.x;
+  if (!ok || m >= P.pv.header[PH_NUM_DENSE]) {
+    pdl_wait();
+    return;
+  }
+  const int ntiles = P.pv.header[PH_NCHUNK1];
+  const int t0 = P.pv.dense_tile[m];
+  const TileDesc d0 = P.pv.tile_desc[t0];
+  // the 128-row tile = up to four consecutive 32-token tiles of the segment
+  int nrows = d0.len;
+  for (int i = 1; i < 4 && nrows == 32 * i && t0 + i < ntiles; ++i) {
+    const TileDesc di = P.pv.tile_desc[t0 + i];
+    if (!di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
+    nrows += di.len;
+  }
+  const int r = d0.rank;
+  if (r > pb.r_max || r > kMaxRank || r < 1) {
+    if (tid == 0) report(P.status, MINT_ERR_RANK_TOO_LARGE, d0.slot);
+    pdl_wait();
+    return;
+  }
+  const int n_mma = (r + 15) / 16 * 16;
+  for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&mma_done[s], 1);
+    mbar_init(&all_done, 1);
+    fence_mbar_init();
+    failed = 0;
+  }
+  if (warp == 0) tmem_alloc(&tmem_base_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = tmem_base_slot;
+  const uint32_t stage0 = (smem_addr(dyn_raw) + 1023u) & ~1023u;   // swizzle atoms are 1024-byte aligned
+  const uint16_t *A_rows = pb.A + (int64_t)d0.slot * pb.r_max * pb.d;
+  const uint32_t idesc = instr_desc(n_mma);
+  const int nchunks = (pb.d + kChunk - 1) / kChunk;
+
+  pdl_wait();
+
+  // this thread's 16-byte pieces of a stage: row q >> 3, chunk q & 7 for q = tid + 128 i
+  auto issue = [&](int kc) {
+    if (kc < nchunks) {
+      const uint32_t xs = stage0 + (uint32_t)((kc % kStages) * kStageBytes), as = xs + kXStageBytes;
+      const int c = tid & 7;
+      const int col = kc * kChunk + c * 8;
+      const bool col_ok = col < pb.d;
+#pragma unroll
+      for (int i = 0; i < kTileRows / 16; ++i) {
+        const int row = (tid >> 3) + 16 * i;
+        const bool v = col_ok && row < nrows;
+        cp_async16(xs + (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((c ^ (row & 7)) << 4)),
+                   v ? pb.x + (int64_t)rows[row] * pb.ldx + col : pb.x, v);
+      }
+      for (int row = tid >> 3; row < n_mma; row += 16) {
+        const bool v = col_ok && row < r;
+        cp_async16(as + (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((c ^ (row & 7)) << 4)),
+                   v ? A_rows + (int64_t)row * pb.d + col : pb.A, v);
+      }
+    }
+    cp_async_commit();
+  };
+
+  for (int kc = 0; kc < kStages - 1; ++kc) issue(kc);
+  for (int kc = 0; kc < nchunks; ++kc) {
+    const int s = kc % kStages;
+    cp_async_wait<kStages - 2>();   // this thread's copies of chunk kc have landed
+    fence_async_smem();             // ... and are visible to the tensor core's reads of shared memory
+    __syncthreads();
+    if (tid == 0 && !failed) {
+      tc_fence_after();
+      const uint32_t xs = stage0 + (uint32_t)(s * kStageBytes), as = xs + kXStageBytes;
+      const uint64_t da = smem_desc_k_sw128(xs), db = smem_desc_k_sw128(as);
+#pragma unroll
+      for (int ks = 0; ks < kChunk / 16; ++ks)   // 16 columns = 32 bytes further along the swizzled rows
+        umma_bf16(tmem_d, da + (uint64_t)(2 * ks), db + (uint64_t)(2 * ks), idesc, kc > 0 || ks > 0);
+      umma_commit(&mma_done[s]);
+    }
+    // chunk kc + kStages - 1 reuses the stage of chunk kc - 1: wait for the MMAs that read it
+    if (!failed && kc >= 1 && kc + kStages - 1 < nchunks) {
+      const int sp = (kc - 1) % kStages;
+      if (!mbar_wait(&mma_done[sp], ((kc - 1) / kStages) & 1u)) failed = 1;
+    }
+    issue(kc + kStages - 1);
+  }
+  cp_async_wait<0>();
+  if (tid == 0) umma_commit(&all_done);
+  if (!failed && !mbar_wait(&all_done, 0)) failed = 1;
+  tc_fence_after();
+  __syncthreads();
+  if (!failed) {
+    // warp w owns accumulator rows 32 w .. 32 w + 31 (tensor-memory lanes), one row per thread
+    const int row = warp * 32 + lane;
+    const size_t slot_floats = (size_t)32 * pb.r_max;
+    float *dst = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
+    for (int j0 = 0; j0 < n_mma; j0 += 16) {
+      float v[16];
+      tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, v);
+      if (row < nrows) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j0 + j < r) dst[j0 + j] = v[j];
+      }
+    }
+  } else if (tid == 0) {
+    report(P.status, MINT_ERR_TIMEOUT, m);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_d, kTmemCols);
+}
+
+}  // namespace
+
+int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                      (int)kDynSmem), "dense_shrink shared memory");
+    if (st) return st;
+    attr_set = true;
+  }
+  const int32_t T = args[0].T;
+  const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
+  if (tiles == 0) return MINT_OK;
+  DenseParams P = {};
+  for (int i = 0; i < nprob; ++i) {
+    DenseProblem &pb = P.prob[i];
+    pb.A = args[i].A;
+    pb.x = args[i].x;
+    pb.ldx = args[i].ldx;
+    pb.d = args[i].d;
+    pb.r_max = args[i].r_max;
+    pb.ws_part = static_cast<float *>(workspaces[i]);
+  }
+  P.T = T;
+  P.lanes = lanes;
+  P.dense_slot0 = dense_slot0;
+  P.status = args[0].status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)nprob);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kDynSmem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_shrink_kernel, P), "dense_shrink launch");
+}

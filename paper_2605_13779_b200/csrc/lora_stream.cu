@@ -84,7 +84,8 @@ struct StreamProblem {
   int64_t ldx, ldy;
   int32_t d, n, r_max;
   int32_t cb0_shrink, cb0_expand;  // first virtual column block of this problem
-  float *ws_part;      // [tiles_ub + lanes][32 * r_max]  slot (tile + lane): that lane's sum, [len][rank] packed
+  float *ws_part;      // [2 tiles_ub + lanes][32 * r_max]  slot (tile + lane): that lane's sum, [len][rank] packed;
+                       // slot (tiles_ub + lanes + tile): the v of a dense segment's tile
 };
 
 struct StreamParams {
@@ -94,6 +95,7 @@ struct StreamParams {
   int32_t lanes;                      // grid size = the plan's lane count
   int32_t cb_shrink, cb_expand;       // virtual column blocks of the whole call
   int32_t cb_shrink_widest;           // column blocks of the widest d of the call
+  int32_t dense_slot0;                // first workspace slot of the dense segments' tiles (slot dense_slot0 + tile)
   int32_t *status;
   TableDev tab;
   PlanView pv;
@@ -212,7 +214,7 @@ struct CtaRange {
 struct CtaShared {
   TileDesc desc[kBatchTiles];
   int32_t rows[kBatchItems];
-  int16_t part_first[kBatchTiles * kMaxProblems];   // expand: first shrink lane holding a part of (tile, problem)
+  int32_t part_first[kBatchTiles * kMaxProblems];   // expand: first shrink lane holding a part of (tile, problem)
   int16_t part_count[kBatchTiles * kMaxProblems];   //         and how many consecutive lanes do
   int32_t range[4];
 };
@@ -288,6 +290,7 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     const int va = (t == R.t0) ? R.cb0 : 0;
     const int vb = (t == R.t1) ? R.cb1 : area.CB;
     if (va >= vb) continue;
+    if (!kExpand && sh.desc[ti].dense) continue;   // its shrink runs on the 128-row tensor-core kernel
     Piece pc;
     pc.t = t;
     pc.ti = ti;
@@ -730,6 +733,11 @@ __device__ __forceinline__ void shrink_parts(const StreamParams &P, const Area &
   const int c_b = (int)(((unsigned)(d.lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
   first = 0;
   count = 0;
+  if (d.dense) {   // the tensor-core shrink leaves the complete v of the tile in the slot dense_slot0 + tile
+    first = P.dense_slot0;
+    count = 1;
+    return;
+  }
   int64_t p0 = lane_offset(sa, sa.table[lane_index(sa, c_a)], d.rows_shrink);
   for (int c2 = c_a; c2 <= c_b; ++c2) {
     const int64_t p1 = lane_offset(sa, sa.table[lane_index(sa, c2 + 1)], d.rows_shrink);
@@ -840,7 +848,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
       const int ti = i / P.nprob, p = i - ti * P.nprob;
       int first, count;
       shrink_parts(P, shrink_area, S.sh.desc[ti], p, first, count);
-      S.sh.part_first[ti * kMaxProblems + p] = (int16_t)first;
+      S.sh.part_first[ti * kMaxProblems + p] = first;
       S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
     }
     if (!waited) {
@@ -857,7 +865,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
 
 // ---- host side -----------------------------------------------------------------
 size_t workspace_bytes(int64_t tiles, int32_t r_max) {
-  return (size_t)(tiles + MINT_MAX_LANES) * kTileRowsMax * r_max * sizeof(float) + 256;
+  return (size_t)(2 * tiles + MINT_MAX_LANES) * kTileRowsMax * r_max * sizeof(float) + 256;
 }
 
 }  // namespace
@@ -909,6 +917,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   P.cb_shrink = cb_s;
   P.cb_expand = cb_e;
   P.cb_shrink_widest = cb_widest;
+  P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
   P.status = args[0].status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
@@ -925,6 +934,10 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   cfg.numAttrs = 1;
   st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel, P), "shrink_stream launch");
   if (st) return st;
+  if (T >= MINT_DENSE_MIN_BATCH) {   // the plan may have given dense segments to the tensor-core shrink
+    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);
+    if (st) return st;
+  }
   return mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
 }
 

@@ -32,7 +32,8 @@ enum {
   PH_LANES,     // number of cost lanes G the lane tables were cut for
   PH_ROWS_SHRINK,  // sum over list-1 tiles of (rank + len)
   PH_ROWS_EXPAND,  // sum over list-1 tiles of (rank + 2 len)
-  PH_MAX_TILE_ROWS,  // largest (rank + len) of a list-1 tile
+  PH_MAX_TILE_ROWS,  // largest (rank + len) of a list-1 tile that the streamed shrink handles
+  PH_NUM_DENSE,      // number of 128-row tiles of dense segments (tensor-core shrink)
   PH_WORDS = 32
 };
 #define MINT_PLAN_MAGIC 0x4D4C5032  // "MLP2"
@@ -60,8 +61,17 @@ struct __align__(16) TileDesc {
   int32_t rows_expand;
   int32_t lane_lo;
   int32_t lane_hi;
-  int32_t pad0, pad1;
+  int32_t dense;   // 1: the tile belongs to a dense segment; its shrink runs on the 128-row tensor-core kernel
+  int32_t pad1;
 };
+
+// A batch of at least MINT_DENSE_MIN_BATCH items may hold dense segments: runs of
+// at least MINT_DENSE_MIN_SEGMENT items of one adapter (segmented prefill).  Their
+// shrink (the d -> r contraction over 128-row tiles) runs on the tcgen05 kernel;
+// the plan excludes their tiles from the streamed shrink's area and lists the
+// 128-row tiles (every fourth 32-item tile of such a segment) in dense_tile.
+#define MINT_DENSE_MIN_BATCH 4096
+#define MINT_DENSE_MIN_SEGMENT 128
 
 // Start of cost lane j in the rows x column-blocks area: the tile that holds it
 // and j * rows_total = q * G + r, so that the position for CB column blocks is
@@ -84,6 +94,7 @@ struct PlanOffsets {
   int64_t tile_seg[MINT_NUM_TILE_LISTS];  // int32[P]  segment of tile c
   int64_t tile_off[MINT_NUM_TILE_LISTS];  // int32[P]  first position (in perm) of tile c
   int64_t tile_desc;   // TileDesc[tile upper bound of list 1]
+  int64_t dense_tile;  // int32[tile upper bound of list 1]  first list-1 tile of every 128-row dense tile
   int64_t lane_shrink; // LaneStart[MINT_MAX_LANES + 1]  start of cost lane j in the shrink rows
   int64_t lane_expand; // LaneStart[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
@@ -104,6 +115,7 @@ struct PlanView {
   const int32_t *tile_seg[MINT_NUM_TILE_LISTS];
   const int32_t *tile_off[MINT_NUM_TILE_LISTS];
   const TileDesc *tile_desc;
+  const int32_t *dense_tile;
   const LaneStart *lane_shrink;
   const LaneStart *lane_expand;
 };
@@ -172,6 +184,9 @@ int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *p
 // shrink and one expand launch cover up to 8 projections that share a plan.
 bool mint_stream_supported(int32_t max_bound_rank);
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);
+// Tensor-core shrink of the dense segments' 128-row tiles (between the two streamed kernels).
+int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s);
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);
 

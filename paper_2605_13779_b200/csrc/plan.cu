@@ -267,23 +267,33 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   LaneStart *lane_tab[2] = {reinterpret_cast<LaneStart *>(p.blob + p.off.lane_shrink),
                             reinterpret_cast<LaneStart *>(p.blob + p.off.lane_expand)};
   int rows_total[2];
+  int num_dense = 0;
   {
     const int32_t *tseg = reinterpret_cast<const int32_t *>(p.blob + p.off.tile_seg[1]);
     const int32_t *toff = reinterpret_cast<const int32_t *>(p.blob + p.off.tile_off[1]);
     const int ntile = tile_total[1];
     const int per = (ntile + kThreads - 1) / kThreads;
     const int c_begin = min(ntile, tid * per), c_end = min(ntile, (tid + 1) * per);
-    int sum_s = 0, sum_e = 0;
+    // dense segments (segmented prefill): dense plans of large batches only
+    const bool dense_on = p.expert_ids == nullptr && P >= MINT_DENSE_MIN_BATCH;
+    auto is_dense = [&](int sg) { return dense_on && seg_start[sg + 1] - seg_start[sg] >= MINT_DENSE_MIN_SEGMENT; };
+    int sum_s = 0, sum_e = 0, sum_m = 0;
     for (int c = c_begin; c < c_end; ++c) {
       const int sg = tseg[c];
       const int len = min(mint_tile_tokens(1), seg_start[sg + 1] - toff[c]);
       const int r = p.tab.slot_rank[seg_slot[sg]];
-      sum_s += r + len;
+      if (is_dense(sg)) {
+        sum_m += ((toff[c] - seg_start[sg]) % 128) == 0;
+      } else {
+        sum_s += r + len;
+        atomicMax(&counters[7], r + len);
+      }
       sum_e += r + 2 * len;
-      atomicMax(&counters[7], r + len);
     }
     int run_s = block_exclusive_scan(sum_s, warp_tot, rows_total[0]);
     int run_e = block_exclusive_scan(sum_e, warp_tot, rows_total[1]);
+    int run_m = block_exclusive_scan(sum_m, warp_tot, num_dense);
+    int32_t *dense_tile = reinterpret_cast<int32_t *>(p.blob + p.off.dense_tile);
     const int64_t G = p.lanes;
     for (int c = c_begin; c < c_end; ++c) {
       const int sg = tseg[c];
@@ -297,18 +307,24 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       dsc.scale = p.tab.slot_scale[slot];
       dsc.rows_shrink = run_s;
       dsc.rows_expand = run_e;
+      dsc.dense = is_dense(sg) ? 1 : 0;
+      if (dsc.dense && ((toff[c] - seg_start[sg]) % 128) == 0) dense_tile[run_m++] = c;
       const int begin[2] = {run_s, run_e};
-      const int end[2] = {run_s + dsc.rank + dsc.len, run_e + dsc.rank + 2 * dsc.len};
+      const int end[2] = {run_s + (dsc.dense ? 0 : dsc.rank + dsc.len), run_e + dsc.rank + 2 * dsc.len};
       // shrink lanes that can meet this tile: from the last lane starting at or
       // before the tile's first row to the last lane starting before its end
-      dsc.lane_lo = (int32_t)(begin[0] * G / rows_total[0]);
-      dsc.lane_hi = (int32_t)min(G - 1, (end[0] * G - 1) / rows_total[0]);
-      dsc.pad0 = dsc.pad1 = 0;
+      dsc.lane_lo = dsc.lane_hi = 0;
+      if (!dsc.dense) {
+        dsc.lane_lo = (int32_t)(begin[0] * G / rows_total[0]);
+        dsc.lane_hi = (int32_t)min(G - 1, (end[0] * G - 1) / rows_total[0]);
+      }
+      dsc.pad1 = 0;
       desc[c] = dsc;
       // lanes whose start falls inside this tile: rows[c]*G <= j*total < rows[c+1]*G
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         const int64_t tot = rows_total[q];
+        if (tot == 0 || begin[q] == end[q]) continue;
         const int64_t j_lo = (begin[q] * G + tot - 1) / tot;
         const int64_t j_hi = (end[q] * G + tot - 1) / tot;   // exclusive
         for (int64_t j = j_lo; j < j_hi && j < G; ++j) lane_tab[q][j].tile = c;
@@ -323,7 +339,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
         lane_tab[q][j].q = (int32_t)(jw / G);
         lane_tab[q][j].r = (int32_t)(jw % G);
         lane_tab[q][j].pad = 0;
-        if (j == p.lanes || ntile == 0) lane_tab[q][j].tile = (j == p.lanes) ? ntile : 0;
+        if (j == p.lanes || rows_total[q] == 0) lane_tab[q][j].tile = (j == p.lanes) ? ntile : 0;
       }
     }
   }
@@ -350,7 +366,8 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     hdr[PH_ROWS_SHRINK] = rows_total[0];
     hdr[PH_ROWS_EXPAND] = rows_total[1];
     hdr[PH_MAX_TILE_ROWS] = counters[7];
-    for (int w = PH_MAX_TILE_ROWS + 1; w < PH_WORDS; ++w) hdr[w] = 0;
+    hdr[PH_NUM_DENSE] = num_dense;
+    for (int w = PH_NUM_DENSE + 1; w < PH_WORDS; ++w) hdr[w] = 0;
     if (counters[1] > 0) {
       mint::report(p.status, MINT_ERR_NOT_RESIDENT, counters[2]);
       if (p.status) atomicAdd(&p.status[1], counters[1]);
@@ -383,6 +400,7 @@ PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
     o.tile_off[g] = take(n);
   }
   o.tile_desc = take((mint_tile_upper_bound(1, P, key_space) + 1) * (int64_t)(sizeof(TileDesc) / 4));
+  o.dense_tile = take(mint_tile_upper_bound(1, P, key_space) + 1);
   o.lane_shrink = take((MINT_MAX_LANES + 1) * (int64_t)(sizeof(LaneStart) / 4));
   o.lane_expand = take((MINT_MAX_LANES + 1) * (int64_t)(sizeof(LaneStart) / 4));
   o.key_a = take(n);
@@ -415,6 +433,7 @@ PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space) {
     v.tile_off[g] = reinterpret_cast<const int32_t *>(b + o.tile_off[g]);
   }
   v.tile_desc = reinterpret_cast<const TileDesc *>(b + o.tile_desc);
+  v.dense_tile = reinterpret_cast<const int32_t *>(b + o.dense_tile);
   v.lane_shrink = reinterpret_cast<const LaneStart *>(b + o.lane_shrink);
   v.lane_expand = reinterpret_cast<const LaneStart *>(b + o.lane_expand);
   return v;

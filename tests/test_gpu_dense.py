@@ -193,3 +193,45 @@ def test_grouped_call_equals_separate_calls():
         twice = harness.y_to_f64(dv.y)
         delta = y_ref - synth.bf16_bits_to_f64(c.y0)
         assert np.abs(twice - (y_ref + delta)).max() <= 6e-2
+
+
+def dense_segment_case(name, lengths, adapters, ranks, d, n, r_max):
+    """Requests of the given lengths, request i bound to adapters[i]; tokens of a
+    request are contiguous, an adapter may own several requests."""
+    num_slots = len(ranks)
+    table = synth.identity_table(num_slots, np.asarray(ranks, dtype=np.int32), 2.0)
+    ids = np.repeat(np.asarray(adapters, dtype=np.int64), np.asarray(lengths, dtype=np.int64))
+    T = int(ids.shape[0])
+    A, B = synth.dense_pool(synth.stream(name, "pool"), table, r_max, d, n)
+    x = synth.normal_bf16(synth.stream(name, "x"), (T, d), 1.0)
+    y0 = synth.normal_bf16(synth.stream(name, "y0"), (T, n), 1.0)
+    return synth.DenseCase(name, T, d, n, r_max, table, ids, A, B, x, y0)
+
+
+def test_dense_segments_take_the_tensor_core_shrink():
+    """A batch of more than 4096 tokens with segments of 128 tokens and more: their
+    shrink runs on the tcgen05 kernel (full and ragged 128-row tiles, ranks that are
+    not multiples of 16, an adapter whose tokens are not contiguous), short segments
+    and tokens without adapter stay on the streamed path."""
+    lengths = [700, 130, 128, 127, 300, 5, 1, 1000, 64, 513, 256, 129, 3, 640, 384, 40]
+    adapters = [0, 1, 2, 3, 4, 5, 6, 7, 8, 0, 9, 10, -1, 11, 12, 6]
+    ranks = [64, 16, 8, 33, 1, 4, 32, 64, 16, 48, 5, 64, 17]
+    case = dense_segment_case("gpu/dense-tc", lengths, adapters, ranks, d=1032, n=520, r_max=64)
+    assert case.T >= 4096
+    check_case(case, "dense segments")
+
+
+def test_dense_segments_config3_shape_sampled():
+    """One config-3 projection at full size on the tensor-core shrink, checked on sampled rows."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    batch = synth.config3_batch()
+    case = synth.config3_projection(batch, 5120, 5120)
+    y, status, _ = run_fused(case)
+    assert status[0] == 0, status
+    rng = synth.stream("gpu/dense-tc/sample")
+    rows = np.sort(rng.choice(case.T, size=96, replace=False))
+    # include the first and last token of some requests (tile edges)
+    edges = np.cumsum(batch.lengths)
+    rows = np.unique(np.concatenate([rows, edges[:8] - 1, edges[:8] % case.T]))
+    y_ref, _, _ = parity.oracle_dense(case, rows=rows)
+    parity.assert_close(y[rows], y_ref, "config3 sampled rows")
