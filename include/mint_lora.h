@@ -200,10 +200,13 @@ int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table *table, co
  * Same result as shrink followed by expand (fp32 accumulation, summation order
  * may differ).  The shrink result never goes to HBM as a tensor of its own: it
  * crosses from the shrink stage to the expand stage through workspace_dev, a
- * few KB per tile that stay in L2.  workspace_dev: at least
- * mint_lora_apply_workspace_bytes(pool, T) bytes, 256-byte aligned, ZERO-FILLED
- * by the caller before its first use; every call leaves it ready for the next
- * one.  Calls that share a workspace must be ordered on one stream.           */
+ * few MB that stay in L2.  workspace_dev: at least
+ * mint_lora_apply_workspace_bytes(pool, T) bytes, 256-byte aligned; it needs no
+ * initialisation (every call writes each entry before it reads it).  Calls
+ * that share a workspace must be ordered on one stream.  Batches of 4096 tokens
+ * and more whose plan holds runs of 128 and more tokens of one adapter
+ * (segmented prefill) run the d -> r contraction of those runs on the tcgen05
+ * tensor cores; the result is the same.                                        */
 size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T);
 int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table,
                               const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
