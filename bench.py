@@ -243,7 +243,8 @@ def run_gpu(args):
         groups_idx = [list(range(ncase))]
     else:
         groups_idx = [[0, 1, 2], [3], [4, 5], [6]] if ncase == 7 else [[i] for i in range(ncase)]
-    workspaces = None if moe else [mb.new_workspace(dv.pool, T) for dv in base]
+    workspaces = ([mb.new_moe_workspace(dv.pool, T, wl["cases"][0].K) for dv in base] if moe
+                  else [mb.new_workspace(dv.pool, T) for dv in base])
     groups = []
     if not moe:
         for row in layers:
@@ -253,7 +254,8 @@ def run_gpu(args):
     def enqueue_layer(li):
         if moe:
             for ci, (pool, x, y) in enumerate(layers[li]):
-                mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row)
+                mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row,
+                                       workspace=workspaces[ci])
         else:
             for grp in groups[li]:
                 mb.mint_lora_apply_fused_grouped(grp, table, plan, status)
@@ -262,7 +264,7 @@ def run_gpu(args):
         for li in range(L):
             enqueue_layer(li)
 
-    kernels_per_call = 1 if moe else 2          # the dense fused call is a shrink and an expand launch
+    kernels_per_call = 2                        # a fused call is a shrink and an expand launch
     calls_per_layer = len(groups_idx)
     launches_per_step = 1 + L * calls_per_layer * kernels_per_call
 
@@ -378,7 +380,7 @@ def run_gpu(args):
     avg_launch_s = ms_apply * 1e-3 / args.steps / n_apply
     avg_launch_bytes = layer_bytes / calls_per_layer
     achieved = avg_launch_bytes / avg_launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "moe_kernel" if moe else "shrink_stream_kernel+expand_stream_kernel",
+    roofline = {"bound": "hbm", "kernel": "shrink_stream_kernel+expand_stream_kernel",
                 "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_8TBps": achieved / 8000.0, "peak_source": peak_src,
                 "bytes_per_launch": avg_launch_bytes, "avg_launch_us": avg_launch_s * 1e6,

@@ -382,6 +382,12 @@ def mint_moe_lora_apply_workspace_bytes(pool: Pool, T: int, K: int) -> int:
     return int(load_library().mint_moe_lora_apply_workspace_bytes(pool.handle, T, K))
 
 
+def new_moe_workspace(pool: Pool, T: int, K: int, device="cuda") -> torch.Tensor:
+    """Workspace of the MoE apply for one projection; it needs no initialisation."""
+    nbytes = max(256, mint_moe_lora_apply_workspace_bytes(pool, T, K))
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
 def mint_moe_lora_apply(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
                         status: torch.Tensor, x_row: Optional[torch.Tensor] = None,
                         pair_weight: Optional[torch.Tensor] = None,
@@ -390,6 +396,8 @@ def mint_moe_lora_apply(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tenso
         assert x_row.dtype == torch.int32 and x_row.is_contiguous()
     if pair_weight is not None:
         assert pair_weight.dtype == torch.float32 and pair_weight.is_contiguous()
+    if workspace is None:
+        workspace = new_moe_workspace(pool, plan.T, plan.K, device=y.device)
     _check(load_library().mint_moe_lora_apply(
         pool.handle, table.handle, _ptr(plan.blob), plan.T, plan.K, _ptr(x), x.stride(0), x.shape[0],
         _ptr(x_row), _ptr(pair_weight), _ptr(y), y.stride(0),

@@ -566,10 +566,11 @@ extern "C" int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_
 // MoE
 // ---------------------------------------------------------------------------
 extern "C" size_t mint_moe_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K) {
-  (void)pool;
-  (void)T;
-  (void)K;
-  return 0;
+  if (!pool || T <= 0 || K < 1 || pool->desc.num_experts < 1) return 0;
+  // pools the streamed kernels do not take (r_max other than 8, 16, 32, 64) need no workspace
+  if (!mint_stream_moe_supported(pool->desc.r_max, 0)) return 0;
+  return mint_stream_moe_workspace_bytes((int64_t)T * K, (int64_t)pool->desc.num_slots * pool->desc.num_experts,
+                                         pool->desc.r_max);
 }
 
 extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
@@ -617,5 +618,10 @@ extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_ta
   a.y = static_cast<uint16_t *>(y_dev);
   a.ldy = ldy;
   a.status = status_dev;
+  if (need > 0 && mint_stream_moe_supported(pool->desc.r_max, table->max_rank)) {
+    if ((reinterpret_cast<uintptr_t>(workspace_dev) & 15) != 0)
+      return mint_fail(MINT_ERR_MISALIGNED, "moe_apply: workspace_dev must be 16-byte aligned");
+    return mint_launch_stream_moe(a, table_dev(table), plan_dev, workspace_dev, static_cast<cudaStream_t>(stream));
+  }
   return mint_launch_moe(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
 }

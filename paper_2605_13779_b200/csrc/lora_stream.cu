@@ -77,8 +77,8 @@ constexpr int kMaxParts = 8;              // shrink lanes that may share one til
 constexpr int kMaxProblems = MINT_MAX_GROUP;
 
 struct StreamProblem {
-  const uint16_t *A;   // [slot][r_max][d]
-  const uint16_t *B;   // [slot][r_max][n]
+  const uint16_t *A;   // [slot][r_max][d]; packed MoE pools: [slot][expert][d][r_max]
+  const uint16_t *B;   // [slot][r_max][n];                   [slot][expert][r_max][n]
   const uint16_t *x;
   uint16_t *y;
   int64_t ldx, ldy;
@@ -92,6 +92,12 @@ struct StreamParams {
   StreamProblem prob[kMaxProblems];
   int32_t nprob;
   int32_t T;
+  int32_t K;                          // items per token: 1, or the routed experts per token of a MoE plan
+  int32_t num_experts;                // 0 for dense projections
+  int32_t weights_per_slot;           // weight blocks per slot: 1, or the number of experts
+  const int32_t *x_row;               // MoE: row of x that pair p reads (nullptr: p)
+  const float *pair_weight;           // MoE: weight of pair p (nullptr: 1)
+  int64_t x_rows;                     // MoE: rows of x (range check of x_row)
   int32_t lanes;                      // grid size = the plan's lane count
   int32_t cb_shrink, cb_expand;       // virtual column blocks of the whole call
   int32_t cb_shrink_widest;           // column blocks of the widest d of the call
@@ -123,6 +129,14 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ uint4 zero4() { return make_uint4(0u, 0u, 0u, 0u); }
+// Four 8x8 bf16 matrices (eight 16-byte rows each; lane i gives the address of row i % 8 of
+// matrix i / 8), transposed: lane (g, t) gets elements [2t][g], [2t+1][g] of each.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 r;
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
@@ -222,7 +236,7 @@ struct CtaShared {
 template <bool kExpand>
 __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, Area &area, CtaRange &R,
                                          bool report_errors) {
-  if (!plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi,
+  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi,
                report_errors ? P.status : nullptr))
     return false;
   if (P.pv.header[PH_LANES] != P.lanes) {
@@ -256,6 +270,10 @@ __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, A
 }
 
 // Stages the descriptors and the row indices of tiles [tb, tb + ntile) (all threads).
+// kRowsOfX (the shrink of a MoE call): the rows are those of x that the pairs
+// read; a pair whose row is out of range is reported and gets row -1 (its x
+// counts as zero, so its y stays as it is).
+template <bool kRowsOfX>
 __device__ __forceinline__ void load_batch(const StreamParams &P, CtaShared &sh, int tb, int ntile) {
   __syncthreads();  // every warp is done with the previous batch
   const int4 *src = reinterpret_cast<const int4 *>(P.pv.tile_desc + tb);
@@ -264,7 +282,18 @@ __device__ __forceinline__ void load_batch(const StreamParams &P, CtaShared &sh,
   __syncthreads();
   const int off0 = sh.desc[0].off;
   const int nitems = sh.desc[ntile - 1].off + sh.desc[ntile - 1].len - off0;
-  for (int i = threadIdx.x; i < nitems; i += kThreads) sh.rows[i] = P.pv.perm[off0 + i];
+  for (int i = threadIdx.x; i < nitems; i += kThreads) {
+    const int p = P.pv.perm[off0 + i];
+    int row = p;
+    if (kRowsOfX) {
+      if (P.x_row) row = P.x_row[p];
+      if (row < 0 || row >= P.x_rows) {
+        report(P.status, MINT_ERR_BAD_INDEX, p);
+        row = -1;
+      }
+    }
+    sh.rows[i] = row;
+  }
   __syncthreads();
 }
 
@@ -274,7 +303,8 @@ struct Piece {
   int lo, hi;   // column blocks of the problem [lo, hi)
   int blocks;   // column blocks of the problem's whole width
   const int32_t *rows;   // the tile's row indices (shared memory)
-  int r, len, slot;
+  int r, len;
+  int slot;     // weight block: the slot, or slot * experts + expert
   float scale;
   int lane_lo, lane_hi;   // bounds of the shrink lanes that can meet this tile
   int ti;                 // index of the tile in the staged batch
@@ -297,7 +327,7 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     pc.r = sh.desc[ti].rank;
     pc.len = sh.desc[ti].len;
     pc.scale = sh.desc[ti].scale;
-    pc.slot = sh.desc[ti].slot;
+    pc.slot = sh.desc[ti].slot * P.weights_per_slot + sh.desc[ti].expert;
     pc.lane_lo = sh.desc[ti].lane_lo;
     pc.lane_hi = sh.desc[ti].lane_hi;
     pc.rows = sh.rows + (sh.desc[ti].off - sh.desc[0].off);
@@ -319,13 +349,18 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
 
 // Pulls the rows of a piece into L2 (all threads): the weight rows, which no apply
 // kernel writes, may go before the dependency wait; activations only after it.
-template <bool kExpand>
+template <bool kExpand, bool kPackedA = false>
 __device__ __forceinline__ void prefetch_piece(const StreamProblem &pb, const Piece &pc, bool weights, bool acts) {
   constexpr int kBlock = kExpand ? kExpandBlock : kShrinkBlock;
   const int width = kExpand ? pb.n : pb.d;
   const int c0 = pc.lo * kBlock, c1 = min(pc.hi * kBlock, width);
   const int lines = ((c1 - c0) * 2 + 127) / 128 + 1;   // one address per 128 bytes, plus the last 16 bytes
-  if (weights) {
+  if (weights && kPackedA) {
+    // A[d][r_max]: the piece's rows c0..c1 are one contiguous run
+    const uint16_t *w = pb.A + ((int64_t)pc.slot * pb.d + c0) * pb.r_max;
+    const int total = (c1 - c0) * pb.r_max;
+    for (int i = threadIdx.x * 64; i < total; i += kThreads * 64) prefetch_l2(w + i);
+  } else if (weights) {
     const uint16_t *w = (kExpand ? pb.B : pb.A) + (int64_t)pc.slot * pb.r_max * width;
     for (int i = threadIdx.x; i < pc.r * lines; i += kThreads) {
       const int row = i / lines, ln = i - row * lines;
@@ -418,6 +453,130 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
           make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
 }
 
+// The same for the packed MoE layout A[d][r_max] (RG = r_max / 8 groups of 8
+// ranks per row of A): the 32 rows of a column block are one contiguous run of
+// memory, which the warp copies with coalesced 16-byte segments into its ring,
+// each segment going where an 8x8 matrix of the transposing ldmatrix expects it:
+// matrix (k-step, k-half, rank group), row j <-> row k = 8 (j / 2) + 4 step + 2 half + j % 2
+// of the block, the same permutation of k that the x fragments use.  A pass covers
+// min(RG, 4) rank groups from rank rh on; segments of rank groups at or beyond
+// the slot's rank are not read.
+template <int XG, int RG>
+__device__ __forceinline__ void shrink_mma_packed(const StreamProblem &pb, const Piece &pc, int rh,
+                                                  uint32_t ring_base, float *scratch) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  constexpr int NT = RG < 4 ? RG : 4;
+  constexpr int N = XG + NT;
+  constexpr int MT = (XG + 1) / 2;
+  Ring<N> ring{ring_base};
+  const uint32_t warp_base = ring_base - (uint32_t)lane * 16;
+  const uint16_t *A_w = pb.A + (int64_t)pc.slot * pb.d * pb.r_max;
+  const uint16_t *xsrc[XG];
+#pragma unroll
+  for (int i = 0; i < XG; ++i) {
+    const int row = i * 8 + g;
+    const int xr = row < pc.len ? pc.rows[row] : -1;
+    xsrc[i] = xr >= 0 ? pb.x + (int64_t)xr * pb.ldx + t * 8 : nullptr;
+  }
+  // this lane's segment of every 512-byte slot of a block of A: where it comes from, where it goes
+  int a_off[NT], a_k[NT];
+  uint32_t a_dst[NT];
+#pragma unroll
+  for (int j = 0; j < NT; ++j) {
+    const int c = j * 32 + lane, k = c / NT, rgl = c % NT, rg = (rh >> 3) + rgl;
+    a_off[j] = k * pb.r_max + rg * 8;
+    a_k[j] = rg * 8 < pc.r ? k : (1 << 30);
+    const int m = (((k >> 2) & 1) * 2 + ((k >> 1) & 1)) * NT + rgl, jj = 2 * (k >> 3) + (k & 1);
+    a_dst[j] = (uint32_t)((m * 8 + jj) * 16);
+  }
+  // ldmatrix addresses: NT == 1: one x4 gives (step 0: half 0, half 1; step 1: half 0, half 1);
+  // otherwise one x4 per (step, pair of rank groups): (group: half 0, half 1; group + 1: half 0, half 1)
+  uint32_t lm_off[NT == 1 ? 1 : NT];
+  if (NT == 1) {
+    lm_off[0] = (uint32_t)lane * 16;
+  } else {
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+      for (int np = 0; np < NT / 2; ++np) {
+        const int mi = lane >> 3, h = mi & 1, nt = 2 * np + (mi >> 1);
+        lm_off[ks * (NT / 2) + np] = (uint32_t)((((ks * 2 + h) * NT + nt) * 8 + (lane & 7)) * 16);
+      }
+  }
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int a = 0; a < MT; ++a)
+#pragma unroll
+    for (int b = 0; b < NT; ++b)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) acc[a][b][e] = 0.f;
+
+  const int first = pc.lo + warp;
+  const int iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
+  auto a_region = [&](int it) { return warp_base + (uint32_t)(((it % Ring<N>::kDepth) * N + XG) * 512); };
+  auto issue = [&](int it) {
+    if (it < iters) {
+      const int col = (first + it * kWarps) * kShrinkBlock;
+      const bool ok = col + t * 8 < pb.d;
+#pragma unroll
+      for (int i = 0; i < XG; ++i) cp_async16(ring.slot(it, i), xsrc[i] ? xsrc[i] + col : pb.A, ok && xsrc[i]);
+      const uint16_t *blk = A_w + (int64_t)col * pb.r_max;
+      const uint32_t dst = a_region(it);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        const bool ok_a = col + a_k[j] < pb.d;
+        cp_async16(dst + a_dst[j], ok_a ? blk + a_off[j] : pb.A, ok_a);
+      }
+    }
+    cp_async_commit();
+  };
+#pragma unroll 1
+  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    issue(it + Ring<N>::kDepth - 1);
+    cp_async_wait<Ring<N>::kDepth - 1>();
+    __syncwarp();   // every lane's segments of this block have landed
+    uint4 xa[2 * MT];
+#pragma unroll
+    for (int i = 0; i < 2 * MT; ++i) xa[i] = i < XG ? lds128(ring.slot(it, i)) : zero4();
+    const uint32_t region = a_region(it);
+    uint32_t wb[2][NT][2];   // [k-step][rank group][k-half]
+    if (NT == 1) {
+      uint32_t r4[4];
+      ldmatrix_x4_trans(r4, region + lm_off[0]);
+      wb[0][0][0] = r4[0]; wb[0][0][1] = r4[1]; wb[1][0][0] = r4[2]; wb[1][0][1] = r4[3];
+    } else {
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+        for (int np = 0; np < NT / 2; ++np) {
+          uint32_t r4[4];
+          ldmatrix_x4_trans(r4, region + lm_off[ks * (NT / 2) + np]);
+          wb[ks][2 * np][0] = r4[0]; wb[ks][2 * np][1] = r4[1];
+          wb[ks][2 * np + 1][0] = r4[2]; wb[ks][2 * np + 1][1] = r4[3];
+        }
+    }
+    __syncwarp();   // all lanes have read the block before its slots are refilled
+#pragma unroll
+    for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+          mma_bf16(acc[mt][nt], word(xa[2 * mt], 2 * ks), word(xa[2 * mt + 1], 2 * ks),
+                   word(xa[2 * mt], 2 * ks + 1), word(xa[2 * mt + 1], 2 * ks + 1), wb[ks][nt][0], wb[ks][nt][1]);
+  }
+  cp_async_wait<0>();
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+      *reinterpret_cast<float4 *>(scratch + (((warp * 2 + mt) * 4 + nt) * 32 + lane) * 4) =
+          make_float4(acc[mt][nt][0], acc[mt][nt][1], acc[mt][nt][2], acc[mt][nt][3]);
+}
+
 // rank-1 tiles of at most L tokens: fp32 FMAs over coalesced 512-byte warp loads.
 template <int L>
 __device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
@@ -474,6 +633,7 @@ struct SmemShrink {
   float scratch[kWarps * 2 * 4 * 128];   // [warp][m-tile][n-tile][lane][4] MMA fragments, or [warp][8] sums
 };
 
+template <bool kPacked>
 __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &S, uint32_t ring_base,
                                              const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
@@ -481,11 +641,22 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   // the sum over this lane's columns; the expand adds the lanes of a tile in lane order
   float *dst = pb.ws_part + (size_t)(pc.t + blockIdx.x) * slot_floats;
-  const bool vec = pc.r == 1 && pc.len <= 8;
+  const bool vec = !kPacked && pc.r == 1 && pc.len <= 8;
   for (int rh = 0; rh < pc.r; rh += 32) {
     const int rr = min(32, pc.r - rh);
     __syncthreads();   // the scratch is free again
-    if (vec) {
+    if (kPacked) {
+      const int rg = pb.r_max >> 3;
+#define MINT_SHRINK_CASE(XG)                                                          \
+  if (rg == 1) shrink_mma_packed<XG, 1>(pb, pc, rh, ring_base, S.scratch);            \
+  else if (rg == 2) shrink_mma_packed<XG, 2>(pb, pc, rh, ring_base, S.scratch);       \
+  else if (rg == 4) shrink_mma_packed<XG, 4>(pb, pc, rh, ring_base, S.scratch);       \
+  else shrink_mma_packed<XG, 8>(pb, pc, rh, ring_base, S.scratch)
+      if (pc.len <= 8) { MINT_SHRINK_CASE(1); }
+      else if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
+      else { MINT_SHRINK_CASE(4); }
+#undef MINT_SHRINK_CASE
+    } else if (vec) {
       if (pc.len == 1) shrink_vec<1>(pb, pc, ring_base, S.scratch);
       else if (pc.len == 2) shrink_vec<2>(pb, pc, ring_base, S.scratch);
       else if (pc.len <= 4) shrink_vec<4>(pb, pc, ring_base, S.scratch);
@@ -522,6 +693,7 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
 
 constexpr size_t kRingsBytes = (size_t)kWarps * kRingBytes;
 
+template <bool kPacked>
 __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(const StreamParams P) {
   extern __shared__ __align__(128) uint8_t dyn_smem[];   // the four warps' rings
   __shared__ SmemShrink S;
@@ -537,15 +709,15 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
-    load_batch(P, S.sh, tb, ntile);
+    load_batch<kPacked>(P, S.sh, tb, ntile);
     if (!waited) {
       // while the previous kernel still runs: pull this lane's A rows into L2
       walk_batch<false>(P, area, R, S.sh, tb, ntile,
-                        [&](const Piece &pc) { prefetch_piece<false>(P.prob[pc.p], pc, true, false); });
+                        [&](const Piece &pc) { prefetch_piece<false, kPacked>(P.prob[pc.p], pc, true, false); });
       pdl_wait();   // activations and the workspace belong to earlier kernels until here
       waited = true;
     }
-    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece(P, S, ring_base, pc); });
+    walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) { shrink_piece<kPacked>(P, S, ring_base, pc); });
   }
 }
 
@@ -780,9 +952,12 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   const int yg = pc.len <= 8 ? 1 : (pc.len <= 16 ? 2 : 4);
   const int kg = pc.r <= 8 ? 1 : (pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8));
   const int MT = (yg + 1) >> 1, KS = (kg + 1) >> 1;
+  // MoE: the pair's routing weight multiplies its row of v
+  auto weight = [&](int row) { return P.pair_weight ? __ldg(P.pair_weight + pc.rows[row]) : 1.f; };
   __syncthreads();   // the previous piece no longer reads v
   if (vec) {
-    if (tid < 8) S.vvec[tid] = tid < pc.len ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, tid) : 0.f;
+    if (tid < 8)
+      S.vvec[tid] = tid < pc.len ? weight(tid) * sum_v(pb.ws_part, slot_floats, pc.t, first, count, tid) : 0.f;
   } else {
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
     for (int i = tid; i < MT * KS * 32; i += kThreads) {
@@ -792,9 +967,12 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int row = mt * 16 + g + (q & 1) * 8, k = ks * 16 + 2 * t + (q >> 1) * 8;
-        a[q] = (row < pc.len && k < pc.r) ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k) : 0.f;
+        const float w = row < pc.len ? weight(row) : 0.f;
+        a[q] = (row < pc.len && k < pc.r)
+                   ? w * sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k)
+                   : 0.f;
         b[q] = (row < pc.len && k + 1 < pc.r)
-                   ? sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k + 1)
+                   ? w * sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k + 1)
                    : 0.f;
       }
       uint32_t hi[4], lo[4];
@@ -842,7 +1020,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
-    load_batch(P, S.sh, tb, ntile);
+    load_batch<false>(P, S.sh, tb, ntile);
     // which shrink lanes hold the parts of v of every (tile, projection) of the batch
     for (int i = threadIdx.x; i < ntile * P.nprob; i += kThreads) {
       const int ti = i / P.nprob, p = i - ti * P.nprob;
@@ -872,6 +1050,85 @@ size_t workspace_bytes(int64_t tiles, int32_t r_max) {
 
 bool mint_stream_supported(int32_t r_max_bound) { return r_max_bound <= kStreamRankCap; }
 
+// The packed-layout shrink reads A[d][r_max] in 16-byte segments of 8 ranks.
+bool mint_stream_moe_supported(int32_t r_max, int32_t r_max_bound) {
+  return r_max_bound <= kStreamRankCap && (r_max == 8 || r_max == 16 || r_max == 32 || r_max == 64);
+}
+
+size_t mint_stream_moe_workspace_bytes(int64_t pairs, int64_t key_space, int32_t r_max) {
+  return workspace_bytes(mint_tile_upper_bound(1, pairs, key_space), r_max);
+}
+
+static int32_t stream_kernel_attributes() {
+  static bool attrs_set = false;
+  if (attrs_set) return MINT_OK;
+  int32_t st;
+  st = mint_check_cuda(cudaFuncSetAttribute(shrink_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kRingsBytes), "shrink_stream shared memory");
+  if (st) return st;
+  st = mint_check_cuda(cudaFuncSetAttribute(shrink_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kRingsBytes), "shrink_stream (packed) shared memory");
+  if (st) return st;
+  st = mint_check_cuda(cudaFuncSetAttribute(expand_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)kRingsBytes), "expand_stream shared memory");
+  if (st) return st;
+  attrs_set = true;
+  return MINT_OK;
+}
+
+// MoE expert LoRA apply on the streamed kernels: the plan's items are the
+// (token, k) pairs grouped by (expert, slot); the weight block of a tile is
+// (slot, expert); the shrink reads row x_row[p] of x, the expand updates row p of y.
+int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, void *workspace,
+                               cudaStream_t s) {
+  int32_t lanes = 0;
+  int32_t st = mint_device_lanes(&lanes);
+  if (st) return st;
+  if ((st = stream_kernel_attributes())) return st;
+  const int64_t pairs = (int64_t)a.T * a.K;
+  const int64_t key_space = (int64_t)tab.num_slots * a.num_experts;
+  const int64_t tiles = mint_tile_upper_bound(1, pairs, key_space);
+  if (tiles == 0) return MINT_OK;
+  StreamParams P = {};
+  StreamProblem &pb = P.prob[0];
+  pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
+  pb.ldx = a.ldx; pb.ldy = a.ldy;
+  pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
+  pb.cb0_shrink = 0;
+  pb.cb0_expand = 0;
+  pb.ws_part = static_cast<float *>(workspace);
+  P.nprob = 1;
+  P.T = a.T;
+  P.K = a.K;
+  P.num_experts = a.num_experts;
+  P.weights_per_slot = a.num_experts;
+  P.x_row = a.x_row;
+  P.pair_weight = a.pair_weight;
+  P.x_rows = a.x_rows;
+  P.lanes = lanes;
+  P.cb_shrink = (a.d + kShrinkBlock - 1) / kShrinkBlock;
+  P.cb_expand = (a.n + kExpandBlock - 1) / kExpandBlock;
+  P.cb_shrink_widest = P.cb_shrink;
+  P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
+  P.status = a.status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, pairs, key_space);
+
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)lanes);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kRingsBytes;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<true>, P), "shrink_stream (packed) launch");
+  if (st) return st;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
+}
+
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max) {
   return workspace_bytes(mint_tile_upper_bound(1, T, num_slots), r_max);
 }
@@ -883,16 +1140,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   int32_t lanes = 0;
   int32_t st = mint_device_lanes(&lanes);
   if (st) return st;
-  static bool attrs_set = false;
-  if (!attrs_set) {
-    st = mint_check_cuda(cudaFuncSetAttribute(shrink_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kRingsBytes), "shrink_stream shared memory");
-    if (st) return st;
-    st = mint_check_cuda(cudaFuncSetAttribute(expand_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)kRingsBytes), "expand_stream shared memory");
-    if (st) return st;
-    attrs_set = true;
-  }
+  if ((st = stream_kernel_attributes())) return st;
   const int32_t T = args[0].T;
   const int64_t tiles = mint_tile_upper_bound(1, T, tab.num_slots);
   if (tiles == 0) return MINT_OK;
@@ -913,6 +1161,9 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   }
   P.nprob = nprob;
   P.T = T;
+  P.K = 1;
+  P.num_experts = 0;
+  P.weights_per_slot = 1;
   P.lanes = lanes;
   P.cb_shrink = cb_s;
   P.cb_expand = cb_e;
@@ -932,7 +1183,7 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel, P), "shrink_stream launch");
+  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
   if (st) return st;
   if (T >= MINT_DENSE_MIN_BATCH) {   // the plan may have given dense segments to the tensor-core shrink
     st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);

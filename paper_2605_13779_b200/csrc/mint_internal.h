@@ -190,6 +190,10 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);
 
+// MoE apply on the streamed kernels (pool r_max of 8, 16, 32 or 64; bound ranks up to 64).
+bool mint_stream_moe_supported(int32_t r_max, int32_t max_bound_rank);
+size_t mint_stream_moe_workspace_bytes(int64_t pairs, int64_t key_space, int32_t r_max);
+
 struct MoEArgs {
   const uint16_t *A;   // [slot][E][d][r_max]
   const uint16_t *B;   // [slot][E][r_max][n]
@@ -204,6 +208,8 @@ struct MoEArgs {
   int32_t *status;
 };
 int32_t mint_launch_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
+int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, void *workspace,
+                               cudaStream_t s);
 
 int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
                                float *slot_scale, int32_t num_slots, cudaStream_t s);

@@ -66,6 +66,25 @@ def test_ragged_moe(T, K, E, d, n, num_slots, rank, p_none):
     check_case(synth.config4_projection(batch, "down", d=d, n=n, tag=tag), tag + "/down")
 
 
+@pytest.mark.parametrize("r_max,ranks,d,n", [
+    (16, [16, 1, 9, 8], 520, 264),
+    (32, [32, 3, 17, 8, 24], 2048, 768),
+    (64, [64, 40, 1, 16, 33, 8], 776, 2048),
+    (8, [8, 2, 5], 264, 136),
+])
+def test_mixed_ranks_in_padded_pools(r_max, ranks, d, n):
+    """Slots of different ranks in one pool of r_max columns; the padding is NaN
+    and must never reach y.  Long and short (expert, adapter) groups."""
+    import dataclasses
+    tag = f"gpu/moe/mixed/{r_max}"
+    S = len(ranks)
+    batch = synth.config4_batch(T=160, E=4, K=2, num_slots=S, rank=r_max, p_none=0.05, tag=tag)
+    table = synth.identity_table(S, np.asarray(ranks, dtype=np.int32), 2.0)
+    batch = dataclasses.replace(batch, table=table)
+    for proj in ("gate", "down"):
+        check_case(synth.config4_projection(batch, proj, d=d, n=n, tag=tag), f"{tag}/{proj}")
+
+
 def test_one_expert_top1_equals_dense_apply():
     from paper_2605_13779_b200 import binding as mb, harness
     batch = synth.config4_batch(T=50, E=1, K=1, num_slots=3, rank=8, tag="gpu/moe1")
