@@ -27,11 +27,14 @@
 //    and every 32-byte sector fetched is used in full.  Rows beyond the tile's
 //    length or the slot's rank are not loaded at all (zero registers).
 //  - expand: B is [rank][n] with n contiguous.  Lane (g, t) loads 16 bytes of
-//    rows 2t, 2t+1, 2t+8, 2t+9 at column 8 g of a 64-column block and pairs
-//    them with one byte-permute per MMA tile; tile j holds the columns 8 g + j,
-//    so the lane ends up owning 16 consecutive columns of y for rows g and g+8:
-//    y is read, updated (one fp32 fma, one round-to-nearest-even) and written
-//    with 128-bit accesses.  v enters as a bf16 head plus a bf16 remainder (two
+//    rows 2t, 2t+1, 2t+8, 2t+9 at the 8-column chunk c(g) = 4 (g & 1) + g / 2
+//    of a 64-column block and pairs them with one byte-permute per MMA tile;
+//    tile j holds the columns 8 c(g) + j, so the lane ends up owning the chunks
+//    t and 4 + t of y for rows g and g+8, and every y access of the warp covers
+//    64 contiguous bytes (two whole sectors) of each of eight rows: y is read,
+//    updated (one fp32 fma, one round-to-nearest-even) and written with 128-bit
+//    accesses.  (Chunks 2t and 2t + 1 would give each lane 32 contiguous bytes
+//    but make every access touch half sectors, which halves the bandwidth.)  v enters as a bf16 head plus a bf16 remainder (two
 //    MMAs), about 16 significant bits of the fp32 shrink result.
 //  - tiles of rank 1 with at most 8 tokens (most of a large-catalog decode
 //    batch) skip the MMA: plain fp32 FMAs over fully coalesced 512-byte warp loads.
@@ -759,32 +762,36 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
   constexpr int MT = (YG + 1) / 2, KS = (KG + 1) / 2;
   Ring<N> ring{ring_base};
   const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
+  // n index g of every MMA tile stands for the 8-column chunk (g & 1) * 4 + (g >> 1) of the block, so that the
+  // accumulators of lane (g, t) (n = 2t and 2t + 1) are the chunks t and 4 + t: one y access of the warp
+  // then covers 64 contiguous bytes of each of 8 rows
+  const int bchunk = (g & 1) * 4 + (g >> 1);
   const uint16_t *bsrc[2 * KG];
   uint16_t *ysrc[YG];
 #pragma unroll
   for (int i = 0; i < 2 * KG; ++i) {
     const int k = (i >> 1) * 8 + 2 * t + (i & 1);
-    bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + g * 8 : nullptr;
+    bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + bchunk * 8 : nullptr;
   }
 #pragma unroll
   for (int i = 0; i < YG; ++i) {
     const int row = i * 8 + g;
-    ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 16 : nullptr;
+    ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 8 : nullptr;
   }
   const int first = pc.lo + warp;
   const int iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
   auto issue = [&](int it) {
     if (it < iters) {
       const int n0 = (first + it * kWarps) * kExpandBlock;
-      const bool ok_b = n0 + g * 8 < pb.n;
-      const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;
+      const bool ok_b = n0 + bchunk * 8 < pb.n;
+      const bool ok_y0 = n0 + t * 8 < pb.n, ok_y1 = n0 + 32 + t * 8 < pb.n;
 #pragma unroll
       for (int i = 0; i < 2 * KG; ++i)
         cp_async16(ring.slot(it, i), bsrc[i] ? bsrc[i] + n0 : pb.B, ok_b && bsrc[i]);
 #pragma unroll
       for (int i = 0; i < YG; ++i) {
         cp_async16(ring.slot(it, 2 * KG + 2 * i), ysrc[i] ? ysrc[i] + n0 : pb.B, ok_y0 && ysrc[i]);
-        cp_async16(ring.slot(it, 2 * KG + 2 * i + 1), ysrc[i] ? ysrc[i] + n0 + 8 : pb.B, ok_y1 && ysrc[i]);
+        cp_async16(ring.slot(it, 2 * KG + 2 * i + 1), ysrc[i] ? ysrc[i] + n0 + 32 : pb.B, ok_y1 && ysrc[i]);
       }
     }
     cp_async_commit();
@@ -796,7 +803,7 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
     issue(it + Ring<N>::kDepth - 1);
     cp_async_wait<Ring<N>::kDepth - 1>();
     const int n0 = (first + it * kWarps) * kExpandBlock;
-    const bool ok_y0 = n0 + t * 16 < pb.n, ok_y1 = n0 + t * 16 + 8 < pb.n;
+    const bool ok_y0 = n0 + t * 8 < pb.n, ok_y1 = n0 + 32 + t * 8 < pb.n;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
       float acc[8][4];
@@ -823,7 +830,7 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
           mma_bf16(acc[j], vl.x, vl.y, vl.z, vl.w, b0, b1);
         }
       }
-      // acc[j][0], [1]: row g, columns 16 t + j and 16 t + 8 + j; acc[j][2], [3]: row g + 8
+      // acc[j][0], [1]: row g, columns 8 t + j and 32 + 8 t + j; acc[j][2], [3]: row g + 8
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (2 * mt + h < YG) {
@@ -831,7 +838,7 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
           if (yr) {
             if (ok_y0) update8(yr + n0, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
             if (ok_y1)
-              update8(yr + n0 + 8, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
+              update8(yr + n0 + 32, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
           }
         }
       }
