@@ -447,6 +447,7 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
                    word(wb[nt], 2 * ks + 1));
   }
   cp_async_wait<0>();
+  __syncthreads();   // the gather of the previous pass has read the scratch
   // scratch[warp][mt][nt][lane][4]
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
@@ -572,6 +573,7 @@ __device__ __forceinline__ void shrink_mma_packed(const StreamProblem &pb, const
                    word(xa[2 * mt], 2 * ks + 1), word(xa[2 * mt + 1], 2 * ks + 1), wb[ks][nt][0], wb[ks][nt][1]);
   }
   cp_async_wait<0>();
+  __syncthreads();   // the gather of the previous pass has read the scratch
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
@@ -624,6 +626,7 @@ __device__ __forceinline__ void shrink_vec(const StreamProblem &pb, const Piece 
     }
   }
   cp_async_wait<0>();
+  __syncthreads();   // the gather of the previous pass has read the scratch
 #pragma unroll
   for (int l = 0; l < L; ++l) {
     const float s = warp_sum(acc[l]);
@@ -647,7 +650,7 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   const bool vec = !kPacked && pc.r == 1 && pc.len <= 8;
   for (int rh = 0; rh < pc.r; rh += 32) {
     const int rr = min(32, pc.r - rh);
-    __syncthreads();   // the scratch is free again
+    // (the bodies wait, right before they write the scratch, until the previous gather has read it)
     if (kPacked) {
       const int rg = pb.r_max >> 3;
 #define MINT_SHRINK_CASE(XG)                                                          \
