@@ -183,7 +183,7 @@ __device__ __forceinline__ uint32_t word(const uint4 &q, int i) {
 // cb = (P - rows(t) * CB) / w_t  where w_t is the tile's row count.
 template <bool kExpand>
 __device__ __forceinline__ int tile_rows(int rank, int len) {
-  return kExpand ? rank + 2 * len : rank + len;
+  return kExpand ? mint_tile_rows_expand(rank, len) : mint_tile_rows_shrink(rank, len);
 }
 
 struct Area {

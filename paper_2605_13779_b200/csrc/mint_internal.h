@@ -30,9 +30,9 @@ enum {
   PH_NCHUNK0,   // number of tiles in list g (MINT_NUM_TILE_LISTS entries)
   PH_NCHUNK1,
   PH_LANES,     // number of cost lanes G the lane tables were cut for
-  PH_ROWS_SHRINK,  // sum over list-1 tiles of (rank + len)
-  PH_ROWS_EXPAND,  // sum over list-1 tiles of (rank + 2 len)
-  PH_MAX_TILE_ROWS,  // largest (rank + len) of a list-1 tile that the streamed shrink handles
+  PH_ROWS_SHRINK,  // sum over list-1 tiles of mint_tile_rows_shrink
+  PH_ROWS_EXPAND,  // sum over list-1 tiles of mint_tile_rows_expand
+  PH_MAX_TILE_ROWS,  // largest mint_tile_rows_shrink of a list-1 tile that the streamed shrink handles
   PH_NUM_DENSE,      // number of 128-row tiles of dense segments (tensor-core shrink)
   PH_WORDS = 32
 };
@@ -41,6 +41,21 @@ enum {
 #define MINT_MAX_LANES 1024
 // Tile list g cuts every segment into runs of at most mint_tile_tokens(g) items.
 __host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 32; }
+
+// Cost of a tile per column block, in rows of streamed bytes: the rows it moves
+// (rank + len for the shrink, rank + 2 len for the expand: y is read and
+// written) plus a constant for what a block costs whatever its height (an
+// iteration of a warp waits for memory once, and narrow tiles do not fill the
+// tensor-core shapes).  The lanes' shares are equal in this cost.
+#define MINT_TILE_COST_SHRINK 8
+#define MINT_TILE_COST_EXPAND 8
+// (tiles of rank 1 with at most 8 tokens take the FMA path, whose cost does follow the rows)
+__host__ __device__ constexpr int mint_tile_rows_shrink(int rank, int len) {
+  return rank + len + ((rank == 1 && len <= 8) ? 0 : MINT_TILE_COST_SHRINK);
+}
+__host__ __device__ constexpr int mint_tile_rows_expand(int rank, int len) {
+  return rank + 2 * len + ((rank == 1 && len <= 8) ? 0 : MINT_TILE_COST_EXPAND);
+}
 
 // One tile of list 1 with everything a streaming kernel needs to start on it:
 // no dependent lookups through segment or slot arrays.  rank and scale are the
