@@ -730,6 +730,12 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
 // ================================================================================
 // expand
 // ================================================================================
+// A piece of the expand runs in three steps.  (1) Every warp requests the first
+// blocks of its share of the piece.  (2) While they are on their way, the CTA
+// adds the shrink lanes' parts of v, element by element with coalesced loads
+// (times the pair's routing weight in a MoE call), and turns the sums into MMA
+// operand fragments.  (3) The warps stream their blocks.
+
 // Splits v into a bf16 head and a bf16 remainder so that two MMAs carry about
 // 16 significant bits of the fp32 shrink result into the expand.
 __device__ __forceinline__ void split_pair(float a, float b, uint32_t &hi, uint32_t &lo) {
@@ -741,7 +747,7 @@ struct SmemExpand {
   CtaShared sh;
   // v of the current tile as MMA A-operand fragments: [m-tile][k-step][head/remainder][lane] x 4 registers
   uint4 vfrag[2 * 4 * 2 * 32];
-  float vvec[8];   // rank-1 path: v per token
+  float vsum[kTileRowsMax * kStreamRankCap];   // v of the current tile, [len][rank], weighted
 };
 
 // 8 output columns of one row: y += scale * acc[j][e] for column j, stored with one 128-bit write
@@ -753,37 +759,43 @@ __device__ __forceinline__ void update8(uint16_t *yp, const uint4 &old, float sc
   *reinterpret_cast<uint4 *>(yp) = pack8(f);
 }
 
-// YG = groups of 8 token rows (two 16-byte segments of y each), KG = groups of 8
-// rank rows of B (rows 8 kg + 2t and 8 kg + 2t + 1): only groups that exist take
-// slots of the staging ring.
+// The addresses a lane streams in a piece of the tensor-core path.  YG = groups
+// of 8 token rows (two 16-byte segments of y each), KG = groups of 8 rank rows
+// of B (rows 8 kg + 2t and 8 kg + 2t + 1): only groups that exist take slots of
+// the staging ring.
 template <int YG, int KG>
-__device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
-                                           const SmemExpand &S) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t = lane & 3;
-  constexpr int N = 2 * KG + 2 * YG;
-  constexpr int MT = (YG + 1) / 2, KS = (KG + 1) / 2;
-  Ring<N> ring{ring_base};
-  const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
-  // n index g of every MMA tile stands for the 8-column chunk (g & 1) * 4 + (g >> 1) of the block, so that the
-  // accumulators of lane (g, t) (n = 2t and 2t + 1) are the chunks t and 4 + t: one y access of the warp
-  // then covers 64 contiguous bytes of each of 8 rows
-  const int bchunk = (g & 1) * 4 + (g >> 1);
+struct ExpandLane {
+  static constexpr int N = 2 * KG + 2 * YG;
+  static constexpr int MT = (YG + 1) / 2, KS = (KG + 1) / 2;
+  Ring<N> ring;
   const uint16_t *bsrc[2 * KG];
   uint16_t *ysrc[YG];
+  int first, iters, t, bchunk;
+
+  __device__ __forceinline__ void init(const StreamProblem &pb, const Piece &pc, uint32_t ring_base) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2;
+    t = lane & 3;
+    ring.base = ring_base;
+    const uint16_t *B_slot = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
+    // n index g of every MMA tile stands for the 8-column chunk (g & 1) * 4 + (g >> 1) of the block, so that
+    // the accumulators of lane (g, t) (n = 2t and 2t + 1) are the chunks t and 4 + t: one y access of the
+    // warp then covers 64 contiguous bytes of each of 8 rows
+    bchunk = (g & 1) * 4 + (g >> 1);
 #pragma unroll
-  for (int i = 0; i < 2 * KG; ++i) {
-    const int k = (i >> 1) * 8 + 2 * t + (i & 1);
-    bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + bchunk * 8 : nullptr;
-  }
+    for (int i = 0; i < 2 * KG; ++i) {
+      const int k = (i >> 1) * 8 + 2 * t + (i & 1);
+      bsrc[i] = k < pc.r ? B_slot + (int64_t)k * pb.n + bchunk * 8 : nullptr;
+    }
 #pragma unroll
-  for (int i = 0; i < YG; ++i) {
-    const int row = i * 8 + g;
-    ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 8 : nullptr;
+    for (int i = 0; i < YG; ++i) {
+      const int row = i * 8 + g;
+      ysrc[i] = row < pc.len ? pb.y + (int64_t)pc.rows[row] * pb.ldy + t * 8 : nullptr;
+    }
+    first = pc.lo + warp;
+    iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
   }
-  const int first = pc.lo + warp;
-  const int iters = first < pc.hi ? (pc.hi - first + kWarps - 1) / kWarps : 0;
-  auto issue = [&](int it) {
+  __device__ __forceinline__ void issue(const StreamProblem &pb, int it) const {
     if (it < iters) {
       const int n0 = (first + it * kWarps) * kExpandBlock;
       const bool ok_b = n0 + bchunk * 8 < pb.n;
@@ -798,14 +810,34 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
       }
     }
     cp_async_commit();
-  };
+  }
+};
+
+// Step 1: the first blocks of this warp.
+template <int YG, int KG>
+__device__ __forceinline__ void expand_mma_fill(const StreamProblem &pb, const Piece &pc, uint32_t ring_base) {
+  ExpandLane<YG, KG> L;
+  L.init(pb, pc, ring_base);
 #pragma unroll 1
-  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+  for (int it = 0; it < Ring<ExpandLane<YG, KG>::N>::kDepth - 1; ++it) L.issue(pb, it);
+}
+
+// Step 3: the blocks of this warp; the requests of expand_mma_fill are under way.
+template <int YG, int KG>
+__device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
+                                           const SmemExpand &S) {
+  using Lane = ExpandLane<YG, KG>;
+  constexpr int N = Lane::N, MT = Lane::MT, KS = Lane::KS;
+  constexpr int kDepth = Ring<N>::kDepth;
+  const int lane = threadIdx.x & 31;
+  Lane L;
+  L.init(pb, pc, ring_base);
+  const int t = L.t;
 #pragma unroll 1
-  for (int it = 0; it < iters; ++it) {
-    issue(it + Ring<N>::kDepth - 1);
-    cp_async_wait<Ring<N>::kDepth - 1>();
-    const int n0 = (first + it * kWarps) * kExpandBlock;
+  for (int it = 0; it < L.iters; ++it) {
+    L.issue(pb, it + kDepth - 1);
+    cp_async_wait<kDepth - 1>();
+    const int n0 = (L.first + it * kWarps) * kExpandBlock;
     const bool ok_y0 = n0 + t * 8 < pb.n, ok_y1 = n0 + 32 + t * 8 < pb.n;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
@@ -820,7 +852,7 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
         uint4 bq[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          bq[i] = (2 * ks + (i >> 1) < KG) ? lds128(ring.slot(it, 2 * (2 * ks + (i >> 1)) + (i & 1))) : zero4();
+          bq[i] = (2 * ks + (i >> 1) < KG) ? lds128(L.ring.slot(it, 2 * (2 * ks + (i >> 1)) + (i & 1))) : zero4();
         const uint4 vh = S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + lane];
         const uint4 vl = S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + lane];
 #pragma unroll
@@ -837,11 +869,12 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         if (2 * mt + h < YG) {
-          uint16_t *yr = ysrc[2 * mt + h];
+          uint16_t *yr = L.ysrc[2 * mt + h];
           if (yr) {
-            if (ok_y0) update8(yr + n0, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
+            if (ok_y0) update8(yr + n0, lds128(L.ring.slot(it, 2 * KG + 2 * (2 * mt + h))), pc.scale, acc, 2 * h);
             if (ok_y1)
-              update8(yr + n0 + 32, lds128(ring.slot(it, 2 * KG + 2 * (2 * mt + h) + 1)), pc.scale, acc, 2 * h + 1);
+              update8(yr + n0 + 32, lds128(L.ring.slot(it, 2 * KG + 2 * (2 * mt + h) + 1)), pc.scale, acc,
+                      2 * h + 1);
           }
         }
       }
@@ -850,51 +883,71 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
   cp_async_wait<0>();
 }
 
+// rank-1 tiles of at most L tokens: fp32 FMAs over coalesced 512-byte warp loads.
 template <int L>
-__device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
-                                           const SmemExpand &S) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int N = 1 + L;
-  Ring<N> ring{ring_base};
-  const uint16_t *w = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
+struct ExpandVecLane {
+  static constexpr int N = 1 + L;
+  static constexpr int kStep = kWarps * 256;
+  Ring<N> ring;
+  const uint16_t *w;
   uint16_t *yr[L];
-  float sv[L];
+  int c0, c1, iters, len;
+  __device__ __forceinline__ void init(const StreamProblem &pb, const Piece &pc, uint32_t ring_base) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    ring.base = ring_base;
+    w = pb.B + (int64_t)pc.slot * pb.r_max * pb.n;
+    len = pc.len;
 #pragma unroll
-  for (int l = 0; l < L; ++l) {
-    yr[l] = pb.y + (int64_t)pc.rows[l < pc.len ? l : 0] * pb.ldy;
-    sv[l] = pc.scale * S.vvec[l];
+    for (int l = 0; l < L; ++l) yr[l] = pb.y + (int64_t)pc.rows[l < pc.len ? l : 0] * pb.ldy;
+    c0 = pc.lo * kExpandBlock + warp * 256 + lane * 8;
+    c1 = min(pc.hi * kExpandBlock, pb.n);
+    iters = (c1 - (pc.lo * kExpandBlock + warp * 256) + kStep - 1) / kStep;   // <= 0: nothing for this warp
   }
-  const int c0 = pc.lo * kExpandBlock + warp * 256 + lane * 8, c1 = min(pc.hi * kExpandBlock, pb.n);
-  constexpr int kStep = kWarps * 256;
-  const int iters = (c1 - (pc.lo * kExpandBlock + warp * 256) + kStep - 1) / kStep;
-  auto issue = [&](int it) {
+  __device__ __forceinline__ void issue(int it) const {
     if (it < iters) {
       const int col = c0 + it * kStep;
       const bool ok = col < c1;
       cp_async16(ring.slot(it, 0), ok ? w + col : w, ok);
 #pragma unroll
-      for (int l = 0; l < L; ++l) cp_async16(ring.slot(it, 1 + l), ok ? yr[l] + col : w, ok && l < pc.len);
+      for (int l = 0; l < L; ++l) cp_async16(ring.slot(it, 1 + l), ok ? yr[l] + col : w, ok && l < len);
     }
     cp_async_commit();
-  };
+  }
+};
+
+template <int L>
+__device__ __forceinline__ void expand_vec_fill(const StreamProblem &pb, const Piece &pc, uint32_t ring_base) {
+  ExpandVecLane<L> V;
+  V.init(pb, pc, ring_base);
 #pragma unroll 1
-  for (int it = 0; it < Ring<N>::kDepth - 1; ++it) issue(it);
+  for (int it = 0; it < Ring<1 + L>::kDepth - 1; ++it) V.issue(it);
+}
+
+template <int L>
+__device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
+                                           const SmemExpand &S) {
+  constexpr int kDepth = Ring<1 + L>::kDepth;
+  ExpandVecLane<L> V;
+  V.init(pb, pc, ring_base);
+  float sv[L];
+#pragma unroll
+  for (int l = 0; l < L; ++l) sv[l] = l < pc.len ? pc.scale * S.vsum[l] : 0.f;
 #pragma unroll 1
-  for (int it = 0; it < iters; ++it) {
-    issue(it + Ring<N>::kDepth - 1);
-    cp_async_wait<Ring<N>::kDepth - 1>();
-    const int col = c0 + it * kStep;
-    if (col < c1) {
+  for (int it = 0; it < V.iters; ++it) {
+    V.issue(it + kDepth - 1);
+    cp_async_wait<kDepth - 1>();
+    const int col = V.c0 + it * ExpandVecLane<L>::kStep;
+    if (col < V.c1) {
       float wf[8];
-      unpack8(lds128(ring.slot(it, 0)), wf);
+      unpack8(lds128(V.ring.slot(it, 0)), wf);
 #pragma unroll
       for (int l = 0; l < L; ++l)
         if (l < pc.len) {
           float yf[8];
-          unpack8(lds128(ring.slot(it, 1 + l)), yf);
+          unpack8(lds128(V.ring.slot(it, 1 + l)), yf);
 #pragma unroll
           for (int e = 0; e < 8; ++e) yf[e] = fmaf(sv[l], wf[e], yf[e]);
-          *reinterpret_cast<uint4 *>(yr[l] + col) = pack8(yf);
+          *reinterpret_cast<uint4 *>(V.yr[l] + col) = pack8(yf);
         }
     }
   }
@@ -935,26 +988,46 @@ __device__ __forceinline__ void shrink_parts(const StreamParams &P, const Area &
   }
 }
 
-// v[idx] of the current tile: the sum, in lane order, of the shrink lanes' parts.
-// The loads of up to eight parts are issued together.
-__device__ __forceinline__ float sum_v(const float *part, size_t slot_floats, int t, int first, int count, int idx) {
-  float s = 0.f;
-  for (int k0 = 0; k0 < count; k0 += 8) {
-    float v[8];
+// Step 2a (all threads): vsum[i] = weight(row of i) * sum, in lane order, of the shrink
+// lanes' parts of element i of the [len][rank] result.  Consecutive threads take
+// consecutive elements, and the loads of four elements times four parts go out together.
+__device__ __forceinline__ void sum_parts(const StreamParams &P, const StreamProblem &pb, const Piece &pc,
+                                          int first, int count, float *vsum) {
+  const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
+  const float *part0 = pb.ws_part + (size_t)(pc.t + first) * slot_floats;
+  const int nel = pc.len * pc.r;
+  for (int i0 = threadIdx.x; i0 < nel; i0 += 4 * kThreads) {
+    float s[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k0 = 0; k0 < count; k0 += 4) {
+      float v[4][4];
 #pragma unroll
-    for (int k = 0; k < 8; ++k)
-      v[k] = (k0 + k < count) ? __ldcg(part + (size_t)(t + first + k0 + k) * slot_floats + idx) : 0.f;
+      for (int k = 0; k < 4; ++k)
 #pragma unroll
-    for (int k = 0; k < 8; ++k) s += v[k];
+        for (int e = 0; e < 4; ++e)
+          v[k][e] = (k0 + k < count && i0 + e * kThreads < nel)
+                        ? __ldcg(part0 + (size_t)(k0 + k) * slot_floats + i0 + e * kThreads)
+                        : 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[e] += v[k][e];
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = i0 + e * kThreads;
+      if (i < nel) {
+        // MoE: the pair's routing weight multiplies its row of v
+        const float w = P.pair_weight ? __ldg(P.pair_weight + pc.rows[i / pc.r]) : 1.f;
+        vsum[i] = w * s[e];
+      }
+    }
   }
-  return s;
 }
 
 __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &S, uint32_t ring_base,
                                              const Piece &pc) {
   const StreamProblem &pb = P.prob[pc.p];
   const int tid = threadIdx.x;
-  const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
   const bool vec = pc.r == 1 && pc.len <= 8;
   const int first = S.sh.part_first[pc.ti * kMaxProblems + pc.p];
   const int count = S.sh.part_count[pc.ti * kMaxProblems + pc.p];
@@ -962,37 +1035,46 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   const int yg = pc.len <= 8 ? 1 : (pc.len <= 16 ? 2 : 4);
   const int kg = pc.r <= 8 ? 1 : (pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8));
   const int MT = (yg + 1) >> 1, KS = (kg + 1) >> 1;
-  // MoE: the pair's routing weight multiplies its row of v
-  auto weight = [&](int row) { return P.pair_weight ? __ldg(P.pair_weight + pc.rows[row]) : 1.f; };
-  __syncthreads();   // the previous piece no longer reads v
+  // step 1
   if (vec) {
-    if (tid < 8)
-      S.vvec[tid] = tid < pc.len ? weight(tid) * sum_v(pb.ws_part, slot_floats, pc.t, first, count, tid) : 0.f;
+    if (pc.len == 1) expand_vec_fill<1>(pb, pc, ring_base);
+    else if (pc.len == 2) expand_vec_fill<2>(pb, pc, ring_base);
+    else if (pc.len <= 4) expand_vec_fill<4>(pb, pc, ring_base);
+    else expand_vec_fill<8>(pb, pc, ring_base);
   } else {
+#define MINT_EXPAND_CASE(YG)                                     \
+  if (kg == 1) expand_mma_fill<YG, 1>(pb, pc, ring_base);        \
+  else if (kg == 2) expand_mma_fill<YG, 2>(pb, pc, ring_base);   \
+  else if (kg == 4) expand_mma_fill<YG, 4>(pb, pc, ring_base);   \
+  else expand_mma_fill<YG, 8>(pb, pc, ring_base)
+    if (yg == 1) { MINT_EXPAND_CASE(1); }
+    else if (yg == 2) { MINT_EXPAND_CASE(2); }
+    else { MINT_EXPAND_CASE(4); }
+#undef MINT_EXPAND_CASE
+  }
+  // step 2
+  __syncthreads();   // the previous piece no longer reads v
+  sum_parts(P, pb, pc, first, count, S.vsum);
+  __syncthreads();
+  if (!vec) {
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
     for (int i = tid; i < MT * KS * 32; i += kThreads) {
       const int ln = i & 31, ks = (i >> 5) % KS, mt = (i >> 5) / KS;
       const int g = ln >> 2, t = ln & 3;
-      float a[4], b[4];
+      uint32_t hi[4], lo[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int row = mt * 16 + g + (q & 1) * 8, k = ks * 16 + 2 * t + (q >> 1) * 8;
-        const float w = row < pc.len ? weight(row) : 0.f;
-        a[q] = (row < pc.len && k < pc.r)
-                   ? w * sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k)
-                   : 0.f;
-        b[q] = (row < pc.len && k + 1 < pc.r)
-                   ? w * sum_v(pb.ws_part, slot_floats, pc.t, first, count, row * pc.r + k + 1)
-                   : 0.f;
+        const float a = (row < pc.len && k < pc.r) ? S.vsum[row * pc.r + k] : 0.f;
+        const float b = (row < pc.len && k + 1 < pc.r) ? S.vsum[row * pc.r + k + 1] : 0.f;
+        split_pair(a, b, hi[q], lo[q]);
       }
-      uint32_t hi[4], lo[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) split_pair(a[q], b[q], hi[q], lo[q]);
       S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + ln] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
       S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + ln] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     }
+    __syncthreads();
   }
-  __syncthreads();
+  // step 3
   if (vec) {
     if (pc.len == 1) expand_vec<1>(pb, pc, ring_base, S);
     else if (pc.len == 2) expand_vec<2>(pb, pc, ring_base, S);
