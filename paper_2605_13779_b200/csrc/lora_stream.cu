@@ -76,6 +76,11 @@ constexpr int kShrinkBlock = 32;          // elements of d per column block
 constexpr int kExpandBlock = 64;          // elements of n per column block
 constexpr int kShrinkGrain = 128;         // smallest lane share in (row x block) units: 128 x 64 B
 constexpr int kExpandGrain = 64;          //                                           64 x 128 B
+// What starting on a (tile, projection) costs a lane, in column blocks of that tile: the pipeline fill, the
+// barriers and the hand-over of v.  Every projection's columns are preceded by this many empty blocks in
+// the area, so a share that meets several projections gets fewer real blocks.
+constexpr int kShrinkPieceBlocks = 24;
+constexpr int kExpandPieceBlocks = 12;
 constexpr int kMaxParts = 8;              // shrink lanes that may share one tile of one projection
 constexpr int kMaxProblems = MINT_MAX_GROUP;
 
@@ -1186,8 +1191,8 @@ int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void
   pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
   pb.ldx = a.ldx; pb.ldy = a.ldy;
   pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
-  pb.cb0_shrink = 0;
-  pb.cb0_expand = 0;
+  pb.cb0_shrink = kShrinkPieceBlocks;
+  pb.cb0_expand = kExpandPieceBlocks;
   pb.ws_part = static_cast<float *>(workspace);
   P.nprob = 1;
   P.T = a.T;
@@ -1198,8 +1203,8 @@ int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void
   P.pair_weight = a.pair_weight;
   P.x_rows = a.x_rows;
   P.lanes = lanes;
-  P.cb_shrink = (a.d + kShrinkBlock - 1) / kShrinkBlock;
-  P.cb_expand = (a.n + kExpandBlock - 1) / kExpandBlock;
+  P.cb_shrink = kShrinkPieceBlocks + (a.d + kShrinkBlock - 1) / kShrinkBlock;
+  P.cb_expand = kExpandPieceBlocks + (a.n + kExpandBlock - 1) / kExpandBlock;
   P.cb_shrink_widest = P.cb_shrink;
   P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
   P.status = a.status;
@@ -1244,6 +1249,8 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
     pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
     pb.ldx = a.ldx; pb.ldy = a.ldy;
     pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
+    cb_s += kShrinkPieceBlocks;
+    cb_e += kExpandPieceBlocks;
     pb.cb0_shrink = cb_s;
     pb.cb0_expand = cb_e;
     cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
