@@ -79,8 +79,8 @@ constexpr int kExpandGrain = 64;          //                                    
 // What starting on a (tile, projection) costs a lane, in column blocks of that tile: the pipeline fill, the
 // barriers and the hand-over of v.  Every projection's columns are preceded by this many empty blocks in
 // the area, so a share that meets several projections gets fewer real blocks.
-constexpr int kShrinkPieceBlocks = 24;
-constexpr int kExpandPieceBlocks = 12;
+constexpr int kShrinkPieceBlocks = 32;
+constexpr int kExpandPieceBlocks = 16;
 constexpr int kMaxParts = 8;              // shrink lanes that may share one tile of one projection
 constexpr int kMaxProblems = MINT_MAX_GROUP;
 
@@ -705,7 +705,7 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
 constexpr size_t kRingsBytes = (size_t)kWarps * kRingBytes;
 
 template <bool kPacked>
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(const StreamParams P) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(const __grid_constant__ StreamParams P) {
   extern __shared__ __align__(128) uint8_t dyn_smem[];   // the four warps' rings
   __shared__ SmemShrink S;
   pdl_launch_dependents();
@@ -1098,7 +1098,7 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   }
 }
 
-__global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(const StreamParams P) {
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(const __grid_constant__ StreamParams P) {
   extern __shared__ __align__(128) uint8_t dyn_smem[];   // the four warps' rings
   __shared__ SmemExpand S;
   pdl_launch_dependents();

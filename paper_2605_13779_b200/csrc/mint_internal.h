@@ -49,12 +49,13 @@ __host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 
 // tensor-core shapes).  The lanes' shares are equal in this cost.
 #define MINT_TILE_COST_SHRINK 8
 #define MINT_TILE_COST_EXPAND 8
-// (tiles of rank 1 with at most 8 tokens take the FMA path, whose cost does follow the rows)
+// Tiles of rank 1 with at most 8 tokens take the FMA path: a row costs less there, but a
+// piece of such a tile costs its latencies whatever its size (measured per piece and per block).
 __host__ __device__ constexpr int mint_tile_rows_shrink(int rank, int len) {
-  return rank + len + ((rank == 1 && len <= 8) ? 0 : MINT_TILE_COST_SHRINK);
+  return (rank == 1 && len <= 8) ? 5 + len : rank + len + MINT_TILE_COST_SHRINK;
 }
 __host__ __device__ constexpr int mint_tile_rows_expand(int rank, int len) {
-  return rank + 2 * len + ((rank == 1 && len <= 8) ? 0 : MINT_TILE_COST_EXPAND);
+  return (rank == 1 && len <= 8) ? 4 + len : rank + 2 * len + MINT_TILE_COST_EXPAND;
 }
 
 // One tile of list 1 with everything a streaming kernel needs to start on it:
