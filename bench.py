@@ -385,9 +385,14 @@ def run_gpu(args):
                 "frac": achieved / peak, "frac_of_8TBps": achieved / 8000.0, "peak_source": peak_src,
                 "bytes_per_launch": avg_launch_bytes, "avg_launch_us": avg_launch_s * 1e6,
                 "launches_timed": n_apply * args.steps, "traffic": None}
-    traffic_path = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.json")
-    if os.path.exists(traffic_path):
-        roofline["traffic"] = json.load(open(traffic_path)).get("dram_bytes_per_launch")
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch pair, as the ncu summary under profiles/ records it
+    # for this workload and grouping (a line "traffic_bytes_per_launch = N"); null when there is no such record
+    summary = os.path.join(ROOT, "profiles", f"stream_kernels_{args.workload}_{args.grouping}.md")
+    if os.path.exists(summary):
+        import re
+        m = re.search(r"traffic_bytes_per_launch\s*=\s*(\d+)", open(summary).read())
+        if m:
+            roofline["traffic"] = int(m.group(1))
 
     cpu_val, cores, sample = oracle_layer_seconds(wl)
     line = {
