@@ -1,20 +1,23 @@
-// Streamed LoRA apply for dense projections: the fused path of
-// mint_lora_apply_fused and of its grouped form.
+// Streamed LoRA apply: the fused path of mint_lora_apply_fused, of its grouped
+// form and (with the packed per-expert layout) of mint_moe_lora_apply.
 //
 //   shrink_stream_kernel : v[tile] = X[tile rows, :] . A_slot           (d -> r)
 //   expand_stream_kernel : Y[tile rows, :] += s_slot * v[tile] . B_slot  (r -> n)
 //
 // Work split.  The work of a call is the area  rows x column blocks  where
-// rows runs over the plan's tiles (a tile = at most 32 tokens of one segment,
-// contributing rank + len rows to the shrink and rank + 2 len rows to the
-// expand) and columns over the column blocks (32 elements of d for the shrink,
-// 64 elements of n for the expand) of all projections of the call, laid side by
-// side.  The grid is four 128-thread CTAs per SM ("lanes"); lane c takes the
-// c-th equal share of the area, walked tile by tile: a share starts in the
-// middle of one tile, covers whole tiles, and ends in the middle of another.
-// The plan tabulates the tile in which every lane starts (that does not depend
-// on the widths), so a lane finds its work with two table reads, and every lane
-// moves the same number of bytes.
+// rows runs over the plan's tiles (a tile = at most 32 tokens of one segment)
+// and columns over the column blocks (32 elements of d for the shrink, 64
+// elements of n for the expand) of all projections of the call, laid side by
+// side.  A tile counts as many rows as a column block of it costs: the rows it
+// streams (rank + len for the shrink, rank + 2 len for the expand) plus a
+// constant (mint_tile_rows_shrink / _expand), and every projection's columns
+// are preceded by a few empty blocks that stand for the fixed cost of starting
+// on a (tile, projection) piece.  The grid is three 128-thread CTAs per SM
+// ("lanes"); lane c takes the c-th equal share of the area, walked tile by
+// tile: a share starts in the middle of one tile, covers whole tiles, and ends
+// in the middle of another.  The plan tabulates the tile in which every lane
+// starts (that does not depend on the widths), so a lane finds its work with
+// two table reads, and the lanes finish at about the same time.
 //
 // Data path.  Nothing is staged in shared memory: the operand fragments of the
 // warp-level tensor-core MMA (m16n8k16, bf16 in, fp32 accumulate) are loaded
@@ -39,8 +42,8 @@
 //  - tiles of rank 1 with at most 8 tokens (most of a large-catalog decode
 //    batch) skip the MMA: plain fp32 FMAs over fully coalesced 512-byte warp loads.
 // The four warps of a CTA split the column blocks of a piece; HBM latency is
-// hidden by 16 warps per SM, by software prefetch into L2 a few blocks ahead and,
-// before the dependency wait of a launch, by prefetching the weights.
+// hidden by the rings of 12 warps per SM and, before the dependency wait of a
+// launch, by prefetching the weights into L2.
 //
 // v travels from the shrink to the expand through a small L2-resident
 // workspace: every shrink lane writes the sum over its own columns of a tile
