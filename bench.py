@@ -264,7 +264,8 @@ def run_gpu(args):
         for li in range(L):
             enqueue_layer(li)
 
-    kernels_per_call = 2                        # a fused call is a shrink and an expand launch
+    # a fused call is a shrink and an expand launch; batches that may hold dense segments add the two tensor-core kernels
+    kernels_per_call = 4 if (not moe and T >= 4096) else 2
     calls_per_layer = len(groups_idx)
     launches_per_step = 1 + L * calls_per_layer * kernels_per_call
 

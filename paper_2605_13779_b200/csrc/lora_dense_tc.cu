@@ -284,6 +284,220 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   if (warp == 0) tmem_dealloc(tmem_d, kTmemCols);
 }
 
+
+// ====================================================================================
+// Tensor-core expand for dense segments:  Y[128-row tile, :] += s * v[tile] . B_slot   (r -> n).
+//
+// One CTA takes a 128-row tile and a range of kColsPerCta columns of n, 128
+// columns at a time.  v (fp32, left by the tensor-core shrink in the workspace)
+// is scaled by s and split into a bf16 head and a bf16 remainder, both stored
+// once as K-major MMA A operands (128 rows x 64 ranks, 128-byte-swizzled).  B
+// is [rank][n] in memory, n contiguous, which is the wrong way round for a
+// K-major operand: a chunk (64 ranks x 128 columns) is copied as it is into a
+// staging buffer (double buffered, cp.async) and transposed through the
+// registers (ldmatrix.trans, 32-bit stores) into the swizzled K-major layout.
+// Two chains of tcgen05.mma (head, then remainder, M = 128, N = 128, K = 16
+// each) leave Y's update in 128 columns of tensor memory; every thread then
+// reads its row back (tcgen05.ld), adds it to its 256 bytes of y and writes
+// them.  B is read once per 128 tokens (the streamed expand reads it once per
+// 32).  Waits are bounded as in the shrink.
+constexpr int kExpChunk = 128;                 // columns of n per MMA (N)
+constexpr int kColsPerCta = 1024;
+constexpr int kStageRowBytes = kExpChunk * 2 + 16;   // padded: ldmatrix rows fall into different banks
+constexpr int kBStageBytes = kMaxRank * kStageRowBytes;          // 17408
+constexpr int kVBytes = kTileRows * 128;                         // one A operand: 16 KB
+constexpr int kBkmBytes = kExpChunk * 128;                       // 16 KB
+constexpr size_t kExpDynSmem = 2 * kVBytes + kBkmBytes + 2 * kBStageBytes + 1024;
+constexpr int kExpTmemCols = 128;
+
+struct DenseExpandProblem {
+  const uint16_t *B;   // [slot][r_max][n]
+  uint16_t *y;
+  int64_t ldy;
+  int32_t n, r_max;
+  const float *ws_part;
+};
+struct DenseExpandParams {
+  DenseExpandProblem prob[kMaxProblems];
+  int32_t T;
+  int32_t lanes;
+  int32_t dense_slot0;
+  int32_t *status;
+  TableDev tab;
+  PlanView pv;
+};
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr)
+               : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// byte offset of (row, 16-byte chunk c) in a 128-byte-swizzled K-major tile
+__device__ __forceinline__ uint32_t sw128(int row, int c) {
+  return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((c ^ (row & 7)) << 4));
+}
+
+__global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseExpandParams P) {
+  extern __shared__ uint8_t dyn_raw[];
+  __shared__ uint64_t mma_done;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int32_t rows[kTileRows];
+  __shared__ int32_t failed;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const DenseExpandProblem &pb = P.prob[blockIdx.z];
+
+  pdl_launch_dependents();
+  const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
+                  P.pv.header[PH_LANES] == P.lanes;
+  const int m = blockIdx.x;
+  const int col_begin = blockIdx.y * kColsPerCta;
+  if (!ok || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n) {
+    pdl_wait();
+    return;
+  }
+  const int col_end = min(pb.n, col_begin + kColsPerCta);
+  const int ntiles = P.pv.header[PH_NCHUNK1];
+  const int t0 = P.pv.dense_tile[m];
+  const TileDesc d0 = P.pv.tile_desc[t0];
+  int nrows = d0.len;
+  for (int i = 1; i < 4 && nrows == 32 * i && t0 + i < ntiles; ++i) {
+    const TileDesc di = P.pv.tile_desc[t0 + i];
+    if (!di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
+    nrows += di.len;
+  }
+  const int r = d0.rank;
+  if (r > pb.r_max || r > kMaxRank || r < 1) {   // reported by the shrink
+    pdl_wait();
+    return;
+  }
+  const int k_mma = (r + 15) / 16 * 16;
+  for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
+  if (tid == 0) {
+    mbar_init(&mma_done, 1);
+    fence_mbar_init();
+    failed = 0;
+  }
+  if (warp == 0) tmem_alloc(&tmem_base_slot, kExpTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = tmem_base_slot;
+  const uint32_t base = (smem_addr(dyn_raw) + 1023u) & ~1023u;
+  const uint32_t v_hi = base, v_lo = base + kVBytes, b_km = base + 2 * kVBytes;
+  const uint32_t stage0 = b_km + kBkmBytes;
+  const uint16_t *B_rows = pb.B + (int64_t)d0.slot * pb.r_max * pb.n;
+  const uint32_t idesc = instr_desc(kExpChunk);
+  const int nchunks = (col_end - col_begin + kExpChunk - 1) / kExpChunk;
+
+  // B chunk kc into staging buffer kc & 1: rows k < k_mma (zero beyond the rank), 16 x 16-byte pieces per row
+  auto issue = [&](int kc) {
+    if (kc < nchunks) {
+      const uint32_t st = stage0 + (uint32_t)((kc & 1) * kBStageBytes);
+      const int c = tid & 15;
+      const int col = col_begin + kc * kExpChunk + c * 8;
+      for (int k = tid >> 4; k < k_mma; k += 8) {
+        const bool v = k < r && col < col_end;
+        cp_async16(st + (uint32_t)(k * kStageRowBytes + c * 16), v ? B_rows + (int64_t)k * pb.n + col : pb.B, v);
+      }
+    }
+    cp_async_commit();
+  };
+  issue(0);   // weights: not written by any kernel of the stream
+
+  pdl_wait();   // v and y belong to the earlier kernels until here
+
+  // v of this thread's row, scaled, as head and remainder: 16-byte chunks of 8 ranks
+  {
+    const int row = tid;
+    const size_t slot_floats = (size_t)32 * pb.r_max;
+    const float *src = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
+    for (int c = 0; c < k_mma / 8; ++c) {
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int k = c * 8 + 2 * q;
+        const float a = (row < nrows && k < r) ? d0.scale * __ldcg(src + k) : 0.f;
+        const float b = (row < nrows && k + 1 < r) ? d0.scale * __ldcg(src + k + 1) : 0.f;
+        hi[q] = pack_bf16x2(a, b);
+        lo[q] = pack_bf16x2(a - bf16lo(hi[q]), b - bf16hi(hi[q]));
+      }
+      sts128(v_hi + sw128(row, c), make_uint4(hi[0], hi[1], hi[2], hi[3]));
+      sts128(v_lo + sw128(row, c), make_uint4(lo[0], lo[1], lo[2], lo[3]));
+    }
+  }
+
+  uint16_t *yrow = pb.y + (int64_t)rows[tid] * pb.ldy;   // this thread's row of y (tid = accumulator row)
+  for (int kc = 0; kc < nchunks; ++kc) {
+    issue(kc + 1);
+    cp_async_wait<1>();   // this thread's copies of chunk kc have landed
+    __syncthreads();      // ... everybody's; and the MMAs of chunk kc - 1 were waited for by every thread
+    // transpose staging [k][128 columns] into the K-major operand [column][k]:
+    // a transposed 8x8 block gives lane (g, t) the pair (k0 + 2t, k0 + 2t + 1) of column n0 + g
+    {
+      const uint32_t st = stage0 + (uint32_t)((kc & 1) * kBStageBytes);
+      const int g = lane >> 2, t = lane & 3;
+      for (int blk = warp; blk < (k_mma / 8) * (kExpChunk / 32); blk += kThreads / 32) {
+        const int kb = blk / (kExpChunk / 32), nb = blk % (kExpChunk / 32);   // 8 ranks x 32 columns
+        uint32_t q4[4];
+        // matrix i of the x4 = columns nb*32 + 8 i .. + 7; lane L gives the address of row L % 8 of matrix L / 8
+        ldmatrix_x4_trans(q4, st + (uint32_t)((kb * 8 + (lane & 7)) * kStageRowBytes + (nb * 32 + (lane >> 3) * 8) * 2));
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int n = nb * 32 + i * 8 + g;
+          sts32(b_km + sw128(n, kb) + (uint32_t)(t * 4), q4[i]);
+        }
+      }
+    }
+    fence_async_smem();   // the operand writes are visible to the tensor core
+    __syncthreads();
+    if (tid == 0 && !failed) {
+      tc_fence_after();
+      const uint64_t dh = smem_desc_k_sw128(v_hi), dl = smem_desc_k_sw128(v_lo), db = smem_desc_k_sw128(b_km);
+      for (int ks = 0; ks < k_mma / 16; ++ks) umma_bf16(tmem_d, dh + (uint64_t)(2 * ks), db + (uint64_t)(2 * ks), idesc, ks > 0);
+      for (int ks = 0; ks < k_mma / 16; ++ks) umma_bf16(tmem_d, dl + (uint64_t)(2 * ks), db + (uint64_t)(2 * ks), idesc, true);
+      umma_commit(&mma_done);
+    }
+    if (!failed && !mbar_wait(&mma_done, (uint32_t)(kc & 1))) failed = 1;
+    tc_fence_after();
+    if (!__any_sync(0xffffffffu, failed != 0)) {   // the accumulator loads are warp-wide
+      const int col0 = col_begin + kc * kExpChunk;
+#pragma unroll 1
+      for (int j0 = 0; j0 < kExpChunk; j0 += 16) {
+        float acc[16];
+        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, acc);   // warp-wide: every lane takes part
+        if (tid < nrows && col0 + j0 < col_end) {
+          uint4 *yp = reinterpret_cast<uint4 *>(yrow + col0 + j0);
+          const bool second = col0 + j0 + 8 < col_end;
+          uint4 y0 = yp[0], y1 = second ? yp[1] : make_uint4(0u, 0u, 0u, 0u);
+          float f[8];
+          unpack8(y0, f);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) f[e] += acc[e];
+          yp[0] = pack8(f);
+          if (second) {
+            unpack8(y1, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] += acc[8 + e];
+            yp[1] = pack8(f);
+          }
+        }
+      }
+    }
+    tc_fence_before();   // the accumulator reads are done before the next chunk's MMAs overwrite it
+  }
+  cp_async_wait<0>();
+  if (failed && tid == 0) report(P.status, MINT_ERR_TIMEOUT, m);
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_d, kExpTmemCols);
+}
+
 }  // namespace
 
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
@@ -325,4 +539,48 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_shrink_kernel, P), "dense_shrink launch");
+}
+
+
+int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                      (int)kExpDynSmem), "dense_expand shared memory");
+    if (st) return st;
+    attr_set = true;
+  }
+  const int32_t T = args[0].T;
+  const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
+  if (tiles == 0) return MINT_OK;
+  DenseExpandParams P = {};
+  int32_t n_max = 0;
+  for (int i = 0; i < nprob; ++i) {
+    DenseExpandProblem &pb = P.prob[i];
+    pb.B = args[i].B;
+    pb.y = args[i].y;
+    pb.ldy = args[i].ldy;
+    pb.n = args[i].n;
+    pb.r_max = args[i].r_max;
+    pb.ws_part = static_cast<const float *>(workspaces[i]);
+    n_max = pb.n > n_max ? pb.n : n_max;
+  }
+  P.T = T;
+  P.lanes = lanes;
+  P.dense_slot0 = dense_slot0;
+  P.status = args[0].status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)((n_max + kColsPerCta - 1) / kColsPerCta), (unsigned)nprob);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kExpDynSmem;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_expand_kernel, P), "dense_expand launch");
 }

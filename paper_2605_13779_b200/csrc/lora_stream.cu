@@ -331,7 +331,7 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     const int va = (t == R.t0) ? R.cb0 : 0;
     const int vb = (t == R.t1) ? R.cb1 : area.CB;
     if (va >= vb) continue;
-    if (!kExpand && sh.desc[ti].dense) continue;   // its shrink runs on the 128-row tensor-core kernel
+    if (sh.desc[ti].dense) continue;   // it runs on the 128-row tensor-core kernels
     Piece pc;
     pc.t = t;
     pc.ti = ti;
@@ -1287,11 +1287,14 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   cfg.numAttrs = 1;
   st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
   if (st) return st;
-  if (T >= MINT_DENSE_MIN_BATCH) {   // the plan may have given dense segments to the tensor-core shrink
+  const bool dense = T >= MINT_DENSE_MIN_BATCH;   // the plan may have given dense segments to the tensor-core kernels
+  if (dense) {
     st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);
     if (st) return st;
   }
-  return mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
+  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
+  if (st || !dense) return st;
+  return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);
 }
 
 // ---- fused apply without a caller-provided workspace -------------------------------

@@ -77,7 +77,7 @@ struct __align__(16) TileDesc {
   int32_t rows_expand;
   int32_t lane_lo;
   int32_t lane_hi;
-  int32_t dense;   // 1: the tile belongs to a dense segment; its shrink runs on the 128-row tensor-core kernel
+  int32_t dense;   // 1: the tile belongs to a dense segment; it runs on the 128-row tensor-core kernels
   int32_t pad1;
 };
 
@@ -202,6 +202,9 @@ bool mint_stream_supported(int32_t max_bound_rank);
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);
 // Tensor-core shrink of the dense segments' 128-row tiles (between the two streamed kernels).
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s);
+// Tensor-core expand of the same tiles (after the streamed expand, which skips them).
+int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                  void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s);
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);

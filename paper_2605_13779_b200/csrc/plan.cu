@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
         sum_s += mint_tile_rows_shrink(r, len);
         atomicMax(&counters[7], mint_tile_rows_shrink(r, len));
       }
-      sum_e += mint_tile_rows_expand(r, len);
+      if (!is_dense(sg)) sum_e += mint_tile_rows_expand(r, len);
     }
     int run_s = block_exclusive_scan(sum_s, warp_tot, rows_total[0]);
     int run_e = block_exclusive_scan(sum_e, warp_tot, rows_total[1]);
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       if (dsc.dense && ((toff[c] - seg_start[sg]) % 128) == 0) dense_tile[run_m++] = c;
       const int begin[2] = {run_s, run_e};
       const int end[2] = {run_s + (dsc.dense ? 0 : mint_tile_rows_shrink(dsc.rank, dsc.len)),
-                          run_e + mint_tile_rows_expand(dsc.rank, dsc.len)};
+                          run_e + (dsc.dense ? 0 : mint_tile_rows_expand(dsc.rank, dsc.len))};
       // shrink lanes that can meet this tile: from the last lane starting at or
       // before the tile's first row to the last lane starting before its end
       dsc.lane_lo = dsc.lane_hi = 0;
