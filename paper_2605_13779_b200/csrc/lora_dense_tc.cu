@@ -294,20 +294,27 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
 // once as K-major MMA A operands (128 rows x 64 ranks, 128-byte-swizzled).  B
 // is [rank][n] in memory, n contiguous, which is the wrong way round for a
 // K-major operand: a chunk (64 ranks x 128 columns) is copied as it is into a
-// staging buffer (double buffered, cp.async) and transposed through the
-// registers (ldmatrix.trans, 32-bit stores) into the swizzled K-major layout.
-// Two chains of tcgen05.mma (head, then remainder, M = 128, N = 128, K = 16
-// each) leave Y's update in 128 columns of tensor memory; every thread then
-// reads its row back (tcgen05.ld), adds it to its 256 bytes of y and writes
-// them.  B is read once per 128 tokens (the streamed expand reads it once per
-// 32).  Waits are bounded as in the shrink.
+// staging buffer (cp.async) and transposed through the registers
+// (ldmatrix.trans, 32-bit stores) into the swizzled K-major layout; the next
+// chunk's copy starts as soon as the staging buffer has been read.  Two chains
+// of tcgen05.mma (head, then remainder, M = 128, N = 128, K = 16 each) leave
+// Y's update in 128 columns of tensor memory.  The 128 x 128 tile of y comes
+// into shared memory with coalesced 16-byte copies while all that happens;
+// every thread then adds its accumulator row (tcgen05.ld) to its row of the
+// tile, and the warp writes its 32 rows back to memory, two whole rows per
+// store instruction.  (A thread reading and writing its row of y in memory
+// directly touches 32 cache lines per instruction; that version ran at a third
+// of the speed.)  B is read once per 128 tokens; the streamed expand reads it
+// once per 32.  Waits are bounded as in the shrink.
 constexpr int kExpChunk = 128;                 // columns of n per MMA (N)
-constexpr int kColsPerCta = 1024;
-constexpr int kStageRowBytes = kExpChunk * 2 + 16;   // padded: ldmatrix rows fall into different banks
+constexpr int kColsPerCta = 2048;
+constexpr int kStageRowBytes = kExpChunk * 2 + 16;   // padded: rows of a transposing 8x8 load fall into different banks
 constexpr int kBStageBytes = kMaxRank * kStageRowBytes;          // 17408
+constexpr int kYRowBytes = kExpChunk * 2 + 16;                   // padded: a warp's 16-byte accesses to 8 rows do not collide
+constexpr int kYTileBytes = kTileRows * kYRowBytes;              // 34816
 constexpr int kVBytes = kTileRows * 128;                         // one A operand: 16 KB
 constexpr int kBkmBytes = kExpChunk * 128;                       // 16 KB
-constexpr size_t kExpDynSmem = 2 * kVBytes + kBkmBytes + 2 * kBStageBytes + 1024;
+constexpr size_t kExpDynSmem = 2 * kVBytes + kBkmBytes + kBStageBytes + kYTileBytes + 1024;
 constexpr int kExpTmemCols = 128;
 
 struct DenseExpandProblem {
@@ -338,6 +345,11 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v) {
 }
 __device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
   asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 r;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr) : "memory");
+  return r;
 }
 // byte offset of (row, 16-byte chunk c) in a 128-byte-swizzled K-major tile
 __device__ __forceinline__ uint32_t sw128(int row, int c) {
@@ -391,63 +403,82 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
   const uint32_t tmem_d = tmem_base_slot;
   const uint32_t base = (smem_addr(dyn_raw) + 1023u) & ~1023u;
   const uint32_t v_hi = base, v_lo = base + kVBytes, b_km = base + 2 * kVBytes;
-  const uint32_t stage0 = b_km + kBkmBytes;
+  const uint32_t stage = b_km + kBkmBytes, ytile = stage + kBStageBytes;
   const uint16_t *B_rows = pb.B + (int64_t)d0.slot * pb.r_max * pb.n;
   const uint32_t idesc = instr_desc(kExpChunk);
   const int nchunks = (col_end - col_begin + kExpChunk - 1) / kExpChunk;
 
-  // B chunk kc into staging buffer kc & 1: rows k < k_mma (zero beyond the rank), 16 x 16-byte pieces per row
-  auto issue = [&](int kc) {
+  // B chunk kc into the staging buffer: rows k < k_mma (zero beyond the rank), 16 x 16-byte pieces per row
+  auto issue_b = [&](int kc) {
     if (kc < nchunks) {
-      const uint32_t st = stage0 + (uint32_t)((kc & 1) * kBStageBytes);
       const int c = tid & 15;
       const int col = col_begin + kc * kExpChunk + c * 8;
       for (int k = tid >> 4; k < k_mma; k += 8) {
         const bool v = k < r && col < col_end;
-        cp_async16(st + (uint32_t)(k * kStageRowBytes + c * 16), v ? B_rows + (int64_t)k * pb.n + col : pb.B, v);
+        cp_async16(stage + (uint32_t)(k * kStageRowBytes + c * 16), v ? B_rows + (int64_t)k * pb.n + col : pb.B, v);
       }
     }
     cp_async_commit();
   };
-  issue(0);   // weights: not written by any kernel of the stream
+  // the y tile of chunk kc: 16 consecutive threads copy the 256 bytes of a row
+  auto issue_y = [&](int kc) {
+    const int c = tid & 15;
+    const int col = col_begin + kc * kExpChunk + c * 8;
+#pragma unroll 4
+    for (int row = tid >> 4; row < kTileRows; row += 8) {
+      const bool v = row < nrows && col < col_end;
+      cp_async16(ytile + (uint32_t)(row * kYRowBytes + c * 16), v ? pb.y + (int64_t)rows[row] * pb.ldy + col : pb.y, v);
+    }
+    cp_async_commit();
+  };
+  issue_b(0);   // weights: not written by any kernel of the stream
 
   pdl_wait();   // v and y belong to the earlier kernels until here
 
-  // v of this thread's row, scaled, as head and remainder: 16-byte chunks of 8 ranks
+  // v, scaled, as head and remainder: consecutive threads take consecutive pairs of ranks of a row
   {
-    const int row = tid;
     const size_t slot_floats = (size_t)32 * pb.r_max;
-    const float *src = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
-    for (int c = 0; c < k_mma / 8; ++c) {
-      uint32_t hi[4], lo[4];
+    const int pairs = k_mma / 2;
+    for (int q0 = tid; q0 < kTileRows * pairs; q0 += 8 * kThreads) {
+      float a[8], b[8];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int k = c * 8 + 2 * q;
-        const float a = (row < nrows && k < r) ? d0.scale * __ldcg(src + k) : 0.f;
-        const float b = (row < nrows && k + 1 < r) ? d0.scale * __ldcg(src + k + 1) : 0.f;
-        hi[q] = pack_bf16x2(a, b);
-        lo[q] = pack_bf16x2(a - bf16lo(hi[q]), b - bf16hi(hi[q]));
+      for (int u = 0; u < 8; ++u) {
+        const int q = q0 + u * kThreads;
+        const int row = q / pairs, k = 2 * (q - row * pairs);
+        const bool in = q < kTileRows * pairs && row < nrows;
+        const float *src = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
+        a[u] = (in && k < r) ? __ldcg(src + k) : 0.f;
+        b[u] = (in && k + 1 < r) ? __ldcg(src + k + 1) : 0.f;
       }
-      sts128(v_hi + sw128(row, c), make_uint4(hi[0], hi[1], hi[2], hi[3]));
-      sts128(v_lo + sw128(row, c), make_uint4(lo[0], lo[1], lo[2], lo[3]));
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int q = q0 + u * kThreads;
+        if (q < kTileRows * pairs) {
+          const int row = q / pairs, k = 2 * (q - row * pairs);
+          const float fa = d0.scale * a[u], fb = d0.scale * b[u];
+          const uint32_t hi = pack_bf16x2(fa, fb);
+          const uint32_t lo = pack_bf16x2(fa - bf16lo(hi), fb - bf16hi(hi));
+          const uint32_t off = sw128(row, k >> 3) + (uint32_t)((k & 7) * 2);
+          sts32(v_hi + off, hi);
+          sts32(v_lo + off, lo);
+        }
+      }
     }
   }
 
-  uint16_t *yrow = pb.y + (int64_t)rows[tid] * pb.ldy;   // this thread's row of y (tid = accumulator row)
   for (int kc = 0; kc < nchunks; ++kc) {
-    issue(kc + 1);
-    cp_async_wait<1>();   // this thread's copies of chunk kc have landed
+    issue_y(kc);          // (the previous chunk's tile was stored and all warps passed a barrier since)
+    cp_async_wait<1>();   // this thread's copies of B chunk kc have landed (the y tile may still be on its way)
     __syncthreads();      // ... everybody's; and the MMAs of chunk kc - 1 were waited for by every thread
     // transpose staging [k][128 columns] into the K-major operand [column][k]:
     // a transposed 8x8 block gives lane (g, t) the pair (k0 + 2t, k0 + 2t + 1) of column n0 + g
     {
-      const uint32_t st = stage0 + (uint32_t)((kc & 1) * kBStageBytes);
       const int g = lane >> 2, t = lane & 3;
       for (int blk = warp; blk < (k_mma / 8) * (kExpChunk / 32); blk += kThreads / 32) {
         const int kb = blk / (kExpChunk / 32), nb = blk % (kExpChunk / 32);   // 8 ranks x 32 columns
         uint32_t q4[4];
         // matrix i of the x4 = columns nb*32 + 8 i .. + 7; lane L gives the address of row L % 8 of matrix L / 8
-        ldmatrix_x4_trans(q4, st + (uint32_t)((kb * 8 + (lane & 7)) * kStageRowBytes + (nb * 32 + (lane >> 3) * 8) * 2));
+        ldmatrix_x4_trans(q4, stage + (uint32_t)((kb * 8 + (lane & 7)) * kStageRowBytes + (nb * 32 + (lane >> 3) * 8) * 2));
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int n = nb * 32 + i * 8 + g;
@@ -456,7 +487,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
       }
     }
     fence_async_smem();   // the operand writes are visible to the tensor core
-    __syncthreads();
+    __syncthreads();      // the staging buffer has been read by everybody
+    issue_b(kc + 1);
     if (tid == 0 && !failed) {
       tc_fence_after();
       const uint64_t dh = smem_desc_k_sw128(v_hi), dl = smem_desc_k_sw128(v_lo), db = smem_desc_k_sw128(b_km);
@@ -464,33 +496,42 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
       for (int ks = 0; ks < k_mma / 16; ++ks) umma_bf16(tmem_d, dl + (uint64_t)(2 * ks), db + (uint64_t)(2 * ks), idesc, true);
       umma_commit(&mma_done);
     }
+    cp_async_wait<1>();   // this thread's copies of the y tile have landed (B chunk kc + 1 may still be on its way)
     if (!failed && !mbar_wait(&mma_done, (uint32_t)(kc & 1))) failed = 1;
     tc_fence_after();
+    __syncthreads();      // everybody's copies of the y tile have landed
+    const int col0 = col_begin + kc * kExpChunk;
     if (!__any_sync(0xffffffffu, failed != 0)) {   // the accumulator loads are warp-wide
-      const int col0 = col_begin + kc * kExpChunk;
-#pragma unroll 1
+      // this thread's row of the tile: y += accumulator
+      const uint32_t yr = ytile + (uint32_t)(tid * kYRowBytes);
+#pragma unroll
       for (int j0 = 0; j0 < kExpChunk; j0 += 16) {
         float acc[16];
-        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, acc);   // warp-wide: every lane takes part
-        if (tid < nrows && col0 + j0 < col_end) {
-          uint4 *yp = reinterpret_cast<uint4 *>(yrow + col0 + j0);
-          const bool second = col0 + j0 + 8 < col_end;
-          uint4 y0 = yp[0], y1 = second ? yp[1] : make_uint4(0u, 0u, 0u, 0u);
+        tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, acc);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
           float f[8];
-          unpack8(y0, f);
+          unpack8(lds128(yr + (uint32_t)((j0 + 8 * h) * 2)), f);
 #pragma unroll
-          for (int e = 0; e < 8; ++e) f[e] += acc[e];
-          yp[0] = pack8(f);
-          if (second) {
-            unpack8(y1, f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) f[e] += acc[8 + e];
-            yp[1] = pack8(f);
-          }
+          for (int e = 0; e < 8; ++e) f[e] += acc[8 * h + e];
+          sts128(yr + (uint32_t)((j0 + 8 * h) * 2), pack8(f));
+        }
+      }
+      __syncwarp();
+      // the warp's 32 rows go back to memory, two rows (2 x 256 bytes) per instruction
+      const int c = lane & 15;
+      if (col0 + c * 8 < col_end) {
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+          const int row = warp * 32 + 2 * i + (lane >> 4);
+          if (row < nrows)
+            *reinterpret_cast<uint4 *>(pb.y + (int64_t)rows[row] * pb.ldy + col0 + c * 8) =
+                lds128(ytile + (uint32_t)(row * kYRowBytes + c * 16));
         }
       }
     }
     tc_fence_before();   // the accumulator reads are done before the next chunk's MMAs overwrite it
+    __syncthreads();      // the y tile is free for the next chunk's copies
   }
   cp_async_wait<0>();
   if (failed && tid == 0) report(P.status, MINT_ERR_TIMEOUT, m);
