@@ -256,6 +256,8 @@ __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, A
   }
   const int ntiles = P.pv.header[PH_NCHUNK1];
   if (ntiles == 0) return false;
+  // nothing streamed: every tile belongs to a dense segment (the tensor-core kernels take those)
+  if (P.pv.header[kExpand ? PH_ROWS_EXPAND : PH_ROWS_SHRINK] == 0) return false;
   area = make_area<kExpand>(P);
   const int c = blockIdx.x;
   if (c >= area.active) return false;
