@@ -208,9 +208,9 @@ def dense_segment_case(name, lengths, adapters, ranks, d, n, r_max):
     return synth.DenseCase(name, T, d, n, r_max, table, ids, A, B, x, y0)
 
 
-def test_dense_segments_take_the_tensor_core_shrink():
+def test_dense_segments_take_the_tensor_core_kernels():
     """A batch of more than 4096 tokens with segments of 128 tokens and more: their
-    shrink runs on the tcgen05 kernel (full and ragged 128-row tiles, ranks that are
+    shrink and their expand run on the tcgen05 kernels (full and ragged 128-row tiles, ranks that are
     not multiples of 16, an adapter whose tokens are not contiguous), short segments
     and tokens without adapter stay on the streamed path."""
     lengths = [700, 130, 128, 127, 300, 5, 1, 1000, 64, 513, 256, 129, 3, 640, 384, 40]
@@ -219,6 +219,33 @@ def test_dense_segments_take_the_tensor_core_shrink():
     case = dense_segment_case("gpu/dense-tc", lengths, adapters, ranks, d=1032, n=520, r_max=64)
     assert case.T >= 4096
     check_case(case, "dense segments")
+
+
+def test_dense_segments_grouped_projections_of_different_widths():
+    """Two projections in one grouped call over a batch with dense segments: the
+    tensor-core expand splits a wide n into several column ranges per 128-row tile
+    (with a ragged last chunk), and the narrow projection leaves part of the grid
+    without work."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    lengths = [900, 128, 257, 60, 1100, 131, 2, 640, 512, 400]
+    adapters = [0, 1, 2, 3, 4, 5, 3, 0, 6, -1]
+    ranks = [64, 24, 16, 8, 40, 1, 64]
+    wide = dense_segment_case("gpu/dense-tc/wide", lengths, adapters, ranks, d=520, n=2184, r_max=64)
+    narrow = dense_segment_case("gpu/dense-tc/narrow", lengths, adapters, ranks, d=520, n=264, r_max=64)
+    assert wide.T >= 4096
+    devs = [harness.upload_dense(c) for c in (wide, narrow)]
+    table, status = devs[0].table, devs[0].status
+    plan = mb.mint_lora_plan(table, devs[0].ids, status)
+    ws = [mb.new_workspace(dv.pool, wide.T) for dv in devs]
+    group = mb.ApplyGroup([(dv.pool, dv.x, dv.y, w) for dv, w in zip(devs, ws)])
+    mb.mint_lora_apply_fused_grouped(group, table, plan, status)
+    torch.cuda.synchronize()
+    assert status[0].item() == 0
+    for dv, c in zip(devs, (wide, narrow)):
+        y_ref, _, _ = parity.oracle_dense(c)
+        parity.assert_close(harness.y_to_f64(dv.y), y_ref, c.name)
+        none = c.ids < 0
+        np.testing.assert_array_equal(harness.y_to_f64(dv.y)[none], synth.bf16_bits_to_f64(c.y0)[none])
 
 
 def test_dense_segments_config3_shape_sampled():
