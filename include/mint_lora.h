@@ -205,8 +205,9 @@ int32_t mint_lora_expand(const mint_pool *pool, const mint_slot_table *table, co
  * initialisation (every call writes each entry before it reads it).  Calls
  * that share a workspace must be ordered on one stream.  Batches of 4096 tokens
  * and more whose plan holds runs of 128 and more tokens of one adapter
- * (segmented prefill) run the d -> r contraction of those runs on the tcgen05
- * tensor cores; the result is the same.                                        */
+ * (segmented prefill) run both contractions of those runs (d -> r, and r -> n
+ * with the update of y) on the tcgen05 tensor cores in 128-token tiles; the
+ * result is the same.                                                         */
 size_t mint_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T);
 int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_table *table,
                               const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,

@@ -1,4 +1,6 @@
-// Tensor-core shrink for dense segments:  v[128-row tile] = X[tile rows, :] . A_slot^T   (d -> r).
+// Tensor-core kernels for dense segments.  First the shrink:
+//   v[128-row tile] = X[tile rows, :] . A_slot^T   (d -> r);
+// the expand (r -> n with the update of y) follows further down.
 //
 // A segmented-prefill batch holds runs of hundreds of tokens of one adapter; for
 // those the d -> r contraction is a genuinely dense [128 x d] . [d x r] product
