@@ -966,35 +966,41 @@ __device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece 
 
 // The shrink lanes whose share met the columns of problem p in the tile: they
 // are consecutive lanes, found from the area arithmetic of the shrink kernel
-// alone (one thread per piece of the batch).
+// alone.  Eight threads share one (tile, problem): thread k looks at the
+// candidate lanes c_a + k, c_a + k + 8, ... (all its table reads go out
+// together), and the eight combine their findings with shuffles.  All threads
+// of the CTA call this together; item = the (tile, problem) of this group of
+// eight threads, valid = whether there is one.
 __device__ __forceinline__ void shrink_parts(const StreamParams &P, const Area &sa, const TileDesc &d, int p,
-                                             int &first, int &count) {
-  const StreamProblem &pb = P.prob[p];
+                                             bool valid, int &first, int &count) {
+  const int k = threadIdx.x & 7;
+  const StreamProblem &pb = P.prob[valid ? p : 0];
   const int w_t = tile_rows<false>(d.rank, d.len);
   const int blocks = (pb.d + kShrinkBlock - 1) / kShrinkBlock;
   const int span = w_t * sa.CB;   // the tile's extent in area units
   // active lanes c with table index in [lane_lo, lane_hi]: index(c) = c G / active
   const int c_a = (int)(((unsigned)(d.lane_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
   const int c_b = (int)(((unsigned)(d.lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
-  first = 0;
-  count = 0;
-  if (d.dense) {   // the tensor-core shrink leaves the complete v of the tile in the slot dense_slot0 + tile
-    first = P.dense_slot0;
-    count = 1;
-    return;
-  }
-  int64_t p0 = lane_offset(sa, sa.table[lane_index(sa, c_a)], d.rows_shrink);
-  for (int c2 = c_a; c2 <= c_b; ++c2) {
-    const int64_t p1 = lane_offset(sa, sa.table[lane_index(sa, c2 + 1)], d.rows_shrink);
-    if (p0 < span && p1 > 0) {
-      const int va = p0 <= 0 ? 0 : (int)p0 / w_t;
-      const int vb = p1 >= span ? sa.CB : (int)p1 / w_t;
-      if (max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks)) {
-        if (count == 0) first = c2;
-        ++count;
+  unsigned long long mask = 0;   // bit i: lane c_a + i holds a part
+  if (valid && !d.dense) {
+    for (int i = k; c_a + i <= c_b && i < 64; i += 8) {
+      const int c2 = c_a + i;
+      const int64_t p0 = lane_offset(sa, sa.table[lane_index(sa, c2)], d.rows_shrink);
+      const int64_t p1 = lane_offset(sa, sa.table[lane_index(sa, c2 + 1)], d.rows_shrink);
+      if (p0 < span && p1 > 0) {
+        const int va = p0 <= 0 ? 0 : (int)p0 / w_t;
+        const int vb = p1 >= span ? sa.CB : (int)p1 / w_t;
+        if (max(va, pb.cb0_shrink) < min(vb, pb.cb0_shrink + blocks)) mask |= 1ull << i;
       }
     }
-    p0 = p1;
+  }
+#pragma unroll
+  for (int o = 1; o < 8; o <<= 1) mask |= __shfl_xor_sync(0xffffffffu, mask, o);
+  first = mask ? c_a + __ffsll((long long)mask) - 1 : 0;
+  count = __popcll(mask);
+  if (valid && d.dense) {   // the tensor-core shrink leaves the complete v of the tile in the slot dense_slot0 + tile
+    first = P.dense_slot0;
+    count = 1;
   }
 }
 
@@ -1124,12 +1130,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
     const int ntile = min(kBatchTiles, R.t_end - tb);
     load_batch<false>(P, S.sh, tb, ntile);
     // which shrink lanes hold the parts of v of every (tile, projection) of the batch
-    for (int i = threadIdx.x; i < ntile * P.nprob; i += kThreads) {
-      const int ti = i / P.nprob, p = i - ti * P.nprob;
+    for (int i0 = 0; i0 < ntile * P.nprob; i0 += kThreads / 8) {
+      const int i = i0 + (int)(threadIdx.x >> 3);
+      const bool valid = i < ntile * P.nprob;
+      const int ti = valid ? i / P.nprob : 0, p = valid ? i - ti * P.nprob : 0;
       int first, count;
-      shrink_parts(P, shrink_area, S.sh.desc[ti], p, first, count);
-      S.sh.part_first[ti * kMaxProblems + p] = first;
-      S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
+      shrink_parts(P, shrink_area, S.sh.desc[ti], p, valid, first, count);
+      if (valid && (threadIdx.x & 7) == 0) {
+        S.sh.part_first[ti * kMaxProblems + p] = first;
+        S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
+      }
     }
     if (!waited) {
       // while the shrink kernel still runs: pull this lane's B rows into L2
