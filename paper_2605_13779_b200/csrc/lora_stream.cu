@@ -247,6 +247,12 @@ struct CtaShared {
 template <bool kExpand>
 __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, Area &area, CtaRange &R,
                                          bool report_errors) {
+  // With every lane active (any call that is not tiny) lane c starts at table entry c:
+  // that entry is requested together with the header words, not after them.
+  const int c = blockIdx.x;
+  const LaneStart *table = kExpand ? P.pv.lane_expand : P.pv.lane_shrink;
+  LaneStart ls = {};
+  if (threadIdx.x < 2) ls = table[min(c + (int)threadIdx.x, P.lanes)];
   if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi,
                report_errors ? P.status : nullptr))
     return false;
@@ -259,17 +265,11 @@ __device__ __forceinline__ bool prologue(const StreamParams &P, CtaShared &sh, A
   // nothing streamed: every tile belongs to a dense segment (the tensor-core kernels take those)
   if (P.pv.header[kExpand ? PH_ROWS_EXPAND : PH_ROWS_SHRINK] == 0) return false;
   area = make_area<kExpand>(P);
-  const int c = blockIdx.x;
   if (c >= area.active) return false;
   if (threadIdx.x < 2) {   // thread 0: the cut where this lane starts; thread 1: where it ends
     const int j = lane_index(area, c + threadIdx.x);
-    const LaneStart ls = area.table[j];
-    int cb = 0;
-    if (j < area.G) {
-      const TileDesc d = P.pv.tile_desc[ls.tile];
-      cb = (int)(lane_offset(area, ls, kExpand ? d.rows_expand : d.rows_shrink) /
-                 tile_rows<kExpand>(d.rank, d.len));
-    }
+    if (j != c + (int)threadIdx.x) ls = area.table[j];   // a small call: fewer lanes than the table has
+    const int cb = j < area.G ? (int)(lane_offset(area, ls, ls.rows) / ls.w) : 0;
     sh.range[2 * threadIdx.x] = ls.tile;
     sh.range[2 * threadIdx.x + 1] = cb;
   }
@@ -1128,7 +1128,22 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
   bool waited = false;
   for (int tb = R.t0; tb < R.t_end; tb += kBatchTiles) {
     const int ntile = min(kBatchTiles, R.t_end - tb);
-    load_batch<false>(P, S.sh, tb, ntile);
+    // descriptors first; then the row indices and the lane-table entries are requested together
+    __syncthreads();   // every warp is done with the previous batch
+    {
+      const int4 *src = reinterpret_cast<const int4 *>(P.pv.tile_desc + tb);
+      int4 *dst = reinterpret_cast<int4 *>(S.sh.desc);
+      for (int i = threadIdx.x; i < ntile * (int)(sizeof(TileDesc) / 16); i += kThreads) dst[i] = src[i];
+    }
+    __syncthreads();
+    const int off0 = S.sh.desc[0].off;
+    const int nitems = S.sh.desc[ntile - 1].off + S.sh.desc[ntile - 1].len - off0;
+    int row_of[kBatchItems / kThreads];
+#pragma unroll
+    for (int u = 0; u < kBatchItems / kThreads; ++u) {
+      const int i = threadIdx.x + u * kThreads;
+      row_of[u] = i < nitems ? P.pv.perm[off0 + i] : 0;
+    }
     // which shrink lanes hold the parts of v of every (tile, projection) of the batch
     for (int i0 = 0; i0 < ntile * P.nprob; i0 += kThreads / 8) {
       const int i = i0 + (int)(threadIdx.x >> 3);
@@ -1140,6 +1155,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
         S.sh.part_first[ti * kMaxProblems + p] = first;
         S.sh.part_count[ti * kMaxProblems + p] = (int16_t)count;
       }
+    }
+#pragma unroll
+    for (int u = 0; u < kBatchItems / kThreads; ++u) {
+      const int i = threadIdx.x + u * kThreads;
+      if (i < nitems) S.sh.rows[i] = row_of[u];
     }
     if (!waited) {
       // while the shrink kernel still runs: pull this lane's B rows into L2

@@ -92,11 +92,15 @@ struct __align__(16) TileDesc {
 // Start of cost lane j in the rows x column-blocks area: the tile that holds it
 // and j * rows_total = q * G + r, so that the position for CB column blocks is
 // q * CB + r * CB / G without any 64-bit division.
+// rows / w: the row prefix sum and the row count of that tile, so that a lane
+// finds its first column block without reading the tile's descriptor.
 struct __align__(16) LaneStart {
   int32_t tile;
   int32_t q;
   int32_t r;
-  int32_t pad;
+  int32_t rows;
+  int32_t w;
+  int32_t pad[3];
 };
 
 // Byte offsets of every array inside the plan blob (host-computed, passed by value).

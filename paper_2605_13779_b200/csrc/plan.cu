@@ -328,7 +328,11 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
         if (tot == 0 || begin[q] == end[q]) continue;
         const int64_t j_lo = (begin[q] * G + tot - 1) / tot;
         const int64_t j_hi = (end[q] * G + tot - 1) / tot;   // exclusive
-        for (int64_t j = j_lo; j < j_hi && j < G; ++j) lane_tab[q][j].tile = c;
+        for (int64_t j = j_lo; j < j_hi && j < G; ++j) {
+          lane_tab[q][j].tile = c;
+          lane_tab[q][j].rows = begin[q];
+          lane_tab[q][j].w = end[q] - begin[q];
+        }
       }
       run_s = end[0];
       run_e = end[1];
@@ -339,8 +343,12 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
         const int64_t jw = (int64_t)j * rows_total[q];
         lane_tab[q][j].q = (int32_t)(jw / G);
         lane_tab[q][j].r = (int32_t)(jw % G);
-        lane_tab[q][j].pad = 0;
-        if (j == p.lanes || rows_total[q] == 0) lane_tab[q][j].tile = (j == p.lanes) ? ntile : 0;
+        lane_tab[q][j].pad[0] = lane_tab[q][j].pad[1] = lane_tab[q][j].pad[2] = 0;
+        if (j == p.lanes || rows_total[q] == 0) {
+          lane_tab[q][j].tile = (j == p.lanes) ? ntile : 0;
+          lane_tab[q][j].rows = 0;
+          lane_tab[q][j].w = 1;
+        }
       }
     }
   }
