@@ -40,7 +40,13 @@ enum {
 #define MINT_NUM_TILE_LISTS 2
 #define MINT_MAX_LANES 1024
 // Tile list g cuts every segment into runs of at most mint_tile_tokens(g) items.
+// In list 1, the list of the streamed kernels, the segments of rank-1 adapters
+// (other than dense segments) are cut into runs of 8 instead: a rank-1 tile of
+// up to 8 tokens takes the FMA path, which costs a fraction of what a tensor-core
+// tile of rank 1 costs (one useful column in eight), for one more read of the
+// single row of A and of B per 8 tokens.
 __host__ __device__ constexpr int mint_tile_tokens(int g) { return g == 0 ? 8 : 32; }
+__host__ __device__ constexpr int mint_tile_tokens_rank1(int g) { return 8; }
 
 // Cost of a tile per column block, in rows of streamed bytes: the rows it moves
 // (rank + len for the shrink, rank + 2 len for the expand: y is read and

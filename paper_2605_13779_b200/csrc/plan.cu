@@ -236,20 +236,33 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     s0 = lo;
   }
   int tile_total[MINT_NUM_TILE_LISTS];
+  // dense segments (segmented prefill): dense plans of large batches only
+  const bool dense_plan = p.expert_ids == nullptr && P >= MINT_DENSE_MIN_BATCH;
+  auto tile_len = [&](int g, int sg) {   // the run length list g cuts segment sg into
+    const bool dense_seg = dense_plan && seg_start[sg + 1] - seg_start[sg] >= MINT_DENSE_MIN_SEGMENT;
+    return (p.tab.slot_rank[seg_slot[sg]] == 1 && !dense_seg) ? mint_tile_tokens_rank1(g) : mint_tile_tokens(g);
+  };
 #pragma unroll
   for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
-    const int G = mint_tile_tokens(g);
     int cnt = 0, s = s0;
+    int G = r_begin < r_end ? tile_len(g, s) : 1;
     for (int i = r_begin; i < r_end; ++i) {
-      while (i >= seg_start[s + 1]) ++s;
+      while (i >= seg_start[s + 1]) {
+        ++s;
+        G = tile_len(g, s);
+      }
       cnt += ((i - seg_start[s]) % G) == 0;
     }
     int pos = block_exclusive_scan(cnt, warp_tot, tile_total[g]);
     int32_t *tseg = reinterpret_cast<int32_t *>(p.blob + p.off.tile_seg[g]);
     int32_t *toff = reinterpret_cast<int32_t *>(p.blob + p.off.tile_off[g]);
     s = s0;
+    G = r_begin < r_end ? tile_len(g, s) : 1;
     for (int i = r_begin; i < r_end; ++i) {
-      while (i >= seg_start[s + 1]) ++s;
+      while (i >= seg_start[s + 1]) {
+        ++s;
+        G = tile_len(g, s);
+      }
       if (((i - seg_start[s]) % G) == 0) {
         tseg[pos] = s;
         toff[pos] = i;
@@ -274,13 +287,12 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     const int ntile = tile_total[1];
     const int per = (ntile + kThreads - 1) / kThreads;
     const int c_begin = min(ntile, tid * per), c_end = min(ntile, (tid + 1) * per);
-    // dense segments (segmented prefill): dense plans of large batches only
-    const bool dense_on = p.expert_ids == nullptr && P >= MINT_DENSE_MIN_BATCH;
+    const bool dense_on = dense_plan;
     auto is_dense = [&](int sg) { return dense_on && seg_start[sg + 1] - seg_start[sg] >= MINT_DENSE_MIN_SEGMENT; };
     int sum_s = 0, sum_e = 0, sum_m = 0;
     for (int c = c_begin; c < c_end; ++c) {
       const int sg = tseg[c];
-      const int len = min(mint_tile_tokens(1), seg_start[sg + 1] - toff[c]);
+      const int len = min(tile_len(1, sg), seg_start[sg + 1] - toff[c]);
       const int r = p.tab.slot_rank[seg_slot[sg]];
       if (is_dense(sg)) {
         sum_m += ((toff[c] - seg_start[sg]) % 128) == 0;
@@ -300,7 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       const int slot = seg_slot[sg];
       TileDesc dsc;
       dsc.off = toff[c];
-      dsc.len = min(mint_tile_tokens(1), seg_start[sg + 1] - toff[c]);
+      dsc.len = min(tile_len(1, sg), seg_start[sg + 1] - toff[c]);
       dsc.slot = slot;
       dsc.expert = seg_expert[sg];
       dsc.rank = p.tab.slot_rank[slot];
@@ -421,7 +433,8 @@ PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
 }
 
 int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space) {
-  const int64_t G = mint_tile_tokens(g);
+  // (list 1 may cut rank-1 segments into runs of mint_tile_tokens_rank1)
+  const int64_t G = mint_tile_tokens(g) < mint_tile_tokens_rank1(g) ? mint_tile_tokens(g) : mint_tile_tokens_rank1(g);
   const int64_t max_segments = key_space < P ? key_space : P;
   int64_t ub = P / G + max_segments;
   return ub < P ? ub : P;
