@@ -47,6 +47,7 @@ struct DenseProblem {
   const uint16_t *x;
   int64_t ldx;
   int32_t d, r_max;
+  int32_t splits;      // CTAs per tile, each over an equal share of the 64-column chunks of d
   float *ws_part;      // slots of 32 * r_max floats, [len][rank] packed fp32
 };
 
@@ -54,7 +55,8 @@ struct DenseParams {
   DenseProblem prob[kMaxProblems];
   int32_t T;
   int32_t lanes;
-  int32_t dense_slot0;   // the v of dense tile t goes to workspace slot dense_slot0 + t
+  int32_t dense_slot0;   // part s of the v of dense tile t goes to workspace slot dense_slot0 + s * dense_stride + t
+  int32_t dense_stride;
   int32_t *status;
   TableDev tab;
   PlanView pv;
@@ -166,7 +168,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   __shared__ int32_t rows[kTileRows];
   __shared__ int32_t failed;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const DenseProblem &pb = P.prob[blockIdx.y];
+  const DenseProblem &pb = P.prob[blockIdx.y / MINT_DENSE_SPLIT_MAX];
+  const int split = blockIdx.y % MINT_DENSE_SPLIT_MAX;
 
   pdl_launch_dependents();
   // The plan and the pool weights were complete before this call's kernels
@@ -174,7 +177,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
                   P.pv.header[PH_LANES] == P.lanes;
   const int m = blockIdx.x;
-  if (!ok || m >= P.pv.header[PH_NUM_DENSE]) {
+  if (!ok || m >= P.pv.header[PH_NUM_DENSE] || split >= pb.splits) {
     pdl_wait();
     return;
   }
@@ -210,7 +213,10 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   const uint32_t stage0 = (smem_addr(dyn_raw) + 1023u) & ~1023u;   // swizzle atoms are 1024-byte aligned
   const uint16_t *A_rows = pb.A + (int64_t)d0.slot * pb.r_max * pb.d;
   const uint32_t idesc = instr_desc(n_mma);
-  const int nchunks = (pb.d + kChunk - 1) / kChunk;
+  // this CTA's share of the chunks of d: [chunk0, chunk0 + nchunks)
+  const int all_chunks = (pb.d + kChunk - 1) / kChunk;
+  const int chunk0 = (int)((int64_t)all_chunks * split / pb.splits);
+  const int nchunks = (int)((int64_t)all_chunks * (split + 1) / pb.splits) - chunk0;
 
   pdl_wait();
 
@@ -219,7 +225,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
     if (kc < nchunks) {
       const uint32_t xs = stage0 + (uint32_t)((kc % kStages) * kStageBytes), as = xs + kXStageBytes;
       const int c = tid & 7;
-      const int col = kc * kChunk + c * 8;
+      const int col = (chunk0 + kc) * kChunk + c * 8;
       const bool col_ok = col < pb.d;
 #pragma unroll
       for (int i = 0; i < kTileRows / 16; ++i) {
@@ -268,7 +274,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
     // warp w owns accumulator rows 32 w .. 32 w + 31 (tensor-memory lanes), one row per thread
     const int row = warp * 32 + lane;
     const size_t slot_floats = (size_t)32 * pb.r_max;
-    float *dst = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
+    float *dst = pb.ws_part + (size_t)(P.dense_slot0 + split * P.dense_stride + t0 + (row >> 5)) * slot_floats +
+                 (size_t)(row & 31) * r;
     for (int j0 = 0; j0 < n_mma; j0 += 16) {
       float v[16];
       tmem_ld16(tmem_d + ((uint32_t)(warp * 32) << 16) + (uint32_t)j0, v);
@@ -324,6 +331,7 @@ struct DenseExpandProblem {
   uint16_t *y;
   int64_t ldy;
   int32_t n, r_max;
+  int32_t splits;      // parts of v per tile (the shrink's split of d)
   const float *ws_part;
 };
 struct DenseExpandParams {
@@ -331,6 +339,7 @@ struct DenseExpandParams {
   int32_t T;
   int32_t lanes;
   int32_t dense_slot0;
+  int32_t dense_stride;
   int32_t *status;
   TableDev tab;
   PlanView pv;
@@ -444,13 +453,24 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
     for (int q0 = tid; q0 < kTileRows * pairs; q0 += 8 * kThreads) {
       float a[8], b[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int q = q0 + u * kThreads;
-        const int row = q / pairs, k = 2 * (q - row * pairs);
-        const bool in = q < kTileRows * pairs && row < nrows;
-        const float *src = pb.ws_part + (size_t)(P.dense_slot0 + t0 + (row >> 5)) * slot_floats + (size_t)(row & 31) * r;
-        a[u] = (in && k < r) ? __ldcg(src + k) : 0.f;
-        b[u] = (in && k + 1 < r) ? __ldcg(src + k + 1) : 0.f;
+      for (int u = 0; u < 8; ++u) a[u] = b[u] = 0.f;
+      for (int sp = 0; sp < pb.splits; ++sp) {   // the parts of the shrink's CTAs, in their order; 16 loads go out together
+        float pa[8], pbv[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int q = q0 + u * kThreads;
+          const int row = q / pairs, k = 2 * (q - row * pairs);
+          const bool in = q < kTileRows * pairs && row < nrows;
+          const float *src = pb.ws_part + (size_t)(P.dense_slot0 + sp * P.dense_stride + t0 + (row >> 5)) * slot_floats +
+                             (size_t)(row & 31) * r;
+          pa[u] = (in && k < r) ? __ldcg(src + k) : 0.f;
+          pbv[u] = (in && k + 1 < r) ? __ldcg(src + k + 1) : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          a[u] += pa[u];
+          b[u] += pbv[u];
+        }
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
@@ -544,7 +564,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
 }  // namespace
 
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s) {
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
+                                 cudaStream_t s) {
   static bool attr_set = false;
   if (!attr_set) {
     int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -563,11 +584,13 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
     pb.ldx = args[i].ldx;
     pb.d = args[i].d;
     pb.r_max = args[i].r_max;
+    pb.splits = mint_dense_splits(args[i].d);
     pb.ws_part = static_cast<float *>(workspaces[i]);
   }
   P.T = T;
   P.lanes = lanes;
   P.dense_slot0 = dense_slot0;
+  P.dense_stride = dense_stride;
   P.status = args[0].status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
@@ -575,7 +598,7 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)tiles, (unsigned)nprob);
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)(nprob * MINT_DENSE_SPLIT_MAX));
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kDynSmem;
   cfg.stream = s;
@@ -586,7 +609,8 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
 
 
 int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s) {
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
+                                 cudaStream_t s) {
   static bool attr_set = false;
   if (!attr_set) {
     int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -606,12 +630,14 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
     pb.ldy = args[i].ldy;
     pb.n = args[i].n;
     pb.r_max = args[i].r_max;
+    pb.splits = mint_dense_splits(args[i].d);
     pb.ws_part = static_cast<const float *>(workspaces[i]);
     n_max = pb.n > n_max ? pb.n : n_max;
   }
   P.T = T;
   P.lanes = lanes;
   P.dense_slot0 = dense_slot0;
+  P.dense_stride = dense_stride;
   P.status = args[0].status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);

@@ -95,8 +95,8 @@ struct StreamProblem {
   int64_t ldx, ldy;
   int32_t d, n, r_max;
   int32_t cb0_shrink, cb0_expand;  // first virtual column block of this problem
-  float *ws_part;      // [2 tiles_ub + lanes][32 * r_max]  slot (tile + lane): that lane's sum, [len][rank] packed;
-                       // slot (tiles_ub + lanes + tile): the v of a dense segment's tile
+  float *ws_part;      // slots of 32 * r_max floats: slot (tile + lane): that lane's sum, [len][rank] packed;
+                       // slot (dense_slot0 + s * tiles_ub + tile): part s of the v of a dense segment's tile
 };
 
 struct StreamParams {
@@ -1174,8 +1174,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
 }
 
 // ---- host side -----------------------------------------------------------------
-size_t workspace_bytes(int64_t tiles, int32_t r_max) {
-  return (size_t)(2 * tiles + MINT_MAX_LANES) * kTileRowsMax * r_max * sizeof(float) + 256;
+// Slots of 32 x r_max floats: tile + lane for the streamed parts; with dense segments (batches of at
+// least MINT_DENSE_MIN_BATCH tokens) MINT_DENSE_SPLIT_MAX more per tile for the parts of the tensor-core shrink.
+size_t workspace_bytes(int64_t tiles, int32_t r_max, bool dense) {
+  const int64_t slots = tiles + MINT_MAX_LANES + (dense ? (int64_t)MINT_DENSE_SPLIT_MAX * tiles : 0);
+  return (size_t)slots * kTileRowsMax * r_max * sizeof(float) + 256;
 }
 
 }  // namespace
@@ -1188,7 +1191,7 @@ bool mint_stream_moe_supported(int32_t r_max, int32_t r_max_bound) {
 }
 
 size_t mint_stream_moe_workspace_bytes(int64_t pairs, int64_t key_space, int32_t r_max) {
-  return workspace_bytes(mint_tile_upper_bound(1, pairs, key_space), r_max);
+  return workspace_bytes(mint_tile_upper_bound(1, pairs, key_space), r_max, false);
 }
 
 static int32_t stream_kernel_attributes() {
@@ -1262,7 +1265,7 @@ int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void
 }
 
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max) {
-  return workspace_bytes(mint_tile_upper_bound(1, T, num_slots), r_max);
+  return workspace_bytes(mint_tile_upper_bound(1, T, num_slots), r_max, T >= MINT_DENSE_MIN_BATCH);
 }
 
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
@@ -1321,12 +1324,12 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   if (st) return st;
   const bool dense = T >= MINT_DENSE_MIN_BATCH;   // the plan may have given dense segments to the tensor-core kernels
   if (dense) {
-    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);
+    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
     if (st) return st;
   }
   st = mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
   if (st || !dense) return st;
-  return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, s);
+  return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
 }
 
 // ---- fused apply without a caller-provided workspace -------------------------------

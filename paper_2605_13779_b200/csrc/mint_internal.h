@@ -94,6 +94,15 @@ struct __align__(16) TileDesc {
 // 128-row tiles (every fourth 32-item tile of such a segment) in dense_tile.
 #define MINT_DENSE_MIN_BATCH 4096
 #define MINT_DENSE_MIN_SEGMENT 128
+// The tensor-core shrink splits a wide d over up to MINT_DENSE_SPLIT_MAX CTAs per
+// tile (one per MINT_DENSE_SPLIT_COLUMNS columns); part s of the v of dense tile t is
+// workspace slot  dense_slot0 + s * tiles_ub + t,  and the tensor-core expand adds the parts.
+#define MINT_DENSE_SPLIT_MAX 4
+#define MINT_DENSE_SPLIT_COLUMNS 5120
+__host__ __device__ constexpr int mint_dense_splits(int d) {
+  return d / MINT_DENSE_SPLIT_COLUMNS < 1 ? 1
+         : (d / MINT_DENSE_SPLIT_COLUMNS > MINT_DENSE_SPLIT_MAX ? MINT_DENSE_SPLIT_MAX : d / MINT_DENSE_SPLIT_COLUMNS);
+}
 
 // Start of cost lane j in the rows x column-blocks area: the tile that holds it
 // and j * rows_total = q * G + r, so that the position for CB column blocks is
@@ -212,10 +221,12 @@ bool mint_stream_supported(int32_t max_bound_rank);
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);
 // Tensor-core shrink of the dense segments' 128-row tiles (between the two streamed kernels).
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s);
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
+                                 cudaStream_t s);
 // Tensor-core expand of the same tiles (after the streamed expand, which skips them).
 int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, cudaStream_t s);
+                                 void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
+                                 cudaStream_t s);
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);
 
