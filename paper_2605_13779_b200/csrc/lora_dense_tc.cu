@@ -186,10 +186,16 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   const TileDesc d0 = P.pv.tile_desc[t0];
   // the 128-row tile = up to four consecutive 32-token tiles of the segment
   int nrows = d0.len;
-  for (int i = 1; i < 4 && nrows == 32 * i && t0 + i < ntiles; ++i) {
-    const TileDesc di = P.pv.tile_desc[t0 + i];
-    if (!di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
-    nrows += di.len;
+  {
+    TileDesc dn[3];   // the three descriptors that may follow, requested together
+#pragma unroll
+    for (int i = 1; i < 4; ++i) dn[i - 1] = P.pv.tile_desc[min(t0 + i, ntiles - 1)];
+#pragma unroll
+    for (int i = 1; i < 4; ++i) {
+      const TileDesc &di = dn[i - 1];
+      if (nrows != 32 * i || t0 + i >= ntiles || !di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
+      nrows += di.len;
+    }
   }
   const int r = d0.rank;
   if (r > pb.r_max || r > kMaxRank || r < 1) {
@@ -390,10 +396,16 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
   const int t0 = P.pv.dense_tile[m];
   const TileDesc d0 = P.pv.tile_desc[t0];
   int nrows = d0.len;
-  for (int i = 1; i < 4 && nrows == 32 * i && t0 + i < ntiles; ++i) {
-    const TileDesc di = P.pv.tile_desc[t0 + i];
-    if (!di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
-    nrows += di.len;
+  {
+    TileDesc dn[3];   // the three descriptors that may follow, requested together
+#pragma unroll
+    for (int i = 1; i < 4; ++i) dn[i - 1] = P.pv.tile_desc[min(t0 + i, ntiles - 1)];
+#pragma unroll
+    for (int i = 1; i < 4; ++i) {
+      const TileDesc &di = dn[i - 1];
+      if (nrows != 32 * i || t0 + i >= ntiles || !di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
+      nrows += di.len;
+    }
   }
   const int r = d0.rank;
   if (r > pb.r_max || r > kMaxRank || r < 1) {   // reported by the shrink
