@@ -865,14 +865,23 @@ __device__ __forceinline__ void expand_mma(const StreamProblem &pb, const Piece 
           bq[i] = (2 * ks + (i >> 1) < KG) ? lds128(L.ring.slot(it, 2 * (2 * ks + (i >> 1)) + (i & 1))) : zero4();
         const uint4 vh = S.vfrag[((mt * 4 + ks) * 2 + 0) * 32 + lane];
         const uint4 vl = S.vfrag[((mt * 4 + ks) * 2 + 1) * 32 + lane];
+        // four tiles at a time: the four head MMAs, then the four remainder MMAs, so that the two
+        // MMAs into one accumulator are not back to back
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const uint32_t b0 = (j & 1) ? pair_hi(word(bq[0], j >> 1), word(bq[1], j >> 1))
-                                      : pair_lo(word(bq[0], j >> 1), word(bq[1], j >> 1));
-          const uint32_t b1 = (j & 1) ? pair_hi(word(bq[2], j >> 1), word(bq[3], j >> 1))
-                                      : pair_lo(word(bq[2], j >> 1), word(bq[3], j >> 1));
-          mma_bf16(acc[j], vh.x, vh.y, vh.z, vh.w, b0, b1);
-          mma_bf16(acc[j], vl.x, vl.y, vl.z, vl.w, b0, b1);
+        for (int j0 = 0; j0 < 8; j0 += 4) {
+          uint32_t b0[4], b1[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int j = j0 + i;
+            b0[i] = (j & 1) ? pair_hi(word(bq[0], j >> 1), word(bq[1], j >> 1))
+                            : pair_lo(word(bq[0], j >> 1), word(bq[1], j >> 1));
+            b1[i] = (j & 1) ? pair_hi(word(bq[2], j >> 1), word(bq[3], j >> 1))
+                            : pair_lo(word(bq[2], j >> 1), word(bq[3], j >> 1));
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_bf16(acc[j0 + i], vh.x, vh.y, vh.z, vh.w, b0[i], b1[i]);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) mma_bf16(acc[j0 + i], vl.x, vl.y, vl.z, vl.w, b0[i], b1[i]);
         }
       }
       // acc[j][0], [1]: row g, columns 8 t + j and 32 + 8 t + j; acc[j][2], [3]: row g + 8
