@@ -934,23 +934,42 @@ struct ExpandVecLane {
   }
 };
 
+// An FMA-path piece needs no barrier of the CTA: every thread adds the shrink lanes' parts of the few v it
+// needs by itself (the same few addresses for all threads) while the first blocks are on their way, so the
+// warps of a CTA run through such pieces independently of one another.
 template <int L>
-__device__ __forceinline__ void expand_vec_fill(const StreamProblem &pb, const Piece &pc, uint32_t ring_base) {
-  ExpandVecLane<L> V;
-  V.init(pb, pc, ring_base);
-#pragma unroll 1
-  for (int it = 0; it < Ring<1 + L>::kDepth - 1; ++it) V.issue(it);
-}
-
-template <int L>
-__device__ __forceinline__ void expand_vec(const StreamProblem &pb, const Piece &pc, uint32_t ring_base,
-                                           const SmemExpand &S) {
+__device__ __forceinline__ void expand_vec(const StreamParams &P, const StreamProblem &pb, const Piece &pc,
+                                           uint32_t ring_base, int first, int count) {
   constexpr int kDepth = Ring<1 + L>::kDepth;
   ExpandVecLane<L> V;
   V.init(pb, pc, ring_base);
+#pragma unroll 1
+  for (int it = 0; it < kDepth - 1; ++it) V.issue(it);
   float sv[L];
+  {
+    const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
+    const float *part0 = pb.ws_part + (size_t)(pc.t + first) * slot_floats;
 #pragma unroll
-  for (int l = 0; l < L; ++l) sv[l] = l < pc.len ? pc.scale * S.vsum[l] : 0.f;
+    for (int l = 0; l < L; ++l) sv[l] = 0.f;
+    for (int k0 = 0; k0 < count; k0 += 4) {   // in lane order; the loads of four parts go out together
+      float v[4][L];
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int l = 0; l < L; ++l)
+          v[k][l] = (k0 + k < count && l < pc.len) ? __ldcg(part0 + (size_t)(k0 + k) * slot_floats + l) : 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int l = 0; l < L; ++l) sv[l] += v[k][l];
+    }
+#pragma unroll
+    for (int l = 0; l < L; ++l) {
+      // MoE: the pair's routing weight multiplies its v
+      const float w = (P.pair_weight && l < pc.len) ? __ldg(P.pair_weight + pc.rows[l]) : 1.f;
+      sv[l] = pc.scale * (w * sv[l]);
+    }
+  }
 #pragma unroll 1
   for (int it = 0; it < V.iters; ++it) {
     V.issue(it + kDepth - 1);
@@ -1060,13 +1079,15 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   const int yg = pc.len <= 8 ? 1 : (pc.len <= 16 ? 2 : 4);
   const int kg = pc.r <= 8 ? 1 : (pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8));
   const int MT = (yg + 1) >> 1, KS = (kg + 1) >> 1;
-  // step 1
   if (vec) {
-    if (pc.len == 1) expand_vec_fill<1>(pb, pc, ring_base);
-    else if (pc.len == 2) expand_vec_fill<2>(pb, pc, ring_base);
-    else if (pc.len <= 4) expand_vec_fill<4>(pb, pc, ring_base);
-    else expand_vec_fill<8>(pb, pc, ring_base);
-  } else {
+    if (pc.len == 1) expand_vec<1>(P, pb, pc, ring_base, first, count);
+    else if (pc.len == 2) expand_vec<2>(P, pb, pc, ring_base, first, count);
+    else if (pc.len <= 4) expand_vec<4>(P, pb, pc, ring_base, first, count);
+    else expand_vec<8>(P, pb, pc, ring_base, first, count);
+    return;
+  }
+  // step 1
+  {
 #define MINT_EXPAND_CASE(YG)                                     \
   if (kg == 1) expand_mma_fill<YG, 1>(pb, pc, ring_base);        \
   else if (kg == 2) expand_mma_fill<YG, 2>(pb, pc, ring_base);   \
@@ -1081,7 +1102,7 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   __syncthreads();   // the previous piece no longer reads v
   sum_parts(P, pb, pc, first, count, S.vsum);
   __syncthreads();
-  if (!vec) {
+  {
     // one thread per (m-tile, k-step, lane): four (head, remainder) register pairs
     for (int i = tid; i < MT * KS * 32; i += kThreads) {
       const int ln = i & 31, ks = (i >> 5) % KS, mt = (i >> 5) / KS;
@@ -1100,12 +1121,7 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
     __syncthreads();
   }
   // step 3
-  if (vec) {
-    if (pc.len == 1) expand_vec<1>(pb, pc, ring_base, S);
-    else if (pc.len == 2) expand_vec<2>(pb, pc, ring_base, S);
-    else if (pc.len <= 4) expand_vec<4>(pb, pc, ring_base, S);
-    else expand_vec<8>(pb, pc, ring_base, S);
-  } else {
+  {
 #define MINT_EXPAND_CASE(YG)                                        \
   if (kg == 1) expand_mma<YG, 1>(pb, pc, ring_base, S);             \
   else if (kg == 2) expand_mma<YG, 2>(pb, pc, ring_base, S);        \
