@@ -1075,9 +1075,10 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   const bool vec = pc.r == 1 && pc.len <= 8;
   const int first = S.sh.part_first[pc.ti * kMaxProblems + pc.p];
   const int count = S.sh.part_count[pc.ti * kMaxProblems + pc.p];
-  // row groups as the tensor-core body is instantiated: 1, 2 or 4 groups of 8 tokens; 1, 2, 4 or 8 of 8 ranks
+  // row groups as the tensor-core body is instantiated: 1, 2 or 4 groups of 8 tokens; 2, 4 or 8 of 8 ranks
+  // (a single group of ranks would run the same MMAs as two; fewer bodies keep the kernel's code small)
   const int yg = pc.len <= 8 ? 1 : (pc.len <= 16 ? 2 : 4);
-  const int kg = pc.r <= 8 ? 1 : (pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8));
+  const int kg = pc.r <= 16 ? 2 : (pc.r <= 32 ? 4 : 8);
   const int MT = (yg + 1) >> 1, KS = (kg + 1) >> 1;
   if (vec) {
     if (pc.len == 1) expand_vec<1>(P, pb, pc, ring_base, first, count);
@@ -1089,8 +1090,7 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   // step 1
   {
 #define MINT_EXPAND_CASE(YG)                                     \
-  if (kg == 1) expand_mma_fill<YG, 1>(pb, pc, ring_base);        \
-  else if (kg == 2) expand_mma_fill<YG, 2>(pb, pc, ring_base);   \
+  if (kg == 2) expand_mma_fill<YG, 2>(pb, pc, ring_base);        \
   else if (kg == 4) expand_mma_fill<YG, 4>(pb, pc, ring_base);   \
   else expand_mma_fill<YG, 8>(pb, pc, ring_base)
     if (yg == 1) { MINT_EXPAND_CASE(1); }
@@ -1123,8 +1123,7 @@ __device__ __forceinline__ void expand_piece(const StreamParams &P, SmemExpand &
   // step 3
   {
 #define MINT_EXPAND_CASE(YG)                                        \
-  if (kg == 1) expand_mma<YG, 1>(pb, pc, ring_base, S);             \
-  else if (kg == 2) expand_mma<YG, 2>(pb, pc, ring_base, S);        \
+  if (kg == 2) expand_mma<YG, 2>(pb, pc, ring_base, S);             \
   else if (kg == 4) expand_mma<YG, 4>(pb, pc, ring_base, S);        \
   else expand_mma<YG, 8>(pb, pc, ring_base, S)
     if (yg == 1) { MINT_EXPAND_CASE(1); }
