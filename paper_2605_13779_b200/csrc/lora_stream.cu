@@ -668,8 +668,8 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   else if (rg == 2) shrink_mma_packed<XG, 2>(pb, pc, rh, ring_base, S.scratch);       \
   else if (rg == 4) shrink_mma_packed<XG, 4>(pb, pc, rh, ring_base, S.scratch);       \
   else shrink_mma_packed<XG, 8>(pb, pc, rh, ring_base, S.scratch)
-      if (pc.len <= 8) { MINT_SHRINK_CASE(1); }
-      else if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
+      // (one group of 8 token rows would run the same MMAs as two; fewer bodies keep the kernel's code small)
+      if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
       else { MINT_SHRINK_CASE(4); }
 #undef MINT_SHRINK_CASE
     } else if (vec) {
@@ -683,8 +683,8 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   if (ng == 1) shrink_mma<XG, 1>(pb, pc, rh, ring_base, S.scratch);                 \
   else if (ng == 2) shrink_mma<XG, 2>(pb, pc, rh, ring_base, S.scratch);            \
   else shrink_mma<XG, 4>(pb, pc, rh, ring_base, S.scratch)
-      if (pc.len <= 8) { MINT_SHRINK_CASE(1); }
-      else if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
+      // (one group of 8 token rows would run the same MMAs as two; fewer bodies keep the kernel's code small)
+      if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
       else { MINT_SHRINK_CASE(4); }
 #undef MINT_SHRINK_CASE
     }
