@@ -728,8 +728,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) shrink_stream_kernel(con
     load_batch<kPacked>(P, S.sh, tb, ntile);
     if (!waited) {
       // while the previous kernel still runs: pull this lane's A rows into L2
-      walk_batch<false>(P, area, R, S.sh, tb, ntile,
-                        [&](const Piece &pc) { prefetch_piece<false, kPacked>(P.prob[pc.p], pc, true, false); });
+      bool first_piece = true;   // only the piece the lane starts with: the rest follow behind its stream
+      walk_batch<false>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) {
+        if (first_piece) prefetch_piece<false, kPacked>(P.prob[pc.p], pc, true, false);
+        first_piece = false;
+      });
       pdl_wait();   // activations and the workspace belong to earlier kernels until here
       waited = true;
     }
@@ -1187,8 +1190,11 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) expand_stream_kernel(con
     }
     if (!waited) {
       // while the shrink kernel still runs: pull this lane's B rows into L2
-      walk_batch<true>(P, area, R, S.sh, tb, ntile,
-                       [&](const Piece &pc) { prefetch_piece<true>(P.prob[pc.p], pc, true, false); });
+      bool first_piece = true;   // only the piece the lane starts with
+      walk_batch<true>(P, area, R, S.sh, tb, ntile, [&](const Piece &pc) {
+        if (first_piece) prefetch_piece<true>(P.prob[pc.p], pc, true, false);
+        first_piece = false;
+      });
       pdl_wait();   // the shrink kernel has completed: v is final, y belongs to this kernel
       waited = true;
     }
