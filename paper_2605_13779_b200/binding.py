@@ -324,10 +324,10 @@ def mint_lora_apply_workspace_bytes(pool: Pool, T: int) -> int:
 
 
 def new_workspace(pool: Pool, T: int, device="cuda") -> torch.Tensor:
-    """Zero-filled workspace of the fused apply for one projection (the library
-    keeps it zero where it must be between calls)."""
+    """Workspace of the fused apply for one projection; it needs no initialisation
+    (every call writes each entry before it reads it)."""
     nbytes = max(256, mint_lora_apply_workspace_bytes(pool, T))
-    return torch.zeros(nbytes, dtype=torch.uint8, device=device)
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
 
 
 def _ld(t: torch.Tensor, width: int) -> int:
