@@ -1009,10 +1009,19 @@ __device__ __forceinline__ void shrink_parts(const StreamParams &P, const Area &
   const int w_t = tile_rows<false>(d.rank, d.len);
   const int blocks = (pb.d + kShrinkBlock - 1) / kShrinkBlock;
   const int span = w_t * sa.CB;   // the tile's extent in area units
-  // active lanes c with table index in [lane_lo, lane_hi]: index(c) = c G / active
-  const int c_a = (int)(((unsigned)(d.lane_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
-  const int c_b = (int)(((unsigned)(d.lane_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
-  unsigned long long mask = 0;   // bit i: lane c_a + i holds a part
+  // Table lanes that can meet the columns of THIS problem inside the tile: the problem covers the
+  // area positions [pos_lo, pos_hi) and table lane j starts at about j W CB / G (one lane of margin
+  // on either side; the exact test below decides).  A tile of a call with many projections can
+  // meet far more lanes than one problem of it does, so the tile's own bounds are not enough.
+  const int64_t wcb = sa.W * sa.CB;
+  const int64_t pos_lo = (int64_t)d.rows_shrink * sa.CB + (int64_t)pb.cb0_shrink * w_t;
+  const int64_t pos_hi = pos_lo + (int64_t)blocks * w_t;
+  const int j_lo = max(d.lane_lo, (int)(pos_lo * sa.G / wcb) - 1);
+  const int j_hi = min(d.lane_hi, (int)((pos_hi * sa.G + wcb - 1) / wcb) + 1);
+  // active lanes c with table index in [j_lo, j_hi]: index(c) = c G / active
+  const int c_a = (int)(((unsigned)(j_lo + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
+  const int c_b = (int)(((unsigned)(j_hi + 1) * (unsigned)sa.active - 1u) / (unsigned)sa.G);
+  unsigned long long mask = 0;   // bit i: lane c_a + i holds a part (at most kMaxParts + margin candidates)
   if (valid && !d.dense) {
     for (int i = k; c_a + i <= c_b && i < 64; i += 8) {
       const int c2 = c_a + i;

@@ -222,10 +222,11 @@ def test_dense_segments_take_the_tensor_core_kernels():
 
 
 def test_dense_segments_grouped_projections_of_different_widths():
-    """Two projections in one grouped call over a batch with dense segments: the
-    tensor-core expand splits a wide n into several column ranges per 128-row tile
-    (with a ragged last chunk), and the narrow projection leaves part of the grid
-    without work."""
+    """Two projections of different widths in one grouped call over a batch with
+    dense segments: both take one range of columns per 128-row tile in the
+    tensor-core expand, the wide one with a ragged last 128-column chunk (n = 2184),
+    and the narrow one leaves part of the grid without work.  (Several column
+    ranges per tile: test_dense_segments_wide_output_takes_several_column_ranges.)"""
     from paper_2605_13779_b200 import binding as mb, harness
     lengths = [900, 128, 257, 60, 1100, 131, 2, 640, 512, 400]
     adapters = [0, 1, 2, 3, 4, 5, 3, 0, 6, -1]
@@ -262,3 +263,71 @@ def test_dense_segments_config3_shape_sampled():
     rows = np.unique(np.concatenate([rows, edges[:8] - 1, edges[:8] % case.T]))
     y_ref, _, _ = parity.oracle_dense(case, rows=rows)
     parity.assert_close(y[rows], y_ref, "config3 sampled rows")
+
+
+def run_fused_rows(case, rows, y0_zero=False):
+    """The fused apply at full size; only the given rows of y come back to the host."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    dev = harness.upload_dense(case)
+    if y0_zero:
+        dev.y.zero_()
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    mb.mint_lora_apply_fused(dev.pool, dev.table, plan, dev.x, dev.y, dev.status)
+    torch.cuda.synchronize()
+    idx = torch.from_numpy(np.asarray(rows, dtype=np.int64)).cuda()
+    return harness.y_to_f64(dev.y[idx]), dev.status.cpu().numpy()
+
+
+SPLIT_LENGTHS = [700, 130, 128, 127, 300, 5, 1, 1000, 64, 513, 256, 129, 3, 640, 384, 40]
+SPLIT_ADAPTERS = [0, 1, 2, 3, 4, 5, 6, 7, 8, 0, 9, 10, -1, 11, 12, 6]
+SPLIT_RANKS = [64, 16, 8, 33, 1, 4, 32, 64, 16, 48, 5, 64, 17]
+
+
+@pytest.mark.parametrize("d,parts", [(10240, 2), (15360, 3), (25600, 4), (20488, 4)])
+def test_dense_segments_wide_input_is_split_over_several_ctas(d, parts):
+    """Input widths of 10240 and more: the tensor-core shrink of a 128-row tile is
+    split over 2, 3 or 4 CTAs, each over its share of the columns of d, and the
+    expand adds their parts.  Full and ragged 128-row tiles, ranks that are not
+    multiples of 16, a last 64-column chunk that is not full (d = 20488)."""
+    case = dense_segment_case(f"gpu/dense-tc/split/{d}", SPLIT_LENGTHS, SPLIT_ADAPTERS, SPLIT_RANKS,
+                              d=d, n=264, r_max=64)
+    assert case.T >= 4096
+    check_case(case, f"dense segments d={d} ({parts} parts)")
+
+
+@pytest.mark.parametrize("n", [25600, 24584])
+def test_dense_segments_wide_output_takes_several_column_ranges(n):
+    """n = 25600: seven ranges of 4096 columns per 128-row tile in the tensor-core
+    expand; n = 24584 ends with a range of 8 columns (a ragged last chunk)."""
+    case = dense_segment_case(f"gpu/dense-tc/wide-n/{n}", SPLIT_LENGTHS, SPLIT_ADAPTERS, SPLIT_RANKS,
+                              d=520, n=n, r_max=64)
+    y_ref, _, _ = parity.oracle_dense(case)
+    y, status, _ = run_fused(case)
+    assert status[0] == 0, status
+    parity.assert_close(y, y_ref, f"dense segments n={n}")
+    none = case.ids < 0
+    np.testing.assert_array_equal(y[none], synth.bf16_bits_to_f64(case.y0)[none])
+    zero = np.zeros_like(case.y0)
+    y_ref0, _, _ = parity.oracle_dense(case, y0=zero)
+    y0, _, _ = run_fused(case, y0_bits=zero)
+    parity.assert_close(y0, y_ref0, f"dense segments n={n}, y0=0")
+
+
+@pytest.mark.parametrize("d,n", [(5120, 25600), (25600, 5120)])
+def test_config3_wide_projections_full_size_sampled(d, n):
+    """The up (5120 -> 25600) and down (25600 -> 5120) projections of the 32B-dense
+    segmented prefill at full size (about 18k tokens), checked on sampled rows that
+    include the first and last token of requests (edges of 128-row tiles), with
+    the preset y and with y = 0."""
+    batch = synth.config3_batch()
+    case = synth.config3_projection(batch, d, n)
+    rng = synth.stream("gpu/dense-tc/sample", d, n)
+    rows = np.sort(rng.choice(case.T, size=64, replace=False))
+    edges = np.cumsum(batch.lengths)
+    rows = np.unique(np.concatenate([rows, edges[:8] - 1, edges[:8] % case.T, edges[:4] - 129, edges[:4] - 128]))
+    rows = rows[(rows >= 0) & (rows < case.T)]
+    for y0_zero in (False, True):
+        y, status = run_fused_rows(case, rows, y0_zero=y0_zero)
+        assert status[0] == 0, status
+        y_ref, _, _ = parity.oracle_dense(case, rows=rows, y0=np.zeros_like(case.y0) if y0_zero else None)
+        parity.assert_close(y, y_ref, f"config3 {d}->{n} sampled rows y0_zero={y0_zero}")

@@ -45,6 +45,16 @@ def test_config4_reduced_tokens(proj):
     check_case(synth.config4_projection(batch, proj), f"config4/{proj}/T512")
 
 
+@pytest.mark.parametrize("proj", ["gate", "down"])
+def test_config4_full_size(proj):
+    """The 30B-A3B setting as the benchmark runs it: T=4096 tokens, 32 768 pairs in
+    2048 (expert, adapter) groups of 16 pairs on average; unweighted, weighted and
+    with y = 0."""
+    batch = synth.config4_batch()
+    assert batch.T == 4096
+    check_case(synth.config4_projection(batch, proj), f"config4/{proj}/T4096")
+
+
 def test_config4_contiguous_requests_fewer_experts():
     """Fewer experts and contiguous requests give long (expert, adapter) groups."""
     batch = synth.config4_batch(T=768, E=8, K=2, num_slots=4, rank=16, contiguous_requests=True,
