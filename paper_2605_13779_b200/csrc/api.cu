@@ -5,6 +5,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 
 #include "mint_device.cuh"
@@ -38,12 +39,16 @@ int32_t mint_device_lanes(int32_t *lanes_out) {
     st = mint_check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
     if (st) return st;
     if (sms < 1) return mint_fail(MINT_ERR_CUDA, "device reports %d SMs", sms);
-    const int lanes = sms * 3;   // three streaming CTAs per SM
+    const int lanes = sms * 6;
     cached[dev] = lanes > MINT_MAX_LANES ? MINT_MAX_LANES : lanes;
   }
   *lanes_out = cached[dev];
   return MINT_OK;
 }
+
+static std::atomic<bool> g_tables_changed{false};
+void mint_mark_tables_changed() { g_tables_changed.store(true, std::memory_order_release); }
+bool mint_take_tables_changed() { return g_tables_changed.exchange(false, std::memory_order_acq_rel); }
 
 extern "C" const char *mint_last_error_string(void) { return g_err; }
 
@@ -116,6 +121,7 @@ int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_
 
 int32_t mint_launch_bind(int32_t *id_to_slot, int32_t *slot_rank, float *slot_scale,
                          const BindBatch &batch, cudaStream_t s) {
+  mint_mark_tables_changed();
   bind_kernel<<<1, 32, 0, s>>>(id_to_slot, slot_rank, slot_scale, batch);
   return mint_check_cuda(cudaGetLastError(), "slot table bind launch");
 }
@@ -389,6 +395,7 @@ extern "C" int32_t mint_lora_plan(const mint_slot_table *table, const int64_t *i
     return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "plan: plan_bytes=%zu < %zu", plan_bytes, need);
   int32_t lanes = 0;
   if ((st = mint_device_lanes(&lanes))) return st;
+  mint_mark_tables_changed();
   return mint_launch_plan(table_dev(table), ids_dev, T, expert_ids_dev, K, num_experts, lanes, plan_dev,
                           status_dev, static_cast<cudaStream_t>(stream));
 }
