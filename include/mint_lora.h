@@ -109,6 +109,22 @@ int32_t mint_pool_write_slot(mint_pool *pool, int32_t slot, int32_t expert, cons
                              const void *B_src, int32_t rank, int32_t src_is_device,
                              mint_stream_t stream);
 
+/* Admission of a whole adapter projection from the PACKED representation, with
+ * one kernel: the paper's packed MoE LoRA serving representation stacks the
+ * per-expert tensors of a projection along an expert axis so that a cold load
+ * touches few objects (packed MoE LoRA loader table: 37 248 tensors become 672;
+ * the load path was object-bound, not byte-bound).  Both sources are DEVICE
+ * pointers, 16-byte aligned, bf16:
+ *   PACKED_MOE pools: A_packed_dev[expert][d][rank], B_packed_dev[expert][rank][n]
+ *                     -> A[slot][expert][d][r_max],  B[slot][expert][r_max][n]
+ *   RANK_MAJOR pools: A_packed_dev[rank][d], B_packed_dev[rank][n]
+ *                     -> A[slot][r_max][d],    B[slot][r_max][n]
+ * Padding beyond the adapter's rank is left untouched.  The call only enqueues
+ * the copy; binding the id to the slot is mint_slot_table_bind's job (or the
+ * slot manager's, below), and must be enqueued on the same stream.           */
+int32_t mint_pool_admit_packed(mint_pool *pool, int32_t slot, const void *A_packed_dev,
+                               const void *B_packed_dev, int32_t rank, mint_stream_t stream);
+
 /* ---- slot table: catalog id -> slot, slot -> (rank, scale) ---------------
  * The engine-local adapter id of the paper's serving map: a catalog of up to
  * 10^6 addressable ids of which a bounded subset is resident.  The three device
@@ -129,6 +145,34 @@ int32_t mint_slot_table_bind_many(mint_slot_table *table, int64_t count, const i
 int32_t mint_slot_table_evict(mint_slot_table *table, int64_t catalog_id, mint_stream_t stream);
 int32_t mint_slot_table_destroy(mint_slot_table *table);
 int64_t mint_slot_table_generation(const mint_slot_table *table);
+
+/* ---- slot manager: which adapters hold the GPU slots ------------------------
+ * The GPU-batch tier holds a bounded number of distinct adapters, promoted by
+ * the batch scheduler and released at the end of a step (paper, cache-tier
+ * table of "Scale Out: Policy-Population Serving"; the service tracks pinned
+ * adapters, "Worker admission and eviction").  Host-side bookkeeping:
+ * acquire makes catalog_id resident and pins it for the running step:
+ *  - already resident: *slot_out is its slot, *admitted_out = 0;
+ *  - otherwise it takes the lowest-numbered empty slot, or the slot of the
+ *    least recently acquired adapter that no step pins (*evicted_id_out names
+ *    it, else -1), and *admitted_out = 1: the caller now admits the weights
+ *    into that slot of every pool (mint_pool_admit_packed) on the same stream;
+ *  - MINT_ERR_NOT_RESIDENT when every slot is pinned.
+ * With a table (created empty, same num_slots) acquire also evicts the victim
+ * from the table and binds catalog_id to the slot with (rank, scale), which
+ * bumps the table's generation; with table = NULL it only keeps the books
+ * (rank, scale and stream are then ignored).  release removes one pin.  lookup
+ * returns the slot of a resident id or -1.  (The paper names least-recently-used
+ * order for its CPU adapter cache; using it for unpinned GPU slots is this
+ * library's choice.)                                                          */
+typedef struct mint_slot_manager mint_slot_manager;
+int32_t mint_slot_manager_create(mint_slot_manager **out, int32_t num_slots, mint_slot_table *table);
+int32_t mint_slot_manager_destroy(mint_slot_manager *manager);
+int32_t mint_slot_manager_acquire(mint_slot_manager *manager, int64_t catalog_id, int32_t rank, float scale,
+                                  int32_t *slot_out, int32_t *admitted_out, int64_t *evicted_id_out,
+                                  mint_stream_t stream);
+int32_t mint_slot_manager_release(mint_slot_manager *manager, int64_t catalog_id);
+int32_t mint_slot_manager_lookup(const mint_slot_manager *manager, int64_t catalog_id);
 
 /* ---- plan: token -> adapter segmentation, once per batch ------------------
  * Groups the batch's work items by the adapter slot they use (paper: batch

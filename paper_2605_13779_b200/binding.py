@@ -35,7 +35,9 @@ MINT_LAYOUT_PACKED_MOE = 1
 # Every symbol include/mint_lora.h declares (the CPU test checks the export list).
 EXPORTS = [
     "mint_last_error_string", "mint_status_name",
-    "mint_pool_create", "mint_pool_destroy", "mint_pool_write_slot",
+    "mint_pool_create", "mint_pool_destroy", "mint_pool_write_slot", "mint_pool_admit_packed",
+    "mint_slot_manager_create", "mint_slot_manager_destroy", "mint_slot_manager_acquire",
+    "mint_slot_manager_release", "mint_slot_manager_lookup",
     "mint_slot_table_create", "mint_slot_table_bind", "mint_slot_table_bind_many",
     "mint_slot_table_evict", "mint_slot_table_destroy", "mint_slot_table_generation",
     "mint_lora_plan_bytes", "mint_lora_plan_layout", "mint_lora_plan", "mint_plan_fetch_summary",
@@ -101,6 +103,13 @@ def load_library() -> ctypes.CDLL:
         "mint_pool_create": (i32, [ctypes.POINTER(vp), ctypes.POINTER(PoolDesc)]),
         "mint_pool_destroy": (i32, [vp]),
         "mint_pool_write_slot": (i32, [vp, i32, i32, vp, vp, i32, i32, vp]),
+        "mint_pool_admit_packed": (i32, [vp, i32, vp, vp, i32, vp]),
+        "mint_slot_manager_create": (i32, [ctypes.POINTER(vp), i32, vp]),
+        "mint_slot_manager_destroy": (i32, [vp]),
+        "mint_slot_manager_acquire": (i32, [vp, i64, i32, f32, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                            ctypes.POINTER(i64), vp]),
+        "mint_slot_manager_release": (i32, [vp, i64]),
+        "mint_slot_manager_lookup": (i32, [vp, i64]),
         "mint_slot_table_create": (i32, [ctypes.POINTER(vp), i64, i32, vp, vp, vp, vp]),
         "mint_slot_table_bind": (i32, [vp, i64, i32, i32, f32, vp]),
         "mint_slot_table_bind_many": (i32, [vp, i64, vp, vp, vp, vp, vp]),
@@ -197,6 +206,13 @@ class Pool:
         _check(lib.mint_pool_write_slot(self.handle, slot, expert, A_src.data_ptr(), B_src.data_ptr(),
                                         rank, 1 if on_dev else 0, _stream()))
 
+    def admit_packed(self, slot: int, A_packed: torch.Tensor, B_packed: torch.Tensor, rank: int):
+        """The stacked tensors of one adapter projection (device, bf16, contiguous) into a slot:
+        [E][d][rank], [E][rank][n] for packed MoE pools; [rank][d], [rank][n] for dense pools."""
+        assert A_packed.is_cuda and B_packed.is_cuda and A_packed.is_contiguous() and B_packed.is_contiguous()
+        _check(load_library().mint_pool_admit_packed(self.handle, slot, _ptr(A_packed), _ptr(B_packed), rank,
+                                                     _stream()))
+
     def __del__(self):
         if getattr(self, "handle", None) and _lib is not None:
             _lib.mint_pool_destroy(self.handle)
@@ -241,6 +257,37 @@ class SlotTable:
     def __del__(self):
         if getattr(self, "handle", None) and _lib is not None:
             _lib.mint_slot_table_destroy(self.handle)
+            self.handle = None
+
+
+class SlotManager:
+    """Which adapters hold the GPU slots: least-recently-used order over the slots no running
+    step pins.  With a table, acquire also evicts and binds in the table."""
+
+    def __init__(self, num_slots: int, table: Optional[SlotTable] = None):
+        self.table = table
+        h = ctypes.c_void_p()
+        _check(load_library().mint_slot_manager_create(ctypes.byref(h), num_slots,
+                                                       table.handle if table is not None else None))
+        self.handle = h
+
+    def acquire(self, catalog_id: int, rank: int = 1, scale: float = 1.0):
+        """-> (slot, admitted, evicted id or None); pins the id once."""
+        slot, admitted, evicted = ctypes.c_int32(-1), ctypes.c_int32(0), ctypes.c_int64(-1)
+        stream = _stream() if self.table is not None else None
+        _check(load_library().mint_slot_manager_acquire(self.handle, catalog_id, rank, scale, ctypes.byref(slot),
+                                                        ctypes.byref(admitted), ctypes.byref(evicted), stream))
+        return slot.value, bool(admitted.value), (None if evicted.value < 0 else evicted.value)
+
+    def release(self, catalog_id: int):
+        _check(load_library().mint_slot_manager_release(self.handle, catalog_id))
+
+    def lookup(self, catalog_id: int) -> int:
+        return int(load_library().mint_slot_manager_lookup(self.handle, catalog_id))
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.mint_slot_manager_destroy(self.handle)
             self.handle = None
 
 

@@ -39,7 +39,7 @@ int32_t mint_device_lanes(int32_t *lanes_out) {
     st = mint_check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev), "SM count");
     if (st) return st;
     if (sms < 1) return mint_fail(MINT_ERR_CUDA, "device reports %d SMs", sms);
-    const int lanes = sms * 6;
+    const int lanes = sms * 3;   // three streaming CTAs per SM
     cached[dev] = lanes > MINT_MAX_LANES ? MINT_MAX_LANES : lanes;
   }
   *lanes_out = cached[dev];

@@ -155,12 +155,12 @@ struct PlanView {
   const LaneStart *lane_expand;
 };
 PlanView mint_plan_view(const void *plan_dev, int64_t P, int64_t key_space);
-// Number of cost lanes plans are cut for on the current device (six per SM: a multiple of the
-// lanes per SM of every kernel that walks the tables, so that each takes every k-th entry).
+// Number of cost lanes plans are cut for on the current device (three per SM).
 int32_t mint_device_lanes(int32_t *lanes_out);
 // A plan, bind or evict kernel was enqueued: the next apply must not start before it has
-// completed (it reads the plan and the slot table first thing), so its first kernel is launched
-// without programmatic stream serialization.  take returns the mark and clears it.
+// completed (an apply kernel reads the plan and the slot table before its dependency wait), so
+// its first kernel is launched without programmatic stream serialization.  take returns the
+// mark and clears it.
 void mint_mark_tables_changed();
 bool mint_take_tables_changed();
 
@@ -221,7 +221,7 @@ int32_t mint_launch_shrink(const DenseArgs &a, const TableDev &tab, const void *
 int32_t mint_launch_expand(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
 int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
 
-// Streamed fused path (bulk-copy stage rings + warp MMA) for ranks up to 64: one
+// Streamed fused path (per-warp cp.async rings + warp MMA) for ranks up to 64: one
 // shrink and one expand launch cover up to 8 projections that share a plan.
 bool mint_stream_supported(int32_t max_bound_rank);
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);

@@ -86,3 +86,45 @@ def test_null_arguments_are_rejected(lib):
     assert l.mint_lora_apply_fused(None, None, None, 4, None, 8, None, 8, None, 0, None, None) == binding.MINT_ERR_INVALID_ARG
     assert l.mint_moe_lora_apply(None, None, None, 4, 2, None, 8, 8, None, None, None, 8, None, 0, None, None) == binding.MINT_ERR_INVALID_ARG
     assert l.mint_slot_table_evict(None, 0, None) == binding.MINT_ERR_INVALID_ARG
+
+
+def test_slot_manager_without_a_table_follows_the_oracle_model(lib):
+    """The library's slot manager (bookkeeping only, no GPU) against the plain model and the
+    hand-worked sequence."""
+    import random
+    from oracle import admission
+    import test_oracle_admission as golden
+    binding, _ = lib
+    m = binding.SlotManager(3)
+    for op in golden.read_lru_golden():
+        if op[0] == "acquire":
+            assert m.acquire(op[1]) == (op[2], op[3], op[4]), op
+        elif op[0] == "release":
+            m.release(op[1])
+        else:
+            with pytest.raises(binding.MintError) as e:
+                m.acquire(op[1])
+            assert e.value.status == binding.MINT_ERR_NOT_RESIDENT
+    rnd = random.Random(5)
+    m, o, held = binding.SlotManager(7), admission.LruSlots(7), []
+    for step in range(5000):
+        if held and rnd.random() < 0.45:
+            c = held.pop(rnd.randrange(len(held)))
+            m.release(c)
+            o.release(c)
+            continue
+        c = rnd.randrange(1_000_000) if rnd.random() < 0.3 else rnd.randrange(20)
+        try:
+            want = o.acquire(c)
+        except LookupError:
+            want = None
+        try:
+            got = m.acquire(c)
+        except binding.MintError:
+            got = None
+        assert got == want, (step, c, got, want)
+        if got:
+            held.append(c)
+        assert m.lookup(c) == (got[0] if got else o.resident().get(c, -1))
+    with pytest.raises(binding.MintError):
+        m.release(123456789)
