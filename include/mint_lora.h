@@ -321,6 +321,23 @@ int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table,
                             int64_t ldy, void *workspace_dev, size_t workspace_bytes,
                             int32_t *status_dev, mint_stream_t stream);
 
+/* Router-weighted combine: the MoE expert LoRA update of the projection that ends
+ * an expert FFN, summed over a token's routed experts into the token's row
+ * (paper, "Scale Up": per-expert LoRA tensors keyed by expert id):
+ *   Y[t, :] += sum over k of  w[t,k] * s_sigma * (X[row(p), :] . A[sigma][e_k]) . B[sigma][e_k],  p = t*K + k.
+ * y_dev: bf16 [T][ldy].  pair_weight_dev is required.  The sum over k runs in k
+ * order in fp32 and ends in one round-to-nearest-even store; the weighted
+ * per-pair updates pass through workspace_dev as bf16 (T*K*n elements beside the
+ * MoE apply's own workspace).  Rows of tokens without a resident adapter keep
+ * their bits.  Other arguments as for mint_moe_lora_apply.                    */
+size_t mint_moe_lora_apply_combine_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K);
+int32_t mint_moe_lora_apply_combine(const mint_pool *pool, const mint_slot_table *table,
+                                    const void *plan_dev, int32_t T, int32_t K, const void *x_dev,
+                                    int64_t ldx, int64_t x_rows, const int32_t *x_row_dev,
+                                    const float *pair_weight_dev, void *y_dev, int64_t ldy,
+                                    void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                                    mint_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -176,3 +176,30 @@ def moe_lora_apply(ids, expert_ids, id_to_slot, slot_rank, slot_scale, A, B, x, 
         _p(x), ctypes.c_int64(d), _p(x_row), _p(pair_weight),
         _p(y0), ctypes.c_int64(n), _p(y_ref), ctypes.c_int32(num_threads))
     return y_ref, int(missing)
+
+
+def moe_lora_apply_combine(ids, expert_ids, id_to_slot, slot_rank, slot_scale, A, B, x, y0_tokens, pair_weight, *,
+                           x_row=None, num_threads: int = 0):
+    """Router-weighted combine of the MoE expert LoRA update into the token's row
+    (paper, "Scale Up": per-expert LoRA tensors keyed by expert id; the routed
+    experts' outputs of a token are combined with the router's weights):
+
+        Y[t, :] = Y0[t, :] + sum over k of  w[t, k] * s * (X[row(t, k), :] . A[sigma][e]) . B[sigma][e]
+
+    Written as the per-pair oracle on a zero start (each pair's weighted update
+    in fp64) followed by the plain sum over k, in k order.  y0_tokens is bf16
+    bits [T, n]; returns (Y_ref fp64 [T, n], tokens whose id was not resident)."""
+    ids = _c(ids, np.int64)
+    expert_ids = _c(expert_ids, np.int32)
+    T = ids.shape[0]
+    K = expert_ids.shape[1] if expert_ids.ndim == 2 else 1
+    n = np.asarray(B).shape[3]
+    y0_tokens = _c(y0_tokens, np.uint16)
+    assert y0_tokens.shape == (T, n)
+    zero = np.zeros((T * K, n), dtype=np.uint16)
+    per_pair, missing = moe_lora_apply(ids, expert_ids, id_to_slot, slot_rank, slot_scale, A, B, x, zero,
+                                       x_row=x_row, pair_weight=pair_weight, num_threads=num_threads)
+    y_ref = (y0_tokens.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    for k in range(K):
+        y_ref = y_ref + per_pair[k::K]
+    return y_ref, missing

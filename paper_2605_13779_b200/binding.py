@@ -45,6 +45,7 @@ EXPORTS = [
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
     "mint_lora_apply_fused_static",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
+    "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
 ]
 
 
@@ -128,6 +129,8 @@ def load_library() -> ctypes.CDLL:
         "mint_lora_apply_fused_static": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
+        "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
+        "mint_moe_lora_apply_combine": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -450,4 +453,23 @@ def mint_moe_lora_apply(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tenso
         _ptr(x_row), _ptr(pair_weight), _ptr(y), y.stride(0),
         _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
         _ptr(status), _stream()))
+    return y
+
+
+def mint_moe_lora_apply_combine(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,
+                                status: torch.Tensor, pair_weight: torch.Tensor,
+                                x_row: Optional[torch.Tensor] = None,
+                                workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """y: [T][n], updated in place with the router-weighted sum over each token's K experts."""
+    assert pair_weight.dtype == torch.float32 and pair_weight.is_contiguous()
+    if x_row is not None:
+        assert x_row.dtype == torch.int32 and x_row.is_contiguous()
+    lib = load_library()
+    if workspace is None:
+        nbytes = max(256, int(lib.mint_moe_lora_apply_combine_workspace_bytes(pool.handle, plan.T, plan.K)))
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=y.device)
+    _check(lib.mint_moe_lora_apply_combine(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, plan.K, _ptr(x), x.stride(0), x.shape[0],
+        _ptr(x_row), _ptr(pair_weight), _ptr(y), y.stride(0), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
     return y

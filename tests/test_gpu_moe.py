@@ -129,3 +129,62 @@ def test_bad_row_index_is_reported_and_skipped():
     y_ref, _ = parity.oracle_moe(case)
     keep = np.arange(16) != 5
     parity.assert_close(y[keep], y_ref[keep], "other pairs")
+
+
+def run_combine(case, y0_bits):
+    from paper_2605_13779_b200 import binding as mb, harness
+    dev = harness.upload_moe(case)
+    y = mb.bf16_from_bits(y0_bits)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status, expert_ids=dev.expert_ids, num_experts=case.E)
+    mb.mint_moe_lora_apply_combine(dev.pool, dev.table, plan, dev.x, y, dev.status, dev.pair_weight, x_row=dev.x_row)
+    torch.cuda.synchronize()
+    return harness.y_to_f64(y), dev.status.cpu().numpy()
+
+
+def check_combine(case, what):
+    from oracle import oracle
+    t = case.table
+    for zero in (False, True):
+        y0 = synth.normal_bf16(synth.stream(what, "y0 tokens"), (case.T, case.n), 1.0)
+        if zero:
+            y0 = np.zeros_like(y0)
+        y_ref, _ = oracle.moe_lora_apply_combine(case.ids, case.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                                 case.A, case.B, case.x, y0, case.pair_weight, x_row=case.x_row)
+        y, status = run_combine(case, y0)
+        assert status[0] == 0, status
+        parity.assert_close(y, y_ref, f"{what} combine zero={zero}")
+        none = case.ids < 0
+        if none.any():
+            np.testing.assert_array_equal(y[none], synth.bf16_bits_to_f64(y0)[none])
+
+
+def test_combine_config4_down_reduced_tokens():
+    batch = synth.config4_batch(T=512)
+    check_combine(synth.config4_projection(batch, "down"), "config4/down/T512")
+
+
+def test_combine_config4_down_full_size():
+    batch = synth.config4_batch()
+    check_combine(synth.config4_projection(batch, "down"), "config4/down/T4096")
+
+
+@pytest.mark.parametrize("T,K,E,d,n,num_slots,rank,p_none", [
+    (1, 1, 1, 8, 8, 1, 1, 0.0),
+    (9, 2, 3, 72, 40, 2, 3, 0.3),
+    (65, 4, 16, 520, 264, 5, 8, 0.1),
+    (33, 8, 32, 256, 1024, 3, 24, 0.0),
+])
+def test_combine_ragged(T, K, E, d, n, num_slots, rank, p_none):
+    tag = f"gpu/moe/combine/{T}/{K}/{E}"
+    batch = synth.config4_batch(T=T, E=E, K=K, num_slots=num_slots, rank=rank, p_none=p_none, tag=tag)
+    check_combine(synth.config4_projection(batch, "down", d=d, n=n, tag=tag), tag)
+    check_combine(synth.config4_projection(batch, "gate", d=d, n=n, tag=tag), tag + "/rows-of-tokens")
+
+
+def test_combine_is_deterministic():
+    batch = synth.config4_batch(T=256)
+    case = synth.config4_projection(batch, "down")
+    y0 = synth.normal_bf16(synth.stream("gpu/moe/combine/det"), (case.T, case.n), 1.0)
+    a, _ = run_combine(case, y0)
+    b, _ = run_combine(case, y0)
+    np.testing.assert_array_equal(a, b)

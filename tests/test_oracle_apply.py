@@ -321,3 +321,40 @@ def test_bf16_store_error_budget():
     rel = np.linalg.norm(yr - y) / np.linalg.norm(y)
     assert 2.0 ** -9 / np.sqrt(3) < rel < 2.0 ** -8 / np.sqrt(3)
     assert np.abs(yr - y).max() <= 2.0 ** -6 + 1e-12        # half-ulp for |y| in [4, 8)
+
+
+def test_combine_oracle_equals_explicit_weighted_sum_on_a_tiny_case():
+    """Brute force: Y[t] = Y0[t] + sum_k w s x A B with every product written out in numpy."""
+    from paper_2605_13779_b200 import synth
+    batch = synth.config4_batch(T=5, E=3, K=2, num_slots=2, rank=2, tag="oracle/combine")
+    case = synth.config4_projection(batch, "down", d=8, n=6, tag="oracle/combine")
+    y0 = synth.normal_bf16(synth.stream("oracle/combine/y0"), (case.T, case.n), 1.0)
+    t = case.table
+    got, missing = oracle.moe_lora_apply_combine(case.ids, case.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                                 case.A, case.B, case.x, y0, case.pair_weight)
+    assert missing == 0
+    A = synth.bf16_bits_to_f64(case.A)
+    B = synth.bf16_bits_to_f64(case.B)
+    x = synth.bf16_bits_to_f64(case.x)
+    want = synth.bf16_bits_to_f64(y0).copy()
+    for tok in range(case.T):
+        s = t.id_to_slot[case.ids[tok]]
+        for k in range(case.K):
+            p = tok * case.K + k
+            e = case.expert_ids[tok, k]
+            r = t.slot_rank[s]
+            v = x[p] @ A[s, e][:, :r]
+            want[tok] += float(case.pair_weight[p]) * float(t.slot_scale[s]) * (v @ B[s, e][:r, :])
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-14)
+
+
+def test_combine_oracle_with_one_expert_per_token_is_the_per_pair_apply():
+    from paper_2605_13779_b200 import synth
+    batch = synth.config4_batch(T=9, E=4, K=1, num_slots=3, rank=4, tag="oracle/combine1")
+    case = synth.config4_projection(batch, "down", d=16, n=8, tag="oracle/combine1")
+    t = case.table
+    a, _ = oracle.moe_lora_apply_combine(case.ids, case.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                         case.A, case.B, case.x, case.y0, case.pair_weight)
+    b, _ = oracle.moe_lora_apply(case.ids, case.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                 case.A, case.B, case.x, case.y0, pair_weight=case.pair_weight)
+    np.testing.assert_allclose(a, b, rtol=1e-13, atol=1e-15)
