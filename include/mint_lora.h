@@ -283,6 +283,20 @@ int32_t mint_lora_apply_fused_static(const mint_pool *pool, const mint_slot_tabl
                                      const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
                                      void *y_dev, int64_t ldy, int32_t *status_dev, mint_stream_t stream);
 
+/* Self-test of the bounded device-side waits (general rule above: a wait that
+ * ran out is recorded as MINT_ERR_TIMEOUT and the kernel returns).  Runs only the
+ * tensor-core shrink of the plan's dense segments (batches of 4096 tokens and
+ * more with runs of 128 and more tokens of one adapter) with its tensor-core
+ * work withheld and a 2 ms limit, so that nothing ever signals the barriers it
+ * waits on: every CTA that has a tile gives up, records MINT_ERR_TIMEOUT in
+ * status_dev (status_dev[2] = the tile) and writes nothing else; x is only
+ * read, workspace_dev (as for mint_lora_apply_fused) is left as it was.  A
+ * diagnostic for deployments, not part of the apply path.                     */
+int32_t mint_selftest_wait_timeout(const mint_pool *pool, const mint_slot_table *table,
+                                   const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
+                                   void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                                   mint_stream_t stream);
+
 /* Grouped form: the fused apply of up to MINT_MAX_GROUP projections that share
  * one plan (for instance q, k and v, which read the same x; or gate and up), in
  * one pair of launches.  An adapter's target modules come as a set (the paper's

@@ -43,7 +43,7 @@ EXPORTS = [
     "mint_lora_plan_bytes", "mint_lora_plan_layout", "mint_lora_plan", "mint_plan_fetch_summary",
     "mint_lora_shrink", "mint_lora_expand",
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
-    "mint_lora_apply_fused_static",
+    "mint_lora_apply_fused_static", "mint_selftest_wait_timeout",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
     "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
 ]
@@ -127,6 +127,7 @@ def load_library() -> ctypes.CDLL:
         "mint_lora_apply_fused": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, sz, vp, vp]),
         "mint_lora_apply_fused_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, vp, vp]),
         "mint_lora_apply_fused_static": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, vp]),
+        "mint_selftest_wait_timeout": (i32, [vp, vp, vp, i32, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
@@ -407,6 +408,14 @@ def mint_lora_apply_fused_static(pool: Pool, table: SlotTable, plan: Plan, x: to
         pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(y), _ld(y, pool.n),
         _ptr(status), _stream()))
     return y
+
+
+def mint_selftest_wait_timeout(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, status: torch.Tensor,
+                               workspace: torch.Tensor):
+    """Runs the dense-segment shrink with its tensor-core work withheld: its bounded waits run out."""
+    _check(load_library().mint_selftest_wait_timeout(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
 
 
 class ApplyGroup:

@@ -569,6 +569,34 @@ extern "C" int32_t mint_lora_apply_fused(const mint_pool *pool, const mint_slot_
   return mint_lora_apply_fused_grouped(&it, 1, table, plan_dev, T, status_dev, stream);
 }
 
+// Self-test of the bounded device-side waits: the tensor-core shrink of the plan's dense segments
+// alone, with its tensor-core work withheld, so that every wait of every CTA that has a tile runs out.
+extern "C" int32_t mint_selftest_wait_timeout(const mint_pool *pool, const mint_slot_table *table,
+                                              const void *plan_dev, int32_t T, const void *x_dev, int64_t ldx,
+                                              void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                                              mint_stream_t stream) {
+  int32_t st = check_dense(pool, table, plan_dev, T, "selftest_wait_timeout");
+  if (st) return st;
+  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "selftest_wait_timeout: null status_dev");
+  if (T < MINT_DENSE_MIN_BATCH || !mint_stream_supported(table->max_rank))
+    return mint_fail(MINT_ERR_UNSUPPORTED, "selftest_wait_timeout: needs a batch of at least %d tokens and ranks up to 64",
+                     MINT_DENSE_MIN_BATCH);
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "selftest_wait_timeout"))) return st;
+  const size_t need = mint_lora_apply_workspace_bytes(pool, T);
+  if (!workspace_dev || workspace_bytes < need)
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "selftest_wait_timeout: workspace %zu < %zu", workspace_bytes, need);
+  DenseArgs a = dense_args(pool, T);
+  a.x = static_cast<const uint16_t *>(x_dev);
+  a.ldx = ldx;
+  a.status = status_dev;
+  int32_t lanes = 0;
+  if ((st = mint_device_lanes(&lanes))) return st;
+  const int64_t tiles = mint_tile_upper_bound(1, T, table->num_slots);
+  void *ws[1] = {workspace_dev};
+  return mint_launch_dense_shrink(&a, 1, table_dev(table), plan_dev, ws, lanes, (int32_t)(tiles + MINT_MAX_LANES),
+                                  (int32_t)tiles, static_cast<cudaStream_t>(stream), true);
+}
+
 // ---------------------------------------------------------------------------
 // MoE
 // ---------------------------------------------------------------------------

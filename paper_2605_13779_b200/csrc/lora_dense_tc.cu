@@ -57,6 +57,8 @@ struct DenseParams {
   int32_t lanes;
   int32_t dense_slot0;   // part s of the v of dense tile t goes to workspace slot dense_slot0 + s * dense_stride + t
   int32_t dense_stride;
+  int32_t withhold;      // self-test only: no MMA is issued and nothing ever signals the barriers, so the waits run out
+  uint64_t wait_ns;      // limit of every wait
   int32_t *status;
   TableDev tab;
   PlanView pv;
@@ -83,8 +85,9 @@ __device__ __forceinline__ uint64_t global_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait for the phase with the given parity; false after about a second.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+constexpr uint64_t kWaitLimitNs = 1000000000ull;   // about a second
+// Bounded wait for the phase with the given parity; false once limit_ns have passed.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint64_t limit_ns = kWaitLimitNs) {
   const uint32_t a = smem_addr(bar);
   uint64_t t0 = 0;
   for (uint32_t it = 0;; ++it) {
@@ -100,7 +103,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
     if ((it & 63u) == 63u) {
       const uint64_t now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > 1000000000ull) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
 }
@@ -166,7 +169,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   __shared__ uint64_t all_done;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int32_t rows[kTileRows];
-  __shared__ int32_t failed;
+  __shared__ volatile int32_t failed;   // written after a wait that ran out; read only after a CTA barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const DenseProblem &pb = P.prob[blockIdx.y / MINT_DENSE_SPLIT_MAX];
   const int split = blockIdx.y % MINT_DENSE_SPLIT_MAX;
@@ -255,7 +258,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
     cp_async_wait<kStages - 2>();   // this thread's copies of chunk kc have landed
     fence_async_smem();             // ... and are visible to the tensor core's reads of shared memory
     __syncthreads();
-    if (tid == 0 && !failed) {
+    if (tid == 0 && !failed && !P.withhold) {
       tc_fence_after();
       const uint32_t xs = stage0 + (uint32_t)(s * kStageBytes), as = xs + kXStageBytes;
       const uint64_t da = smem_desc_k_sw128(xs), db = smem_desc_k_sw128(as);
@@ -267,13 +270,15 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
     // chunk kc + kStages - 1 reuses the stage of chunk kc - 1: wait for the MMAs that read it
     if (!failed && kc >= 1 && kc + kStages - 1 < nchunks) {
       const int sp = (kc - 1) % kStages;
-      if (!mbar_wait(&mma_done[sp], ((kc - 1) / kStages) & 1u)) failed = 1;
+      if (!mbar_wait(&mma_done[sp], ((kc - 1) / kStages) & 1u, P.wait_ns)) failed = 1;
     }
     issue(kc + kStages - 1);
   }
   cp_async_wait<0>();
-  if (tid == 0) umma_commit(&all_done);
-  if (!failed && !mbar_wait(&all_done, 0)) failed = 1;
+  if (tid == 0 && !P.withhold) umma_commit(&all_done);
+  // Also after an earlier wait ran out: whatever this CTA issued has to be complete (or given up on
+  // for a second time) before its tensor memory is freed.
+  if (!mbar_wait(&all_done, 0, P.wait_ns)) failed = 1;
   tc_fence_after();
   __syncthreads();
   if (!failed) {
@@ -376,9 +381,10 @@ __device__ __forceinline__ uint32_t sw128(int row, int c) {
 __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseExpandParams P) {
   extern __shared__ uint8_t dyn_raw[];
   __shared__ uint64_t mma_done;
+  __shared__ uint64_t drain;            // after a wait ran out: everything issued so far, once more
   __shared__ uint32_t tmem_base_slot;
   __shared__ int32_t rows[kTileRows];
-  __shared__ int32_t failed;
+  __shared__ volatile int32_t failed;   // written after a wait that ran out; read only after a CTA barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const DenseExpandProblem &pb = P.prob[blockIdx.z];
 
@@ -416,6 +422,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
   for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
   if (tid == 0) {
     mbar_init(&mma_done, 1);
+    mbar_init(&drain, 1);
     fence_mbar_init();
     failed = 0;
   }
@@ -568,7 +575,15 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
     __syncthreads();      // the y tile is free for the next chunk's copies
   }
   cp_async_wait<0>();
-  if (failed && tid == 0) report(P.status, MINT_ERR_TIMEOUT, m);
+  if (failed) {
+    // the MMAs of the chunk whose wait ran out may still be under way: give them one more bounded
+    // wait before the tensor memory they write is freed
+    if (tid == 0) {
+      report(P.status, MINT_ERR_TIMEOUT, m);
+      umma_commit(&drain);
+    }
+    mbar_wait(&drain, 0);
+  }
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_d, kExpTmemCols);
 }
@@ -577,7 +592,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
 
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                  void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
-                                 cudaStream_t s) {
+                                 cudaStream_t s, bool withhold_for_selftest) {
   static bool attr_set = false;
   if (!attr_set) {
     int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_shrink_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -603,6 +618,8 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
   P.lanes = lanes;
   P.dense_slot0 = dense_slot0;
   P.dense_stride = dense_stride;
+  P.withhold = withhold_for_selftest ? 1 : 0;
+  P.wait_ns = withhold_for_selftest ? 2000000ull : kWaitLimitNs;   // the self-test gives up after 2 ms
   P.status = args[0].status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);

@@ -226,9 +226,11 @@ int32_t mint_launch_fused(const DenseArgs &a, const TableDev &tab, const void *p
 bool mint_stream_supported(int32_t max_bound_rank);
 size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max);
 // Tensor-core shrink of the dense segments' 128-row tiles (between the two streamed kernels).
+// withhold_for_selftest: the kernel issues no tensor-core work and signals none of its barriers, and its
+// waits give up after 2 ms: every CTA with a tile reports MINT_ERR_TIMEOUT and writes nothing.
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                  void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
-                                 cudaStream_t s);
+                                 cudaStream_t s, bool withhold_for_selftest = false);
 // Tensor-core expand of the same tiles (after the streamed expand, which skips them).
 int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                  void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,

@@ -139,3 +139,40 @@ def test_moe_slot_admission():
     torch.cuda.synchronize()
     y_ref, _ = parity.oracle_moe(case)
     parity.assert_close(harness.y_to_f64(dev.y), y_ref, "moe admitted pool")
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """The tensor-core shrink of a batch with dense segments, with its tensor-core work withheld:
+    nothing ever signals the barriers its CTAs wait on, so every wait runs out after its limit.
+    The kernel reports MINT_ERR_TIMEOUT, writes nothing, frees its tensor memory and returns; the
+    next ordinary call on the same stream is correct."""
+    import time
+    from paper_2605_13779_b200 import binding as mb, harness, synth
+    import parity
+    import test_gpu_dense as dense
+    case = dense.dense_segment_case("gpu/timeout", [700, 130, 128, 3000, 300], [0, 1, 2, 3, 1], [64, 16, 8, 33],
+                                    d=1032, n=520, r_max=64)
+    assert case.T >= 4096
+    dev = harness.upload_dense(case)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    ws = mb.new_workspace(dev.pool, case.T)
+    ws.fill_(0x5A)
+    before = ws.clone()
+    y_before = dev.y.clone()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    mb.mint_selftest_wait_timeout(dev.pool, dev.table, plan, dev.x, dev.status, ws)
+    torch.cuda.synchronize()
+    elapsed = time.perf_counter() - t0
+    st = dev.status.cpu().numpy()
+    assert st[0] == mb.MINT_ERR_TIMEOUT, st
+    assert elapsed < 2.0                       # milliseconds per wait, not the second of the apply path
+    assert torch.equal(ws, before)             # no part of v was written
+    assert torch.equal(dev.y, y_before)
+    # the context is intact: the ordinary apply right after it matches the oracle
+    status = mb.new_status()
+    mb.mint_lora_apply_fused(dev.pool, dev.table, plan, dev.x, dev.y, status, workspace=ws)
+    torch.cuda.synchronize()
+    assert status[0].item() == 0
+    y_ref, _, _ = parity.oracle_dense(case)
+    parity.assert_close(harness.y_to_f64(dev.y), y_ref, "apply after a timed-out wait")
