@@ -1,25 +1,32 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-adapter LoRA apply on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3|config1]
     python bench.py --impl reference ...        # the fp64 CPU oracle, timed on the host cores
 
-A step is one pass of the whole hot path over one batch: one segment plan
-(token -> adapter grouping through the slot table) followed by the fused apply
-of every LoRA target projection of every layer.  The default workload is the
-4B-dense decode layer: T=256 requests, 64 resident adapters with ranks from
-{1, 8, 16, 32}, Zipf(1.1) request->adapter, seven projections per layer, 36
-layers; every layer has its own pool, x and y so that a step streams about
-4.5 GB (far beyond the 126 MB L2).  The step is captured in a CUDA graph and
-replayed; times are CUDA-event times on the launching stream.
+A step is a fixed number of passes of the whole hot path over one batch: each
+pass is one segment plan (token -> adapter grouping through the slot table)
+followed by the fused apply of every LoRA target projection of every layer.
+The default workload is the 4B-dense decode layer: T=256 requests, 64 resident
+adapters with ranks from {1, 8, 16, 32}, Zipf(1.1) request->adapter, seven
+projections per layer, 36 layers; every layer has its own pool, x and y so that
+a pass streams about 4.2 GB (far beyond the 126 MB L2).  The step is captured
+in a CUDA graph and replayed; times are CUDA-event times on the launching
+stream.  The passes per step are chosen once, before timing, so that a step
+lasts about 50 ms and the timed region (K steps) is long enough for the clock
+sampler to see it.
 
-Prints ONE JSON line (rank 0).  metric = tokens/s per layer: T * layers / step
-time, summed over ranks (ranks are independent replicas: the path has no
-exchange step, scaling is weak).
+Prints ONE JSON line (rank 0).  metric = tokens/s per layer: T * layers * passes
+/ step time, summed over ranks (ranks are independent replicas: the path has no
+exchange step, scaling is weak).  Besides the headline the line carries the
+same measurement for the dependency-respecting call grouping, for the other
+workloads, for the unfused pair of calls, for an L2-warm single layer and for
+the admission path.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import subprocess
@@ -35,15 +42,16 @@ if ROOT not in sys.path:
 
 METRIC = "mixed-adapter LoRA apply tokens/s per layer"
 UNIT = "tokens/s"
+STAGES = [[0, 1, 2], [3], [4, 5], [6]]      # q,k,v | o | gate,up | down: what a decoder layer's dependencies allow
 
 
 # --------------------------------------------------------------------------
 # workloads
 # --------------------------------------------------------------------------
 def build_workload(name: str, layers: int):
-    """Host-side description: a list of per-layer lists of cases, plus the
-    batch.  Only `distinct_layers` layers are drawn on the host; the device
-    copies cycle through them (values do not matter for timing, addresses do)."""
+    """Host-side description: the cases of one layer plus the batch.  The device
+    copies of the other layers are clones (values do not matter for timing,
+    addresses do)."""
     from paper_2605_13779_b200 import synth
     if name == "config2":
         batch = synth.config2_batch()
@@ -76,6 +84,13 @@ def algorithmic_bytes(wl) -> list:
     from paper_2605_13779_b200 import accounting
     fn = accounting.algorithmic_bytes_moe if wl["kind"] == "moe" else accounting.algorithmic_bytes_dense
     return [fn(c) for c in wl["cases"]]
+
+
+def hbm_peak():
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return json.load(open(peaks_path))["hbm_gbs"], "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback"
 
 
 # --------------------------------------------------------------------------
@@ -190,10 +205,242 @@ def run_reference(args):
 # --------------------------------------------------------------------------
 # GPU arm
 # --------------------------------------------------------------------------
+class DeviceWorkload:
+    """A workload resident on the device: every layer has its own pool, x and y."""
+
+    def __init__(self, wl, copies: int):
+        import torch
+        from paper_2605_13779_b200 import binding as mb, harness
+        self.mb, self.torch = mb, torch
+        self.wl = wl
+        self.moe = wl["kind"] == "moe"
+        self.T = wl["T"]
+        self.L = copies
+        self.base = [harness.upload_moe(c) if self.moe else harness.upload_dense(c) for c in wl["cases"]]
+        self.table = self.base[0].table
+        self.layers = []
+        for li in range(copies):
+            row = []
+            for dv in self.base:
+                if li == 0:
+                    row.append((dv.pool, dv.x, dv.y))
+                else:
+                    A, B = dv.pool.A.clone(), dv.pool.B.clone()
+                    pool = mb.Pool(A, B, dv.pool.d, dv.pool.n, dv.pool.r_max, dv.pool.num_slots,
+                                   num_experts=dv.pool.num_experts)
+                    row.append((pool, dv.x.clone(), dv.y.clone()))
+            self.layers.append(row)
+        self.ids = self.base[0].ids
+        self.status = mb.new_status()
+        self.expert_ids = self.base[0].expert_ids if self.moe else None
+        self.E = wl["cases"][0].E if self.moe else 0
+        self.K = wl["cases"][0].K if self.moe else 1
+        self.plan = mb.Plan(self.T, self.K, self.table.num_slots, self.E)
+        self.workspaces = ([mb.new_moe_workspace(dv.pool, self.T, self.K) for dv in self.base] if self.moe
+                           else [mb.new_workspace(dv.pool, self.T) for dv in self.base])
+        self.bytes_per_case = algorithmic_bytes(wl)
+        self.layer_bytes = sum(b["total"] for b in self.bytes_per_case)
+        self._groups = {}
+
+    def groups_idx(self, grouping):
+        ncase = len(self.wl["cases"])
+        if self.moe or grouping == "none" or ncase == 1:
+            return [[i] for i in range(ncase)]
+        if grouping == "layer":
+            return [list(range(ncase))]
+        return STAGES if ncase == 7 else [[i] for i in range(ncase)]
+
+    def enqueue_plan(self):
+        self.mb.mint_lora_plan(self.table, self.ids, self.status, expert_ids=self.expert_ids, num_experts=self.E,
+                               plan=self.plan)
+
+    def enqueue_layer(self, li, grouping):
+        mb = self.mb
+        if self.moe:
+            for ci, (pool, x, y) in enumerate(self.layers[li]):
+                mb.mint_moe_lora_apply(pool, self.table, self.plan, x, y, self.status, x_row=self.base[ci].x_row,
+                                       workspace=self.workspaces[ci])
+            return
+        key = (li, grouping)
+        if key not in self._groups:
+            row = self.layers[li]
+            self._groups[key] = [mb.ApplyGroup([(row[i][0], row[i][1], row[i][2], self.workspaces[i]) for i in g])
+                                 for g in self.groups_idx(grouping)]
+        for grp in self._groups[key]:
+            mb.mint_lora_apply_fused_grouped(grp, self.table, self.plan, self.status)
+
+    def enqueue_layer_unfused(self, li, v_bufs):
+        """shrink then expand through a v tensor of its own (dense workloads)."""
+        mb = self.mb
+        for ci, (pool, x, y) in enumerate(self.layers[li]):
+            mb.mint_lora_shrink(pool, self.table, self.plan, x, self.status, v=v_bufs[ci])
+            mb.mint_lora_expand(pool, self.table, self.plan, v_bufs[ci], y, self.status)
+
+    def launches_per_pass(self, grouping):
+        kernels_per_call = 4 if (not self.moe and self.T >= 4096) else 2
+        return 1 + self.L * len(self.groups_idx(grouping)) * kernels_per_call
+
+    def capture(self, stream, fn):
+        torch = self.torch
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g, stream=stream):
+                fn()
+        return g
+
+    def check_status(self, what):
+        st = self.status.cpu().numpy()
+        if st[0] != 0:
+            raise SystemExit(f"device status {self.mb.status_name(int(st[0]))} after {what}: the timed run is invalid")
+
+
+def time_graph(torch, dist, world, stream, graph, steps, warmup):
+    """K replays bracketed by a barrier and a synchronize on both sides; max over ranks (ms)."""
+    with torch.cuda.stream(stream):
+        for _ in range(warmup):
+            graph.replay()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            graph.replay()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def parity_of_first_layer(dw: DeviceWorkload, grouping):
+    """One layer of the call the bench times, on fresh copies of y, against the fp64 oracle."""
+    import torch
+    from oracle import oracle
+    from paper_2605_13779_b200 import harness, synth
+    saved = [y.clone() for (_, _, y) in dw.layers[0]]
+    dw.enqueue_plan()
+    dw.enqueue_layer(0, grouping)
+    torch.cuda.synchronize()
+    out = {"max_abs": 0.0, "rel_fro": 0.0, "max_abs_y_ref": 0.0}
+    for ci, c in enumerate(dw.wl["cases"]):
+        t = c.table
+        y = dw.layers[0][ci][2]
+        if dw.moe:
+            y_ref, _ = oracle.moe_lora_apply(c.ids, c.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B,
+                                             c.x, c.y0, x_row=c.x_row)
+            y_gpu = harness.y_to_f64(y)
+        else:
+            rows = None
+            if c.T * c.n > 64_000_000:      # sampled rows where the full comparison would take minutes
+                rows = np.sort(synth.stream("bench/parity", ci).choice(c.T, size=128, replace=False))
+            sel = slice(None) if rows is None else rows
+            y_ref, _, _ = oracle.lora_apply(c.ids[sel], t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B, c.x[sel], c.y0[sel])
+            y_gpu = harness.y_to_f64(y if rows is None else y[torch.from_numpy(rows).cuda()])
+        out["max_abs"] = max(out["max_abs"], float(np.abs(y_gpu - y_ref).max()))
+        out["rel_fro"] = max(out["rel_fro"], float(np.linalg.norm(y_gpu - y_ref) / np.linalg.norm(y_ref)))
+        out["max_abs_y_ref"] = max(out["max_abs_y_ref"], float(np.abs(y_ref).max()))
+    out["within_tolerance"] = bool(out["max_abs"] <= 3e-2 and out["rel_fro"] <= 5e-3)
+    for (_, _, y), s in zip(dw.layers[0], saved):
+        y.copy_(s)
+    return out
+
+
+def measure_side_workload(torch, dist, world, stream, name, peak):
+    """A short device-timed loop of another workload: us per layer, tokens/s per layer, roofline fraction."""
+    wl = build_workload(name, 0)
+    dw = DeviceWorkload(wl, wl["layers"])
+    dw.enqueue_plan()
+    for li in range(dw.L):
+        dw.enqueue_layer(li, "layer")
+    torch.cuda.synchronize()
+
+    def one_pass():
+        dw.enqueue_plan()
+        for li in range(dw.L):
+            dw.enqueue_layer(li, "layer")
+
+    def applies():
+        for li in range(dw.L):
+            dw.enqueue_layer(li, "layer")
+
+    g = dw.capture(stream, one_pass)
+    ga = dw.capture(stream, applies)
+    est = time_graph(torch, dist, world, stream, g, 2, 2) / 2
+    steps = int(min(200, max(5, 150.0 / max(est, 1e-3))))
+    ms = time_graph(torch, dist, world, stream, g, steps, 3) / steps
+    ms_a = time_graph(torch, dist, world, stream, ga, steps, 1) / steps
+    dw.check_status(name)
+    res = {"workload": wl["name"], "layers": dw.L, "us_per_layer": ms * 1e3 / dw.L,
+           "us_per_layer_apply_only": ms_a * 1e3 / dw.L,
+           "tokens_per_s": world * dw.T * dw.L / (ms * 1e-3), "bytes_per_layer": dw.layer_bytes,
+           "GBps": dw.layer_bytes / (ms * 1e-3 / dw.L) / 1e9,
+           "roofline_frac": dw.layer_bytes / (ms_a * 1e-3 / dw.L) / 1e9 / peak,
+           "roofline_frac_with_plan": dw.layer_bytes / (ms * 1e-3 / dw.L) / 1e9 / peak,
+           "replay_footprint_MB": dw.layer_bytes * dw.L / 1e6}
+    if name != "config3":
+        res["parity"] = parity_of_first_layer(dw, "layer")
+    del g, ga, dw
+    gc.collect()
+    torch.cuda.empty_cache()
+    return res
+
+
+def measure_admission(torch, stream):
+    """Admitting one adapter into the three expert projections of a 30B-A3B-shaped layer (128 experts):
+    the packed representation (one call per projection) against one copy per tensor."""
+    from paper_2605_13779_b200 import binding as mb, synth
+    E, slots = 128, 4
+    out = {}
+    for rank in (1, 16):
+        pools, packed = [], []
+        for d, n in synth.MOE_30B_PROJECTIONS.values():
+            A = torch.zeros(slots, E, d, 16, dtype=torch.bfloat16, device="cuda")
+            B = torch.zeros(slots, E, 16, n, dtype=torch.bfloat16, device="cuda")
+            pools.append(mb.Pool(A, B, d, n, 16, slots, num_experts=E))
+            packed.append((torch.randn(E, d, rank, device="cuda").to(torch.bfloat16),
+                           torch.randn(E, rank, n, device="cuda").to(torch.bfloat16)))
+        nbytes = sum(a.numel() * 2 + b.numel() * 2 for a, b in packed)
+
+        def admit_packed():
+            for pool, (a, b) in zip(pools, packed):
+                pool.admit_packed(1, a, b, rank)
+
+        def admit_per_tensor():
+            for pool, (a, b) in zip(pools, packed):
+                for e in range(E):
+                    pool.write_slot(1, a[e], b[e], rank, expert=e)
+
+        res = {}
+        with torch.cuda.stream(stream):
+            for nm, fn, reps in (("packed", admit_packed, 20), ("per_tensor", admit_per_tensor, 3)):
+                fn()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                for _ in range(reps):
+                    fn()
+                torch.cuda.synchronize()
+                res[nm] = (time.perf_counter() - t0) / reps
+        out[f"rank{rank}"] = {"bytes": nbytes, "tensors_per_layer": {"packed": 6, "per_tensor": 6 * E},
+                              "packed_us": res["packed"] * 1e6, "per_tensor_us": res["per_tensor"] * 1e6,
+                              "packed_GBps": nbytes / res["packed"] / 1e9,
+                              "admissions_per_s_packed_48_layers": 1.0 / (48 * res["packed"]),
+                              "speedup": res["per_tensor"] / res["packed"]}
+    out["what"] = ("one adapter into gate/up/down of one 128-expert layer, device-resident sources, "
+                   "host-timed including launch; per_tensor = one copy call per (expert, tensor)")
+    return out
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
-    from paper_2605_13779_b200 import binding as mb, harness
+    from paper_2605_13779_b200 import binding as mb
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -202,149 +449,130 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     mb.load_library()
+    peak, peak_src = hbm_peak()
 
     wl = build_workload(args.workload, args.layers)
-    L = wl["layers"]
-    T = wl["T"]
-    moe = wl["kind"] == "moe"
-    bytes_per_case = algorithmic_bytes(wl)
-    layer_bytes = sum(b["total"] for b in bytes_per_case)
-
-    # ---- device-resident inputs: every layer has its own pool, x and y -------
-    base = [harness.upload_moe(c) if moe else harness.upload_dense(c) for c in wl["cases"]]
-    table = base[0].table
-    layers = []
-    for li in range(L):
-        row = []
-        for dv in base:
-            if li == 0:
-                row.append((dv.pool, dv.x, dv.y))
-            else:
-                A, B = dv.pool.A.clone(), dv.pool.B.clone()
-                pool = mb.Pool(A, B, dv.pool.d, dv.pool.n, dv.pool.r_max, dv.pool.num_slots,
-                               num_experts=dv.pool.num_experts)
-                row.append((pool, dv.x.clone(), dv.y.clone()))
-        layers.append(row)
-    ids = base[0].ids
-    status = mb.new_status()
-    expert_ids = base[0].expert_ids if moe else None
-    E = wl["cases"][0].E if moe else 0
-    plan = mb.Plan(T, wl["cases"][0].K if moe else 1, table.num_slots, E)
-
-    def enqueue_plan():
-        mb.mint_lora_plan(table, ids, status, expert_ids=expert_ids, num_experts=E, plan=plan)
-
-    # call grouping: "none" = one fused call per projection; "stage" = projections that can run at the
-    # same point of a transformer layer share a call (q,k,v | o | gate,up | down); "layer" = one call per layer
-    ncase = len(wl["cases"])
-    if moe or args.grouping == "none" or ncase == 1:
-        groups_idx = [[i] for i in range(ncase)]
-    elif args.grouping == "layer":
-        groups_idx = [list(range(ncase))]
-    else:
-        groups_idx = [[0, 1, 2], [3], [4, 5], [6]] if ncase == 7 else [[i] for i in range(ncase)]
-    workspaces = ([mb.new_moe_workspace(dv.pool, T, wl["cases"][0].K) for dv in base] if moe
-                  else [mb.new_workspace(dv.pool, T) for dv in base])
-    groups = []
-    if not moe:
-        for row in layers:
-            groups.append([mb.ApplyGroup([(row[i][0], row[i][1], row[i][2], workspaces[i]) for i in g])
-                           for g in groups_idx])
-
-    def enqueue_layer(li):
-        if moe:
-            for ci, (pool, x, y) in enumerate(layers[li]):
-                mb.mint_moe_lora_apply(pool, table, plan, x, y, status, x_row=base[ci].x_row,
-                                       workspace=workspaces[ci])
-        else:
-            for grp in groups[li]:
-                mb.mint_lora_apply_fused_grouped(grp, table, plan, status)
-
-    def enqueue_applies():
-        for li in range(L):
-            enqueue_layer(li)
-
-    # a fused call is a shrink and an expand launch; batches that may hold dense segments add the two tensor-core kernels
-    kernels_per_call = 4 if (not moe and T >= 4096) else 2
-    calls_per_layer = len(groups_idx)
-    launches_per_step = 1 + L * calls_per_layer * kernels_per_call
-
-    # warm-up outside any graph (first launches load the module), then capture
-    enqueue_plan()
-    enqueue_applies()
-    torch.cuda.synchronize()
+    dw = DeviceWorkload(wl, wl["layers"])
+    L, T = dw.L, dw.T
+    grouping = args.grouping
     stream = torch.cuda.Stream()
-    step_graph = torch.cuda.CUDAGraph()
-    apply_graph = torch.cuda.CUDAGraph()
-    with torch.cuda.stream(stream):
-        with torch.cuda.graph(step_graph, stream=stream):
-            enqueue_plan()
-            enqueue_applies()
-        with torch.cuda.graph(apply_graph, stream=stream):
-            enqueue_applies()
-    torch.cuda.synchronize()
 
-    def timed(graph, steps, warmup):
-        with torch.cuda.stream(stream):
-            for _ in range(warmup):
-                graph.replay()
-            torch.cuda.synchronize()
-            if world > 1:
-                dist.barrier()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream)
-            for _ in range(steps):
-                graph.replay()
-            e1.record(stream)
-            torch.cuda.synchronize()
-            if world > 1:
-                dist.barrier()
-            ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+    # warm-up outside any graph (first launches load the module)
+    dw.enqueue_plan()
+    for li in range(L):
+        dw.enqueue_layer(li, grouping)
+    torch.cuda.synchronize()
+    parity = parity_of_first_layer(dw, grouping) if (rank == 0 and not args.profile) else None
+
+    def one_pass(g=grouping):
+        dw.enqueue_plan()
+        for li in range(L):
+            dw.enqueue_layer(li, g)
+
+    def applies(g=grouping):
+        for li in range(L):
+            dw.enqueue_layer(li, g)
+
+    # passes per step: a step of about 50 ms
+    probe = dw.capture(stream, one_pass)
+    est_ms = time_graph(torch, dist, world, stream, probe, 3, 2) / 3
+    passes = 1 if args.profile else int(min(64, max(1, round(50.0 / max(est_ms, 1e-3)))))
+    if world > 1:
+        t = torch.tensor([passes], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        passes = int(t.item())
+
+    def step_fn():
+        for _ in range(passes):
+            one_pass()
+
+    def apply_fn():
+        for _ in range(passes):
+            applies()
+
+    step_graph = dw.capture(stream, step_fn)
+    apply_graph = dw.capture(stream, apply_fn)
+    torch.cuda.synchronize()
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms_total = timed(step_graph, args.steps, args.warmup)
-    ms_apply = timed(apply_graph, args.steps, 1)
+    ms_total = time_graph(torch, dist, world, stream, step_graph, args.steps, args.warmup)
+    ms_apply = time_graph(torch, dist, world, stream, apply_graph, args.steps, 1)
     clocks = sampler.stop() if rank == 0 else None
     ms_step = ms_total / args.steps
-    value = world * T * L / (ms_step * 1e-3)
+    value = world * T * L * passes / (ms_step * 1e-3)
+    calls_per_layer = len(dw.groups_idx(grouping))
+    dw.check_status("the timed region")
 
     if args.profile:
         if rank == 0:
             print(json.dumps({"profile_run": True, "workload": wl["name"], "layers": L, "ms_per_step": ms_step,
-                              "us_per_layer": ms_step * 1e3 / L, "grouping": args.grouping,
-                              "layer_GBps": layer_bytes / (ms_step * 1e-3 / L) / 1e9,
-                              "avg_apply_call_us": ms_apply * 1e3 / args.steps / (L * calls_per_layer)}))
+                              "us_per_layer": ms_step * 1e3 / (L * passes), "grouping": grouping,
+                              "layer_GBps": dw.layer_bytes / (ms_step * 1e-3 / (L * passes)) / 1e9,
+                              "avg_apply_call_us": ms_apply * 1e3 / args.steps / (L * passes * calls_per_layer)}))
         return
+
+    # ---- the other schedules of the same workload (short loops) ---------------------
+    other = {}
+    if rank == 0 and not dw.moe and len(wl["cases"]) == 7:
+        alt = "stage" if grouping == "layer" else "layer"
+        ga = dw.capture(stream, lambda: applies(alt))
+        n = 30
+        ms = time_graph(torch, dist, 1, stream, ga, n, 3) / n
+        other[alt] = {"us_per_layer": ms * 1e3 / L, "calls_per_layer": len(dw.groups_idx(alt)),
+                      "roofline_frac": dw.layer_bytes / (ms * 1e-3 / L) / 1e9 / peak}
+        del ga
+    if rank == 0 and not dw.moe:
+        # the unfused pair of calls: v goes through a tensor of its own
+        v_bufs = [torch.empty(T, dv.pool.r_max, dtype=torch.float32, device="cuda") for dv in dw.base]
+        for li in range(min(L, 2)):
+            dw.enqueue_layer_unfused(li, v_bufs)
+        torch.cuda.synchronize()
+
+        def unfused():
+            for li in range(L):
+                dw.enqueue_layer_unfused(li, v_bufs)
+
+        gu = dw.capture(stream, unfused)
+        n = 10
+        ms = time_graph(torch, dist, 1, stream, gu, n, 2) / n
+        other["unfused_shrink_then_expand"] = {"us_per_layer": ms * 1e3 / L,
+                                               "roofline_frac": dw.layer_bytes / (ms * 1e-3 / L) / 1e9 / peak}
+        del gu, v_bufs
+    if rank == 0:
+        # L2-warm: the same single layer over and over (its working set stays in the 126 MB L2 where it fits)
+        def warm():
+            for _ in range(32):
+                dw.enqueue_layer(0, grouping)
+
+        gw = dw.capture(stream, warm)
+        n = 10
+        ms = time_graph(torch, dist, 1, stream, gw, n, 3) / n
+        other["l2_warm_single_layer"] = {"us_per_layer": ms * 1e3 / 32, "layer_MB": dw.layer_bytes / 1e6}
+        del gw
 
     # ---- end to end through the C ABI with host buffers --------------------------
     # Per step: ids, every x and every y0 come from pinned host memory, the plan and
     # all applies run, and every updated y goes back to pinned host memory.
     e2e_layers = min(L, 4)
-    host_ids = ids.cpu().pin_memory()
-    host_x = [[x.cpu().pin_memory() for (_, x, _) in row] for row in layers[:e2e_layers]]
-    host_y = [[y.cpu().pin_memory() for (_, _, y) in row] for row in layers[:e2e_layers]]
+    host_ids = dw.ids.cpu().pin_memory()
+    host_x = [[x.cpu().pin_memory() for (_, x, _) in row] for row in dw.layers[:e2e_layers]]
+    host_y = [[y.cpu().pin_memory() for (_, _, y) in row] for row in dw.layers[:e2e_layers]]
     h2d = host_ids.numel() * 8 + sum(t.numel() * 2 for row in host_x for t in row) + \
         sum(t.numel() * 2 for row in host_y for t in row)
     d2h = sum(t.numel() * 2 for row in host_y for t in row)
 
     def e2e_step():
-        ids.copy_(host_ids, non_blocking=True)
+        dw.ids.copy_(host_ids, non_blocking=True)
         for li in range(e2e_layers):
-            for ci, (pool, x, y) in enumerate(layers[li]):
+            for ci, (pool, x, y) in enumerate(dw.layers[li]):
                 x.copy_(host_x[li][ci], non_blocking=True)
                 y.copy_(host_y[li][ci], non_blocking=True)
-        enqueue_plan()
+        dw.enqueue_plan()
         for li in range(e2e_layers):
-            enqueue_layer(li)
-            for ci, (pool, x, y) in enumerate(layers[li]):
+            dw.enqueue_layer(li, grouping)
+            for ci, (pool, x, y) in enumerate(dw.layers[li]):
                 host_y[li][ci].copy_(y, non_blocking=True)
 
     with torch.cuda.stream(stream):
@@ -362,22 +590,16 @@ def run_gpu(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
     e2e_value = world * T * e2e_layers / e2e_s
-
-    st = status.cpu().numpy()
-    if st[0] != 0:
-        raise SystemExit(f"device status {mb.status_name(int(st[0]))}: the timed run is invalid")
-
+    dw.check_status("the end-to-end leg")
+    layer_bytes, launches = dw.layer_bytes, dw.launches_per_pass(grouping) * passes
+    del step_graph, apply_graph, probe, host_x, host_y
     if rank != 0:
         return
-    # ---- roofline of the dominant kernel (the fused apply) ------------------------
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_src = json.load(open(peaks_path))["hbm_gbs"], "measured (MEASURED_PEAKS.json hbm_gbs)"
-    else:
-        peak, peak_src = 6650.0, "fallback"
+
+    # ---- roofline of the dominant kernel pair (the fused apply) ------------------------
     # the apply is a shrink launch and an expand launch that overlap (programmatic dependent launch),
     # so the roofline unit is the pair: bytes of one call / time of one call
-    n_apply = L * calls_per_layer
+    n_apply = L * calls_per_layer * passes
     avg_launch_s = ms_apply * 1e-3 / args.steps / n_apply
     avg_launch_bytes = layer_bytes / calls_per_layer
     achieved = avg_launch_bytes / avg_launch_s / 1e9
@@ -388,53 +610,91 @@ def run_gpu(args):
                 "launches_timed": n_apply * args.steps, "traffic": None}
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch pair, as the ncu summary under profiles/ records it
     # for this workload and grouping (a line "traffic_bytes_per_launch = N"); null when there is no such record
-    summary = os.path.join(ROOT, "profiles", f"stream_kernels_{args.workload}_{args.grouping}.md")
+    summary = os.path.join(ROOT, "profiles", f"stream_kernels_{args.workload}_{grouping}.md")
     if os.path.exists(summary):
         import re
         m = re.search(r"traffic_bytes_per_launch\s*=\s*(\d+)", open(summary).read())
         if m:
             roofline["traffic"] = int(m.group(1))
+    us_layer = ms_step * 1e3 / (L * passes)
+    us_layer_apply = ms_apply * 1e3 / args.steps / (L * passes)
 
+    # ---- the other workloads, the admission path, the CPU oracle --------------------------
+    del dw
+    gc.collect()
+    torch.cuda.empty_cache()
+    workloads = {}
+    if args.workload == "config2" and not args.no_side_workloads:
+        for name in ("config5", "config4", "config3"):
+            workloads[name] = measure_side_workload(torch, dist, 1, stream, name, peak)
+    admission = None if args.no_side_workloads else measure_admission(torch, stream)
     cpu_val, cores, sample = oracle_layer_seconds(wl)
+
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 in, f32 accumulate", "data": "synthetic (seeded)",
-        "config": {"workload": wl["name"], "layers_per_step": L, "tokens": T,
-                   "l2": f"inputs larger than L2: every layer has its own pool/x/y, {layer_bytes * L / 1e6:.0f} MB algorithmic bytes per step",
-                   "grouping": args.grouping, "calls_per_layer": calls_per_layer,
-                   "timing": "CUDA graph of plan + all applies, CUDA events on the launching stream"},
-        "us_per_layer": ms_step * 1e3 / L,
+        "config": {"workload": wl["name"], "layers_per_pass": L, "passes_per_step": passes, "tokens": T,
+                   "l2": f"inputs larger than L2: every layer has its own pool/x/y, {layer_bytes * L / 1e6:.0f} MB algorithmic bytes per pass",
+                   "grouping": grouping, "calls_per_layer": calls_per_layer,
+                   "timing": "CUDA graph of (plan + all applies) x passes, CUDA events on the launching stream"},
+        "us_per_layer": us_layer,
+        "us_per_layer_apply_only": us_layer_apply,
+        "plan_share_us_per_layer": us_layer - us_layer_apply,
         "layer_bytes": layer_bytes,
-        "layer_GBps": layer_bytes / (ms_step * 1e-3 / L) / 1e9,
+        "layer_GBps": layer_bytes / (us_layer * 1e-6) / 1e9,
         "clocks": clocks,
+        "parity": parity,
         "roofline": roofline,
+        "schedules": other,
+        "workloads": workloads,
+        "admission": admission,
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "layers_per_step": e2e_layers},
-        "gpu_launches": launches_per_step * args.steps,
+        "gpu_launches": launches * args.steps,
     }
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
 
+def spawn_replicas(args):
+    """--gpus N without a launcher: start N replica processes of this script (one per GPU)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    procs = []
+    for r in range(args.gpus):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(args.gpus),
+                   MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable] + sys.argv, env=env))
+    rc = 0
+    for p in procs:
+        rc = p.wait() or rc
+    sys.exit(rc)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
-    ap.add_argument("--layers", type=int, default=0, help="layers per step (0 = the workload's own)")
+    ap.add_argument("--layers", type=int, default=0, help="layers per pass (0 = the workload's own)")
     ap.add_argument("--grouping", default="layer", choices=["none", "stage", "layer"],
                     help="how the projections of a layer are grouped into fused calls")
     ap.add_argument("--profile", action="store_true",
-                    help="device-timed part only (no end-to-end leg, no CPU oracle): the command profilers wrap")
+                    help="device-timed part only, one pass per step (no end-to-end leg, no CPU oracle): the command profilers wrap")
+    ap.add_argument("--no-side-workloads", action="store_true", help="skip the other workloads and the admission path")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_replicas(args)
     else:
         run_gpu(args)
 
