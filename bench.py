@@ -325,6 +325,8 @@ def parity_of_first_layer(dw: DeviceWorkload, grouping):
     from oracle import oracle
     from paper_2605_13779_b200 import harness, synth
     saved = [y.clone() for (_, _, y) in dw.layers[0]]
+    for (_, _, y), c in zip(dw.layers[0], dw.wl["cases"]):      # (earlier replays have updated y: start from y0 again)
+        y.copy_(dw.mb.bf16_from_bits(c.y0))
     dw.enqueue_plan()
     dw.enqueue_layer(0, grouping)
     torch.cuda.synchronize()

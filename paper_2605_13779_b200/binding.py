@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libmint_lora.so")
+# MINT_LORA_LIBRARY names another build of the same library (a debug or instrumented one).
+LIB_PATH = os.environ.get("MINT_LORA_LIBRARY") or os.path.join(_PKG, "libmint_lora.so")
 
 MINT_OK = 0
 MINT_ERR_INVALID_ARG = -1
