@@ -62,7 +62,7 @@ def build_workload(name: str, layers: int):
     if name == "config5":
         case = synth.config5()
         return {"kind": "dense", "name": "config5: 7168->7168, T=2048, 4096 rank-1 slots of a 10^6 catalog, Zipf(0.9)",
-                "T": case.T, "cases": [case], "layers": layers or 16}
+                "T": case.T, "cases": [case], "layers": layers or 61}   # a 7168-wide model is about 61 layers deep
     if name == "config1":
         case = synth.config1()
         return {"kind": "dense", "name": "config1: 2560->2560, T=64, 4 rank-8 adapters", "T": case.T,
@@ -76,7 +76,7 @@ def build_workload(name: str, layers: int):
         batch = synth.config4_batch()
         cases = [synth.config4_projection(batch, p) for p in ("gate", "up", "down")]
         return {"kind": "moe", "name": "config4: 30B-A3B MoE expert LoRA, T=4096, top-8 of 128 experts, 16 adapters r=16",
-                "T": batch.T, "cases": cases, "layers": layers or 4}
+                "T": batch.T, "cases": cases, "layers": layers or 16}
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -294,8 +294,9 @@ class DeviceWorkload:
             raise SystemExit(f"device status {self.mb.status_name(int(st[0]))} after {what}: the timed run is invalid")
 
 
-def time_graph(torch, dist, world, stream, graph, steps, warmup):
-    """K replays bracketed by a barrier and a synchronize on both sides; max over ranks (ms)."""
+def time_graph(torch, dist, world, stream, graph, steps, warmup, name="timed region"):
+    """K replays bracketed by a barrier and a synchronize on both sides; max over ranks (ms).
+    The timed replays sit in an NVTX range of the given name (visible to profilers)."""
     with torch.cuda.stream(stream):
         for _ in range(warmup):
             graph.replay()
@@ -304,10 +305,12 @@ def time_graph(torch, dist, world, stream, graph, steps, warmup):
             dist.barrier()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.nvtx.range_push(name)
         e0.record(stream)
         for _ in range(steps):
             graph.replay()
         e1.record(stream)
+        torch.cuda.nvtx.range_pop()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
@@ -499,8 +502,8 @@ def run_gpu(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms_total = time_graph(torch, dist, world, stream, step_graph, args.steps, args.warmup)
-    ms_apply = time_graph(torch, dist, world, stream, apply_graph, args.steps, 1)
+    ms_total = time_graph(torch, dist, world, stream, step_graph, args.steps, args.warmup, "steps: plan + applies")
+    ms_apply = time_graph(torch, dist, world, stream, apply_graph, args.steps, 1, "applies only")
     clocks = sampler.stop() if rank == 0 else None
     ms_step = ms_total / args.steps
     value = world * T * L * passes / (ms_step * 1e-3)
