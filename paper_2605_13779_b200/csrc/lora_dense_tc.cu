@@ -24,6 +24,8 @@
 //
 // Every wait on an mbarrier is bounded; a wait that runs out records
 // MINT_ERR_TIMEOUT, and the CTA still frees its tensor memory before it returns.
+#include <cuda.h>   // CUtensorMap and its enums only: the encoder is looked up through the runtime, nothing links to the driver
+
 #include "mint_device.cuh"
 
 using namespace mint;
@@ -48,7 +50,10 @@ struct DenseProblem {
   int64_t ldx;
   int32_t d, r_max;
   int32_t splits;      // CTAs per tile, each over an equal share of the 64-column chunks of d
+  int32_t use_tma;     // the two tensor maps below are valid
   float *ws_part;      // slots of 32 * r_max floats, [len][rank] packed fp32
+  alignas(64) CUtensorMap x_map;   // x as [T][d], boxes of 128 rows x 64 columns, 128-byte swizzle
+  alignas(64) CUtensorMap a_map;   // A as [slots * r_max][d], boxes of 64 rows x 64 columns
 };
 
 struct DenseParams {
@@ -107,6 +112,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint64
     }
   }
 }
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+// One 2-D tile, global -> shared through the tensor map (this GPU's own memory, no multicast); the
+// mbarrier counts the tile's bytes.  x = column (a multiple of 8 elements), y = row.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(smem_addr(bar))
+               : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t cols) {   // one whole warp
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(dst_smem)), "r"(cols)
                : "memory");
@@ -163,9 +178,10 @@ __device__ __forceinline__ uint32_t instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileRows >> 4) << 24);
 }
 
-__global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DenseParams P) {
+__global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_constant__ DenseParams P) {
   extern __shared__ uint8_t dyn_raw[];
-  __shared__ uint64_t mma_done[kStages];
+  __shared__ uint64_t mma_done[kStages];   // a stage's MMAs have read it
+  __shared__ uint64_t full[kStages];       // a stage's tiles have landed (tensor-map path)
   __shared__ uint64_t all_done;
   __shared__ uint32_t tmem_base_slot;
   __shared__ int32_t rows[kTileRows];
@@ -209,7 +225,10 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   const int n_mma = (r + 15) / 16 * 16;
   for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&mma_done[s], 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&mma_done[s], 1);
+      mbar_init(&full[s], 1);
+    }
     mbar_init(&all_done, 1);
     fence_mbar_init();
     failed = 0;
@@ -229,6 +248,55 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
 
   pdl_wait();
 
+  // A tile whose tokens are consecutive rows of x (a request's tokens usually are) comes in through the
+  // tensor maps: one thread asks for the two tiles of a chunk (hardware swizzle, bytes counted on the
+  // stage's mbarrier), another issues the MMAs as soon as a stage is full and hands it back when they
+  // have read it; nobody computes an address per row and no barrier of the CTA sits in the loop.
+  const bool contiguous = pb.use_tma && rows[nrows - 1] - rows[0] == nrows - 1;
+  if (contiguous) {
+    if (warp == 0) {
+     if (lane == 0) {   // producer
+      int kc = 0;
+      for (; kc < nchunks; ++kc) {
+        const int s = kc % kStages;
+        if (kc >= kStages && !mbar_wait(&mma_done[s], ((kc / kStages) - 1) & 1u, P.wait_ns)) {
+          failed = 1;
+          break;
+        }
+        const uint32_t xs = stage0 + (uint32_t)(s * kStageBytes), as = xs + kXStageBytes;
+        mbar_arrive_expect_tx(&full[s], (uint32_t)kStageBytes);
+        const int col = (chunk0 + kc) * kChunk;
+        tma_load_2d(xs, &pb.x_map, col, rows[0], &full[s]);
+        tma_load_2d(as, &pb.a_map, col, d0.slot * pb.r_max, &full[s]);
+      }
+      if (failed)   // the tiles still on their way land before this CTA's memory goes away
+        for (int j = max(0, kc - kStages); j < kc; ++j) mbar_wait(&full[j % kStages], (j / kStages) & 1u, 100000000ull);
+     }
+     __syncwarp();
+    } else if (warp == 1) {
+     if (lane == 0) {   // MMA issuer
+      bool ok_mma = true;
+      for (int kc = 0; kc < nchunks && ok_mma; ++kc) {
+        const int s = kc % kStages;
+        if (!mbar_wait(&full[s], (kc / kStages) & 1u, P.wait_ns)) {
+          failed = 1;
+          ok_mma = false;
+          break;
+        }
+        if (P.withhold) continue;
+        tc_fence_after();
+        const uint32_t xs = stage0 + (uint32_t)(s * kStageBytes), as = xs + kXStageBytes;
+        const uint64_t da = smem_desc_k_sw128(xs), db = smem_desc_k_sw128(as);
+#pragma unroll
+        for (int ks = 0; ks < kChunk / 16; ++ks)
+          umma_bf16(tmem_d, da + (uint64_t)(2 * ks), db + (uint64_t)(2 * ks), idesc, kc > 0 || ks > 0);
+        umma_commit(&mma_done[s]);
+      }
+      if (!P.withhold) umma_commit(&all_done);
+     }
+     __syncwarp();
+    }
+  } else {
   // this thread's 16-byte pieces of a stage: row q >> 3, chunk q & 7 for q = tid + 128 i
   auto issue = [&](int kc) {
     if (kc < nchunks) {
@@ -276,6 +344,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const DensePa
   }
   cp_async_wait<0>();
   if (tid == 0 && !P.withhold) umma_commit(&all_done);
+  }
   // Also after an earlier wait ran out: whatever this CTA issued has to be complete (or given up on
   // for a second time) before its tensor memory is freed.
   if (!mbar_wait(&all_done, 0, P.wait_ns)) failed = 1;
@@ -590,6 +659,41 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
 
 }  // namespace
 
+namespace {
+// The tensor-map encoder lives in the driver; it is looked up through the runtime once.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn tensor_map_encoder() {
+  static EncodeTiledFn fn = nullptr;
+  static bool looked = false;
+  if (!looked) {
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    else
+      (void)cudaGetLastError();
+    looked = true;
+  }
+  return fn;
+}
+// bf16 matrix [rows][cols] with a row stride of ld elements, boxes of box_rows x 64 columns in the
+// 128-byte-swizzled layout; elements outside the matrix read as zero.
+bool make_map_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  EncodeTiledFn enc = tensor_map_encoder();
+  if (!enc || rows == 0) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {ld * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+}  // namespace
+
 int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                  void *const *workspaces, int32_t lanes, int32_t dense_slot0, int32_t dense_stride,
                                  cudaStream_t s, bool withhold_for_selftest) {
@@ -613,6 +717,9 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
     pb.r_max = args[i].r_max;
     pb.splits = mint_dense_splits(args[i].d);
     pb.ws_part = static_cast<float *>(workspaces[i]);
+    pb.use_tma = make_map_2d(&pb.x_map, args[i].x, (uint64_t)T, (uint64_t)args[i].d, (uint64_t)args[i].ldx, kTileRows) &&
+                 make_map_2d(&pb.a_map, args[i].A, (uint64_t)args[i].num_slots * args[i].r_max, (uint64_t)args[i].d,
+                             (uint64_t)args[i].d, kMaxRank);
   }
   P.T = T;
   P.lanes = lanes;
