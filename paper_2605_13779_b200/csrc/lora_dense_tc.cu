@@ -412,7 +412,10 @@ struct DenseExpandProblem {
   int64_t ldy;
   int32_t n, r_max;
   int32_t splits;      // parts of v per tile (the shrink's split of d)
+  int32_t use_tma;     // the two tensor maps below are valid
   const float *ws_part;
+  alignas(64) CUtensorMap b_map;   // B as [slots * r_max][n], boxes of 64 rows x 64 columns, 128-byte swizzle
+  alignas(64) CUtensorMap y_map;   // y as [T][n], boxes of 128 rows x 64 columns
 };
 struct DenseExpandParams {
   DenseExpandProblem prob[kMaxProblems];
@@ -447,7 +450,7 @@ __device__ __forceinline__ uint32_t sw128(int row, int c) {
   return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((c ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseExpandParams P) {
+__global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_constant__ DenseExpandParams P) {
   extern __shared__ uint8_t dyn_raw[];
   __shared__ uint64_t mma_done;
   __shared__ uint64_t drain;            // after a wait ran out: everything issued so far, once more
@@ -488,6 +491,11 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
     return;
   }
   const int k_mma = (r + 15) / 16 * 16;
+  // tiles of consecutive tokens are the tensor-map kernel's
+  if (pb.use_tma && P.pv.perm[d0.off + nrows - 1] - P.pv.perm[d0.off] == nrows - 1) {
+    pdl_wait();
+    return;
+  }
   for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
   if (tid == 0) {
     mbar_init(&mma_done, 1);
@@ -657,6 +665,324 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const DenseEx
   if (warp == 0) tmem_dealloc(tmem_d, kExpTmemCols);
 }
 
+// ------------------------------------------------------------------------------------
+// The same expand for tiles whose tokens are consecutive rows of y (a request's tokens
+// usually are), as a pipeline of three roles over the 128-column chunks of the CTA's
+// column range.  One thread asks for the tiles of a chunk through tensor maps: B as two
+// boxes of 64 ranks x 64 columns, y as two boxes of 128 rows x 64 columns, all in the
+// 128-byte-swizzled layout.  B is used as it lies in memory (columns contiguous): its
+// shared-memory descriptor names the MN-major layout, so nothing is transposed.  One
+// thread issues the MMAs of a chunk as soon as its B has landed, into one of two
+// accumulators in tensor memory.  Four warps add the accumulator to the y tile in shared
+// memory (tcgen05.ld, one row per thread) and hand the tile to a tensor-map store (full
+// tiles) or store its rows themselves (a segment's last, shorter tile: the rows beyond it
+// belong to another CTA).  Three buffers of B and y, two accumulators: the loads and the MMAs of chunk
+// kc + 1 run under the epilogue of chunk kc.  Every wait is bounded.
+constexpr int kEpiThreads = 256;                   // 8 epilogue warps: warp w takes rows 32 (w % 4) .., columns 64 (w / 4) .. of a chunk
+constexpr int kTmaThreads = kEpiThreads + 64;      // + the producer's warp and the MMA warp
+constexpr int kBHalfBytes = kMaxRank * 128;        // 64 ranks x 64 columns
+constexpr int kBBufBytes = 2 * kBHalfBytes;        // 16 KB
+constexpr int kYHalfBytes = kTileRows * 128;       // 128 rows x 64 columns
+constexpr int kYBufBytes = 2 * kYHalfBytes;        // 32 KB
+constexpr int kBufs = 3;                            // chunks whose B and y tiles are in shared memory at a time
+constexpr size_t kTmaDynSmem = 2 * kVBytes + kBufs * kBBufBytes + kBufs * kYBufBytes + 1024;
+constexpr int kTmaTmemCols = 256;                  // two accumulators of 128 columns
+
+// Shared-memory descriptor of an MN-major bf16 operand in the 128-byte-swizzled layout: rows are
+// K, 64 MN elements (128 bytes) per row; groups of 8 rows 1024 bytes apart (stride offset);
+// the next 64 MN elements `lbo` bytes further (leading offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t lbo) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B MN-major, M = 128, N = n
+__device__ __forceinline__ uint32_t instr_desc_b_mn(int n) { return instr_desc(n) | (1u << 16); }
+// One 2-D tile, shared -> global through the tensor map; completion is tracked in the thread's bulk group.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// 16 consecutive fp32 columns of this thread's accumulator row, without waiting for them
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const __grid_constant__ DenseExpandParams P) {
+  extern __shared__ uint8_t dyn_raw[];
+  __shared__ uint64_t b_full[kBufs], b_free[kBufs];   // B of a chunk has landed / its MMAs have read it
+  __shared__ uint64_t y_full[kBufs], y_free[kBufs];   // the y tile has landed / has gone back to memory
+  __shared__ uint64_t acc_full[2], acc_free[2];   // the chunk's MMAs are complete / the accumulator has been read
+  __shared__ uint64_t y_written[kBufs];           // every epilogue thread has updated (and, for short tiles, stored) its row
+  __shared__ uint64_t drain;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile int32_t failed;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const DenseExpandProblem &pb = P.prob[blockIdx.z];
+
+  pdl_launch_dependents();
+  const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
+                  P.pv.header[PH_LANES] == P.lanes;
+  const int m = blockIdx.x;
+  const int col_begin = blockIdx.y * kColsPerCta;
+  if (!ok || !pb.use_tma || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n) {
+    pdl_wait();
+    return;
+  }
+  const int col_end = min(pb.n, col_begin + kColsPerCta);
+  const int ntiles = P.pv.header[PH_NCHUNK1];
+  const int t0 = P.pv.dense_tile[m];
+  const TileDesc d0 = P.pv.tile_desc[t0];
+  int nrows = d0.len;
+  {
+    TileDesc dn[3];   // the three descriptors that may follow, requested together
+#pragma unroll
+    for (int i = 1; i < 4; ++i) dn[i - 1] = P.pv.tile_desc[min(t0 + i, ntiles - 1)];
+#pragma unroll
+    for (int i = 1; i < 4; ++i) {
+      const TileDesc &di = dn[i - 1];
+      if (nrows != 32 * i || t0 + i >= ntiles || !di.dense || di.slot != d0.slot || di.off != d0.off + 32 * i) break;
+      nrows += di.len;
+    }
+  }
+  const int r = d0.rank;
+  const int row0 = P.pv.perm[d0.off];
+  // tiles whose tokens are scattered, and ranks the kernels do not take, are the other kernel's
+  if (r > pb.r_max || r > kMaxRank || r < 1 || P.pv.perm[d0.off + nrows - 1] - row0 != nrows - 1) {
+    pdl_wait();
+    return;
+  }
+  const int k_mma = (r + 15) / 16 * 16;
+  if (tid == 0) {
+    for (int b = 0; b < kBufs; ++b) {
+      mbar_init(&b_full[b], 1);
+      mbar_init(&b_free[b], 1);
+      mbar_init(&y_full[b], 1);
+      mbar_init(&y_free[b], 1);
+      mbar_init(&y_written[b], kEpiThreads);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_free[b], kEpiThreads);
+    }
+    mbar_init(&drain, 1);
+    fence_mbar_init();
+    failed = 0;
+  }
+  if (warp == 0) tmem_alloc(&tmem_base_slot, kTmaTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_d = tmem_base_slot;
+  const uint32_t base = (smem_addr(dyn_raw) + 1023u) & ~1023u;
+  const uint32_t v_hi = base, v_lo = base + kVBytes;
+  const uint32_t b_buf = base + 2 * kVBytes, y_buf = b_buf + kBufs * kBBufBytes;
+  const int nchunks = (col_end - col_begin + kExpChunk - 1) / kExpChunk;
+  const bool full_tile = nrows == kTileRows;   // (the tile's 128 rows are all this CTA's: whole boxes may be stored)
+
+  pdl_wait();   // v and y belong to the earlier kernels until here
+
+  if (warp == kEpiThreads / 32) {
+    // ---- producer ----
+    if (lane == 0) {
+      int kc = 0;
+      for (; kc < nchunks; ++kc) {
+        const int b = kc % kBufs;
+        const uint32_t par = ((kc / kBufs) & 1u) ^ 1u;   // (the buffers start out free)
+        const int col = col_begin + kc * kExpChunk;
+        if (!mbar_wait(&b_free[b], par)) { failed = 1; break; }
+        mbar_arrive_expect_tx(&b_full[b], (uint32_t)kBBufBytes);
+        tma_load_2d(b_buf + (uint32_t)(b * kBBufBytes), &pb.b_map, col, d0.slot * pb.r_max, &b_full[b]);
+        tma_load_2d(b_buf + (uint32_t)(b * kBBufBytes + kBHalfBytes), &pb.b_map, col + 64, d0.slot * pb.r_max, &b_full[b]);
+        if (!mbar_wait(&y_free[b], par)) { failed = 1; break; }
+        mbar_arrive_expect_tx(&y_full[b], (uint32_t)kYBufBytes);
+        tma_load_2d(y_buf + (uint32_t)(b * kYBufBytes), &pb.y_map, col, row0, &y_full[b]);
+        tma_load_2d(y_buf + (uint32_t)(b * kYBufBytes + kYHalfBytes), &pb.y_map, col + 64, row0, &y_full[b]);
+      }
+      if (failed)   // the tiles still on their way land before this CTA's memory goes away
+        for (int j = max(0, kc - kBufs); j < kc; ++j) {
+          mbar_wait(&b_full[j % kBufs], (j / kBufs) & 1u, 100000000ull);
+          mbar_wait(&y_full[j % kBufs], (j / kBufs) & 1u, 100000000ull);
+        }
+    }
+    __syncwarp();
+  } else if (warp == kEpiThreads / 32 + 1) {
+    // ---- MMA issuer (the whole warp clears the rank rows beyond the slot's rank first) ----
+    const uint32_t idesc = instr_desc_b_mn(kExpChunk);
+    for (int kc = 0; kc < nchunks; ++kc) {
+      const int b = kc % kBufs, ab = kc & 1;                          // buffer of B, accumulator
+      const uint32_t par = (kc / kBufs) & 1u, apar = (kc >> 1) & 1u;
+      bool good = mbar_wait(&b_full[b], par);
+      const uint32_t bs = b_buf + (uint32_t)(b * kBBufBytes);
+      if (good && r < k_mma) {
+        // rows r .. k_mma - 1 of the boxes are whatever follows the slot's rows in the pool: v is zero
+        // there, but zero times a NaN is not
+        for (int q = lane; q < (k_mma - r) * 16; q += 32) {
+          const int row = r + (q >> 4), c = q & 15;
+          sts128(bs + (uint32_t)((c >> 3) * kBHalfBytes) + sw128(row, c & 7), make_uint4(0u, 0u, 0u, 0u));
+        }
+        fence_async_smem();
+      }
+      __syncwarp();
+      if (lane == 0) {
+        good = good && mbar_wait(&acc_free[ab], apar);   // (phase 0 of it: v is in place)
+        if (!good) failed = 1;
+        else {
+          tc_fence_after();
+          const uint32_t acc = tmem_d + (uint32_t)(ab * kExpChunk);
+          const uint64_t dh = smem_desc_k_sw128(v_hi), dl = smem_desc_k_sw128(v_lo);
+          const uint64_t db = smem_desc_mn_sw128(bs, (uint32_t)kBHalfBytes);
+          // a step of 16 ranks: 32 bytes further along v's rows, two 8-row groups further down B
+          for (int ks = 0; ks < k_mma / 16; ++ks)
+            umma_bf16(acc, dh + (uint64_t)(2 * ks), db + (uint64_t)(128 * ks), idesc, ks > 0);
+          for (int ks = 0; ks < k_mma / 16; ++ks)
+            umma_bf16(acc, dl + (uint64_t)(2 * ks), db + (uint64_t)(128 * ks), idesc, true);
+          umma_commit(&acc_full[ab]);
+          umma_commit(&b_free[b]);
+        }
+      }
+      __syncwarp();
+      if (failed) break;
+    }
+    if (lane == 0 && failed) {   // whatever was issued is complete (or given up on once more) before tensor memory is freed
+      umma_commit(&drain);
+      mbar_wait(&drain, 0);
+    }
+    __syncwarp();
+  } else {
+    // ---- epilogue warps; first v, scaled, as head and remainder (consecutive threads: consecutive rank pairs of a row) ----
+    {
+      const size_t slot_floats = (size_t)32 * pb.r_max;
+      const int pairs = k_mma / 2;
+      for (int q0 = tid; q0 < kTileRows * pairs; q0 += 8 * kEpiThreads) {
+        float a[8], b[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) a[u] = b[u] = 0.f;
+        for (int sp = 0; sp < pb.splits; ++sp) {   // the parts of the shrink's CTAs, in their order; 16 loads go out together
+          float pa[8], pbv[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int q = q0 + u * kEpiThreads;
+            const int row = q / pairs, k = 2 * (q - row * pairs);
+            const bool in = q < kTileRows * pairs && row < nrows;
+            const float *src = pb.ws_part + (size_t)(P.dense_slot0 + sp * P.dense_stride + t0 + (row >> 5)) * slot_floats +
+                               (size_t)(row & 31) * r;
+            pa[u] = (in && k < r) ? __ldcg(src + k) : 0.f;
+            pbv[u] = (in && k + 1 < r) ? __ldcg(src + k + 1) : 0.f;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            a[u] += pa[u];
+            b[u] += pbv[u];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int q = q0 + u * kEpiThreads;
+          if (q < kTileRows * pairs) {
+            const int row = q / pairs, k = 2 * (q - row * pairs);
+            const float fa = d0.scale * a[u], fb = d0.scale * b[u];
+            const uint32_t hi = pack_bf16x2(fa, fb);
+            const uint32_t lo = pack_bf16x2(fa - bf16lo(hi), fb - bf16hi(hi));
+            const uint32_t off = sw128(row, k >> 3) + (uint32_t)((k & 7) * 2);
+            sts32(v_hi + off, hi);
+            sts32(v_lo + off, lo);
+          }
+        }
+      }
+      fence_async_smem();   // the operand writes are visible to the tensor core
+      // (accumulator 0 and 1 are "read" before their first use: this arrival also tells the MMA thread that v is in place)
+      mbar_arrive(&acc_free[0]);
+      mbar_arrive(&acc_free[1]);
+    }
+    for (int kc = 0; kc < nchunks; ++kc) {
+      const int b = kc % kBufs, ab = kc & 1;
+      const uint32_t par = (kc / kBufs) & 1u, apar = (kc >> 1) & 1u;
+      if (!mbar_wait(&acc_full[ab], apar) || !mbar_wait(&y_full[b], par)) {
+        failed = 1;
+        break;
+      }
+      tc_fence_after();
+      const int col0 = col_begin + kc * kExpChunk;
+      const uint32_t yb = y_buf + (uint32_t)(b * kYBufBytes);
+      // this thread's row of its half of the tile (64 columns): y += accumulator; the four loads of
+      // tensor memory go out together
+      const int row = (warp & 3) * 32 + lane, half = warp >> 2;
+      const uint32_t yh = yb + (uint32_t)(half * kYHalfBytes);
+      {
+        uint32_t acc[4][16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          tmem_ld16_issue(tmem_d + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)(ab * kExpChunk + half * 64 + q * 16), acc[q]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            const uint32_t addr = yh + sw128(row, 2 * q + h);
+            float f[8];
+            unpack8(lds128(addr), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] += __uint_as_float(acc[q][8 * h + e]);
+            sts128(addr, pack8(f));
+          }
+      }
+      tc_fence_before();
+      mbar_arrive(&acc_free[ab]);   // the accumulator may be overwritten
+      if (!full_tile) {
+        // a short tile: the warp's rows of its half go back to memory row by row (four rows per instruction)
+        __syncwarp();
+        const int c = lane & 7;
+        if (col0 + half * 64 + c * 8 < col_end) {
+#pragma unroll 4
+          for (int i = 0; i < 8; ++i) {
+            const int rr = (warp & 3) * 32 + 4 * i + (lane >> 3);
+            if (rr < nrows)
+              *reinterpret_cast<uint4 *>(pb.y + (int64_t)(row0 + rr) * pb.ldy + col0 + half * 64 + c * 8) =
+                  lds128(yh + sw128(rr, c));
+          }
+        }
+      }
+      fence_async_smem();   // this thread's writes to the tile are visible to the store below
+      mbar_arrive(&y_written[b]);
+      if (tid == 0) {
+        if (!mbar_wait(&y_written[b], par)) {
+          failed = 1;
+          break;
+        }
+        if (full_tile) {   // (columns beyond n are clipped by the tensor map)
+          tma_store_2d(&pb.y_map, col0, row0, yb);
+          tma_store_2d(&pb.y_map, col0 + 64, row0, yb + (uint32_t)kYHalfBytes);
+          bulk_commit();
+          bulk_wait_read();   // the tile has been read: the buffer may be refilled
+        }
+        mbar_arrive(&y_free[b]);
+      }
+    }
+    if (tid == 0) bulk_wait_all();   // the stores are complete before the kernel ends
+  }
+  __syncthreads();
+  if (failed && tid == 0) report(P.status, MINT_ERR_TIMEOUT, m);
+  tc_fence_after();
+  if (warp == 0) tmem_dealloc(tmem_d, kTmaTmemCols);
+}
+
 }  // namespace
 
 namespace {
@@ -752,6 +1078,9 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
     int32_t st = mint_check_cuda(cudaFuncSetAttribute(dense_expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                       (int)kExpDynSmem), "dense_expand shared memory");
     if (st) return st;
+    st = mint_check_cuda(cudaFuncSetAttribute(dense_expand_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kTmaDynSmem), "dense_expand (tensor maps) shared memory");
+    if (st) return st;
     attr_set = true;
   }
   const int32_t T = args[0].T;
@@ -759,6 +1088,7 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
   if (tiles == 0) return MINT_OK;
   DenseExpandParams P = {};
   int32_t n_max = 0;
+  bool any_tma = false;
   for (int i = 0; i < nprob; ++i) {
     DenseExpandProblem &pb = P.prob[i];
     pb.B = args[i].B;
@@ -768,6 +1098,10 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
     pb.r_max = args[i].r_max;
     pb.splits = mint_dense_splits(args[i].d);
     pb.ws_part = static_cast<const float *>(workspaces[i]);
+    pb.use_tma = make_map_2d(&pb.b_map, args[i].B, (uint64_t)args[i].num_slots * args[i].r_max, (uint64_t)args[i].n,
+                             (uint64_t)args[i].n, kMaxRank) &&
+                 make_map_2d(&pb.y_map, args[i].y, (uint64_t)T, (uint64_t)args[i].n, (uint64_t)args[i].ldy, kTileRows);
+    any_tma = any_tma || pb.use_tma;
     n_max = pb.n > n_max ? pb.n : n_max;
   }
   P.T = T;
@@ -787,5 +1121,10 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_expand_kernel, P), "dense_expand launch");
+  int32_t st = mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_expand_kernel, P), "dense_expand launch");
+  if (st || !any_tma) return st;
+  // the tiles of consecutive tokens: same grid, six warps, one CTA per SM
+  cfg.blockDim = dim3(kTmaThreads);
+  cfg.dynamicSmemBytes = kTmaDynSmem;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, dense_expand_tma_kernel, P), "dense_expand (tensor maps) launch");
 }
