@@ -201,7 +201,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_
     return;
   }
   const int ntiles = P.pv.header[PH_NCHUNK1];
-  const int t0 = P.pv.dense_tile[m];
+  const int listed = P.pv.dense_tile[m];
+  const int t0 = listed < 0 ? ~listed : listed;   // (~tile: the plan found its tokens scattered)
   const TileDesc d0 = P.pv.tile_desc[t0];
   // the 128-row tile = up to four consecutive 32-token tiles of the segment
   int nrows = d0.len;
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_
   // tensor maps: one thread asks for the two tiles of a chunk (hardware swizzle, bytes counted on the
   // stage's mbarrier), another issues the MMAs as soon as a stage is full and hands it back when they
   // have read it; nobody computes an address per row and no barrier of the CTA sits in the loop.
-  const bool contiguous = pb.use_tma && rows[nrows - 1] - rows[0] == nrows - 1;
+  const bool contiguous = pb.use_tma && listed >= 0;
   if (contiguous) {
     if (warp == 0) {
      if (lane == 0) {   // producer
@@ -465,13 +466,20 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
                   P.pv.header[PH_LANES] == P.lanes;
   const int m = blockIdx.x;
   const int col_begin = blockIdx.y * kColsPerCta;
-  if (!ok || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n) {
+  // (with tensor maps this kernel is left the tiles whose tokens are scattered: usually none)
+  if (!ok || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n ||
+      (pb.use_tma && P.pv.header[PH_NUM_SCATTERED] == 0)) {
     pdl_wait();
     return;
   }
   const int col_end = min(pb.n, col_begin + kColsPerCta);
   const int ntiles = P.pv.header[PH_NCHUNK1];
-  const int t0 = P.pv.dense_tile[m];
+  const int listed = P.pv.dense_tile[m];
+  if (pb.use_tma && listed >= 0) {   // a tile of consecutive tokens is the tensor-map kernel's
+    pdl_wait();
+    return;
+  }
+  const int t0 = listed < 0 ? ~listed : listed;
   const TileDesc d0 = P.pv.tile_desc[t0];
   int nrows = d0.len;
   {
@@ -491,11 +499,6 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
     return;
   }
   const int k_mma = (r + 15) / 16 * 16;
-  // tiles of consecutive tokens are the tensor-map kernel's
-  if (pb.use_tma && P.pv.perm[d0.off + nrows - 1] - P.pv.perm[d0.off] == nrows - 1) {
-    pdl_wait();
-    return;
-  }
   for (int i = tid; i < kTileRows; i += kThreads) rows[i] = i < nrows ? P.pv.perm[d0.off + i] : 0;
   if (tid == 0) {
     mbar_init(&mma_done, 1);
@@ -748,6 +751,10 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
   const int col_end = min(pb.n, col_begin + kColsPerCta);
   const int ntiles = P.pv.header[PH_NCHUNK1];
   const int t0 = P.pv.dense_tile[m];
+  if (t0 < 0) {   // its tokens are scattered: the other kernel's
+    pdl_wait();
+    return;
+  }
   const TileDesc d0 = P.pv.tile_desc[t0];
   int nrows = d0.len;
   {
@@ -763,8 +770,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
   }
   const int r = d0.rank;
   const int row0 = P.pv.perm[d0.off];
-  // tiles whose tokens are scattered, and ranks the kernels do not take, are the other kernel's
-  if (r > pb.r_max || r > kMaxRank || r < 1 || P.pv.perm[d0.off + nrows - 1] - row0 != nrows - 1) {
+  if (r > pb.r_max || r > kMaxRank || r < 1) {   // reported by the shrink
     pdl_wait();
     return;
   }

@@ -33,7 +33,8 @@ enum {
   PH_ROWS_SHRINK,  // sum over list-1 tiles of mint_tile_rows_shrink
   PH_ROWS_EXPAND,  // sum over list-1 tiles of mint_tile_rows_expand
   PH_MAX_TILE_ROWS,  // largest mint_tile_rows_shrink of a list-1 tile that the streamed shrink handles
-  PH_NUM_DENSE,      // number of 128-row tiles of dense segments (tensor-core shrink)
+  PH_NUM_DENSE,      // number of 128-row tiles of dense segments (tensor-core kernels)
+  PH_NUM_SCATTERED,  // how many of them hold tokens that are not consecutive rows (listed as ~tile in dense_tile)
   PH_WORDS = 32
 };
 #define MINT_PLAN_MAGIC 0x4D4C5032  // "MLP2"
@@ -129,7 +130,7 @@ struct PlanOffsets {
   int64_t tile_seg[MINT_NUM_TILE_LISTS];  // int32[P]  segment of tile c
   int64_t tile_off[MINT_NUM_TILE_LISTS];  // int32[P]  first position (in perm) of tile c
   int64_t tile_desc;   // TileDesc[tile upper bound of list 1]
-  int64_t dense_tile;  // int32[tile upper bound of list 1]  first list-1 tile of every 128-row dense tile
+  int64_t dense_tile;  // int32[tile upper bound of list 1]  first list-1 tile c of every 128-row dense tile (~c: its tokens are scattered)
   int64_t lane_shrink; // LaneStart[MINT_MAX_LANES + 1]  start of cost lane j in the shrink rows
   int64_t lane_expand; // LaneStart[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch

@@ -74,8 +74,9 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   __shared__ int32_t hist[kWarps][256];
   __shared__ int32_t bin_base[256];
   __shared__ int warp_tot[kWarps + 1];
-  __shared__ int32_t counters[8];  // 0 inactive, 1 not resident, 2 first missing token, 3 bad expert,
-                                   // 4 first bad item, 5 max segment, 6 sum rank, 7 max tile rows
+  __shared__ int32_t counters[9];  // 0 inactive, 1 not resident, 2 first missing token, 3 bad expert,
+                                   // 4 first bad item, 5 max segment, 6 sum rank, 7 max tile rows,
+                                   // 8 dense 128-row tiles whose tokens are not consecutive rows
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.P;
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   int32_t *idx_a = reinterpret_cast<int32_t *>(p.blob + p.off.idx_a);
   int32_t *idx_b = reinterpret_cast<int32_t *>(p.blob + p.off.idx_b);
 
-  if (tid < 8) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff : 0;
+  if (tid < 9) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff : 0;
   __syncthreads();
 
   // ---- keys: id -> slot through the table, (expert, slot) -> key ----------
@@ -320,7 +321,15 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       dsc.rows_shrink = run_s;
       dsc.rows_expand = run_e;
       dsc.dense = is_dense(sg) ? 1 : 0;
-      if (dsc.dense && ((toff[c] - seg_start[sg]) % 128) == 0) dense_tile[run_m++] = c;
+      if (dsc.dense && ((toff[c] - seg_start[sg]) % 128) == 0) {
+        // a 128-row tile of a dense segment; its tokens are consecutive rows (a request's tokens
+        // usually are) when the last index is the first plus the count: then the tensor-core kernels
+        // fetch it through tensor maps.  Scattered tiles are listed as ~c.
+        const int rows128 = min(128, seg_start[sg + 1] - toff[c]);
+        const bool scattered = perm[toff[c] + rows128 - 1] - perm[toff[c]] != rows128 - 1;
+        if (scattered) atomicAdd(&counters[8], 1);
+        dense_tile[run_m++] = scattered ? ~c : c;
+      }
       const int begin[2] = {run_s, run_e};
       const int end[2] = {run_s + (dsc.dense ? 0 : mint_tile_rows_shrink(dsc.rank, dsc.len)),
                           run_e + (dsc.dense ? 0 : mint_tile_rows_expand(dsc.rank, dsc.len))};
@@ -388,7 +397,8 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     hdr[PH_ROWS_EXPAND] = rows_total[1];
     hdr[PH_MAX_TILE_ROWS] = counters[7];
     hdr[PH_NUM_DENSE] = num_dense;
-    for (int w = PH_NUM_DENSE + 1; w < PH_WORDS; ++w) hdr[w] = 0;
+    hdr[PH_NUM_SCATTERED] = counters[8];
+    for (int w = PH_NUM_SCATTERED + 1; w < PH_WORDS; ++w) hdr[w] = 0;
     if (counters[1] > 0) {
       mint::report(p.status, MINT_ERR_NOT_RESIDENT, counters[2]);
       if (p.status) atomicAdd(&p.status[1], counters[1]);
