@@ -1,8 +1,8 @@
 """Tensor-parallel and expert-parallel placement of the LoRA apply (host side).
 
-The paper places LoRA tensors with the base weights they modify ("Scale Up":
-"LoRA tensors follow the tensor-parallel shards for the dense weights they
-modify", per-expert LoRA tensors are keyed by expert id and live with their
+The paper places LoRA tensors with the base weights they modify (section
+"Scale Up": an adapter's tensors are sharded like the dense weights they
+belong to; per-expert LoRA tensors are keyed by expert id and live with their
 expert).  For one projection d -> n over `world` ranks that gives three cases:
 
 * column-parallel (q, k, v, gate, up: the base weight is split on its output):
