@@ -244,8 +244,10 @@ class DeviceWorkload:
 
     def groups_idx(self, grouping):
         ncase = len(self.wl["cases"])
-        if self.moe or grouping == "none" or ncase == 1:
+        if grouping == "none" or ncase == 1:
             return [[i] for i in range(ncase)]
+        if self.moe:   # gate and up share the routed pairs and the hidden rows; down reads their product
+            return [[0, 1], [2]] if ncase == 3 else [[i] for i in range(ncase)]
         if grouping == "layer":
             return [list(range(ncase))]
         return STAGES if ncase == 7 else [[i] for i in range(ncase)]
@@ -257,9 +259,15 @@ class DeviceWorkload:
     def enqueue_layer(self, li, grouping):
         mb = self.mb
         if self.moe:
-            for ci, (pool, x, y) in enumerate(self.layers[li]):
-                mb.mint_moe_lora_apply(pool, self.table, self.plan, x, y, self.status, x_row=self.base[ci].x_row,
-                                       workspace=self.workspaces[ci])
+            row = self.layers[li]
+            for g in self.groups_idx(grouping):
+                if len(g) == 1:
+                    ci = g[0]
+                    mb.mint_moe_lora_apply(row[ci][0], self.table, self.plan, row[ci][1], row[ci][2], self.status,
+                                           x_row=self.base[ci].x_row, workspace=self.workspaces[ci])
+                else:
+                    mb.mint_moe_lora_apply_grouped([(row[ci][0], row[ci][1], row[ci][2], self.workspaces[ci]) for ci in g],
+                                                   self.table, self.plan, self.status, x_row=self.base[g[0]].x_row)
             return
         key = (li, grouping)
         if key not in self._groups:

@@ -335,6 +335,28 @@ int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table,
                             int64_t ldy, void *workspace_dev, size_t workspace_bytes,
                             int32_t *status_dev, mint_stream_t stream);
 
+/* Grouped form: up to MINT_MAX_GROUP MoE projections that share the plan, the
+ * row map and the pair weights (the gate and the up projection of an expert
+ * FFN: same routed pairs, same hidden rows) in one pair of launches.  Each item
+ * has its own pool, x, y and workspace (rules as for mint_moe_lora_apply); all
+ * pools hold the same number of experts; items must not alias each other's y.
+ * (Paper, "Scale Up": an adapter's per-expert tensors cover each targeted
+ * expert projection.)                                                        */
+typedef struct {
+  const mint_pool *pool;
+  const void *x_dev;
+  int64_t ldx;
+  void *y_dev;
+  int64_t ldy;
+  void *workspace_dev;
+  size_t workspace_bytes;
+} mint_moe_apply_item;
+int32_t mint_moe_lora_apply_grouped(const mint_moe_apply_item *items, int32_t count,
+                                    const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                    int32_t K, int64_t x_rows, const int32_t *x_row_dev,
+                                    const float *pair_weight_dev, int32_t *status_dev,
+                                    mint_stream_t stream);
+
 /* Router-weighted combine: the MoE expert LoRA update of the projection that ends
  * an expert FFN, summed over a token's routed experts into the token's row
  * (paper, "Scale Up": per-expert LoRA tensors keyed by expert id):

@@ -45,7 +45,7 @@ EXPORTS = [
     "mint_lora_shrink", "mint_lora_expand",
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
     "mint_lora_apply_fused_static", "mint_selftest_wait_timeout",
-    "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply",
+    "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply", "mint_moe_lora_apply_grouped",
     "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
 ]
 
@@ -131,6 +131,7 @@ def load_library() -> ctypes.CDLL:
         "mint_selftest_wait_timeout": (i32, [vp, vp, vp, i32, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
+        "mint_moe_lora_apply_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, i32, i64, vp, vp, vp, vp]),
         "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply_combine": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
     }
@@ -464,6 +465,25 @@ def mint_moe_lora_apply(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tenso
         _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
         _ptr(status), _stream()))
     return y
+
+
+def mint_moe_lora_apply_grouped(items, table: SlotTable, plan: Plan, status: torch.Tensor,
+                                x_row: Optional[torch.Tensor] = None,
+                                pair_weight: Optional[torch.Tensor] = None):
+    """items: (pool, x, y, workspace) per projection (the item record has the layout of the dense one);
+    they share the plan, the row map and the pair weights."""
+    assert 1 <= len(items) <= MINT_MAX_GROUP
+    if x_row is not None:
+        assert x_row.dtype == torch.int32 and x_row.is_contiguous()
+    if pair_weight is not None:
+        assert pair_weight.dtype == torch.float32 and pair_weight.is_contiguous()
+    arr = (ApplyItem * len(items))()
+    for i, (pool, x, y, ws) in enumerate(items):
+        arr[i] = ApplyItem(pool.handle, _ptr(x), x.stride(0), _ptr(y), y.stride(0), _ptr(ws),
+                           ws.numel() * ws.element_size())
+    _check(load_library().mint_moe_lora_apply_grouped(
+        arr, len(items), table.handle, _ptr(plan.blob), plan.T, plan.K, items[0][1].shape[0],
+        _ptr(x_row), _ptr(pair_weight), _ptr(status), _stream()))
 
 
 def mint_moe_lora_apply_combine(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, y: torch.Tensor,

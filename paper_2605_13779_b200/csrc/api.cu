@@ -608,34 +608,32 @@ extern "C" size_t mint_moe_lora_apply_workspace_bytes(const mint_pool *pool, int
                                          pool->desc.r_max);
 }
 
-extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
-                                       int32_t T, int32_t K, const void *x_dev, int64_t ldx, int64_t x_rows,
-                                       const int32_t *x_row_dev, const float *pair_weight_dev, void *y_dev,
-                                       int64_t ldy, void *workspace_dev, size_t workspace_bytes,
-                                       int32_t *status_dev, mint_stream_t stream) {
-  if (!pool || !table || !plan_dev || !status_dev)
-    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: null argument");
-  if (T < 0 || K < 1 || (int64_t)T * K > kMaxItems)
-    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: T=%d K=%d", T, K);
+// Checks one MoE projection's arguments and fills its launch record.
+static int32_t fill_moe(const mint_pool *pool, const mint_slot_table *table, int32_t T, int32_t K, const void *x_dev,
+                        int64_t ldx, int64_t x_rows, const int32_t *x_row_dev, const float *pair_weight_dev,
+                        void *y_dev, int64_t ldy, void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                        const char *who, MoEArgs &a, bool &streamed) {
+  if (!pool) return mint_fail(MINT_ERR_INVALID_ARG, "%s: null pool", who);
   if (pool->desc.layout != MINT_LAYOUT_PACKED_MOE || pool->desc.num_experts < 1)
-    return mint_fail(MINT_ERR_UNSUPPORTED, "moe_apply: needs a packed MoE pool");
+    return mint_fail(MINT_ERR_UNSUPPORTED, "%s: needs a packed MoE pool", who);
   if (pool->desc.num_slots != table->num_slots)
-    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "moe_apply: pool has %d slots, table has %d", pool->desc.num_slots,
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "%s: pool has %d slots, table has %d", who, pool->desc.num_slots,
                      table->num_slots);
   if (table->max_rank > pool->desc.r_max)
-    return mint_fail(MINT_ERR_RANK_TOO_LARGE, "moe_apply: a bound adapter has rank %d > pool r_max %d",
+    return mint_fail(MINT_ERR_RANK_TOO_LARGE, "%s: a bound adapter has rank %d > pool r_max %d", who,
                      table->max_rank, pool->desc.r_max);
+  streamed = false;
   if (T == 0) return MINT_OK;
   int32_t st;
-  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "moe_apply"))) return st;
-  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", "moe_apply"))) return st;
-  if (x_rows < 1) return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: x_rows=%lld", (long long)x_rows);
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", who))) return st;
+  if ((st = check_act(y_dev, ldy, pool->desc.n, "y_dev", who))) return st;
+  if (x_rows < 1) return mint_fail(MINT_ERR_INVALID_ARG, "%s: x_rows=%lld", who, (long long)x_rows);
   if (!x_row_dev && x_rows < (int64_t)T * K)
-    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "moe_apply: identity rows need x_rows >= T*K");
+    return mint_fail(MINT_ERR_SHAPE_MISMATCH, "%s: identity rows need x_rows >= T*K", who);
   const size_t need = mint_moe_lora_apply_workspace_bytes(pool, T, K);
   if (need > 0 && (!workspace_dev || workspace_bytes < need))
-    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "moe_apply: workspace %zu < %zu", workspace_bytes, need);
-  MoEArgs a = {};
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu", who, workspace_bytes, need);
+  a = MoEArgs{};
   a.A = static_cast<const uint16_t *>(pool->desc.A_dev);
   a.B = static_cast<const uint16_t *>(pool->desc.B_dev);
   a.d = pool->desc.d;
@@ -653,10 +651,62 @@ extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_ta
   a.y = static_cast<uint16_t *>(y_dev);
   a.ldy = ldy;
   a.status = status_dev;
-  if (need > 0 && mint_stream_moe_supported(pool->desc.r_max, table->max_rank)) {
-    if ((reinterpret_cast<uintptr_t>(workspace_dev) & 15) != 0)
-      return mint_fail(MINT_ERR_MISALIGNED, "moe_apply: workspace_dev must be 16-byte aligned");
-    return mint_launch_stream_moe(a, table_dev(table), plan_dev, workspace_dev, static_cast<cudaStream_t>(stream));
+  streamed = need > 0 && mint_stream_moe_supported(pool->desc.r_max, table->max_rank);
+  if (streamed && (reinterpret_cast<uintptr_t>(workspace_dev) & 15) != 0)
+    return mint_fail(MINT_ERR_MISALIGNED, "%s: workspace_dev must be 16-byte aligned", who);
+  return MINT_OK;
+}
+
+extern "C" int32_t mint_moe_lora_apply(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                       int32_t T, int32_t K, const void *x_dev, int64_t ldx, int64_t x_rows,
+                                       const int32_t *x_row_dev, const float *pair_weight_dev, void *y_dev,
+                                       int64_t ldy, void *workspace_dev, size_t workspace_bytes,
+                                       int32_t *status_dev, mint_stream_t stream) {
+  mint_moe_apply_item it;
+  it.pool = pool;
+  it.x_dev = x_dev;
+  it.ldx = ldx;
+  it.y_dev = y_dev;
+  it.ldy = ldy;
+  it.workspace_dev = workspace_dev;
+  it.workspace_bytes = workspace_bytes;
+  return mint_moe_lora_apply_grouped(&it, 1, table, plan_dev, T, K, x_rows, x_row_dev, pair_weight_dev, status_dev,
+                                     stream);
+}
+
+extern "C" int32_t mint_moe_lora_apply_grouped(const mint_moe_apply_item *items, int32_t count,
+                                               const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                               int32_t K, int64_t x_rows, const int32_t *x_row_dev,
+                                               const float *pair_weight_dev, int32_t *status_dev,
+                                               mint_stream_t stream) {
+  if (!items || count < 1 || count > MINT_MAX_GROUP)
+    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: count=%d (1..%d)", count, MINT_MAX_GROUP);
+  if (!table || !plan_dev || !status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: null argument");
+  if (T < 0 || K < 1 || (int64_t)T * K > kMaxItems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "moe_apply: T=%d K=%d", T, K);
+  MoEArgs args[MINT_MAX_GROUP];
+  void *ws[MINT_MAX_GROUP];
+  bool streamed[MINT_MAX_GROUP];
+  bool all_streamed = true;
+  for (int i = 0; i < count; ++i) {
+    const mint_moe_apply_item &it = items[i];
+    int32_t st = fill_moe(it.pool, table, T, K, it.x_dev, it.ldx, x_rows, x_row_dev, pair_weight_dev, it.y_dev,
+                          it.ldy, it.workspace_dev, it.workspace_bytes, status_dev, "moe_apply", args[i], streamed[i]);
+    if (st) return st;
+    if (it.pool->desc.num_experts != items[0].pool->desc.num_experts)
+      return mint_fail(MINT_ERR_SHAPE_MISMATCH, "moe_apply: the pools of a grouped call hold %d and %d experts",
+                       items[0].pool->desc.num_experts, it.pool->desc.num_experts);
+    ws[i] = it.workspace_dev;
+    all_streamed = all_streamed && streamed[i];
   }
-  return mint_launch_moe(a, table_dev(table), plan_dev, static_cast<cudaStream_t>(stream));
+  if (T == 0) return MINT_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (all_streamed) return mint_launch_stream_moe(args, count, table_dev(table), plan_dev, ws, s);
+  // a pool the streamed kernels do not take: one call per projection
+  for (int i = 0; i < count; ++i) {
+    int32_t st = streamed[i] ? mint_launch_stream_moe(&args[i], 1, table_dev(table), plan_dev, &ws[i], s)
+                             : mint_launch_moe(args[i], table_dev(table), plan_dev, s);
+    if (st) return st;
+  }
+  return MINT_OK;
 }

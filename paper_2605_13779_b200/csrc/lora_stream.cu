@@ -1257,38 +1257,50 @@ static int32_t stream_kernel_attributes() {
 // MoE expert LoRA apply on the streamed kernels: the plan's items are the
 // (token, k) pairs grouped by (expert, slot); the weight block of a tile is
 // (slot, expert); the shrink reads row x_row[p] of x, the expand updates row p of y.
-int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, void *workspace,
-                               cudaStream_t s) {
+int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                               void *const *workspaces, cudaStream_t s) {
+  if (nprob < 1 || nprob > kMaxProblems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "grouped MoE apply: 1..%d problems", kMaxProblems);
   int32_t lanes = 0;
   int32_t st = mint_device_lanes(&lanes);
   if (st) return st;
   if ((st = stream_kernel_attributes())) return st;
-  const int64_t pairs = (int64_t)a.T * a.K;
-  const int64_t key_space = (int64_t)tab.num_slots * a.num_experts;
+  const MoEArgs &a0 = args[0];
+  const int64_t pairs = (int64_t)a0.T * a0.K;
+  const int64_t key_space = (int64_t)tab.num_slots * a0.num_experts;
   const int64_t tiles = mint_tile_upper_bound(1, pairs, key_space);
   if (tiles == 0) return MINT_OK;
   StreamParams P = {};
-  StreamProblem &pb = P.prob[0];
-  pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
-  pb.ldx = a.ldx; pb.ldy = a.ldy;
-  pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
-  pb.cb0_shrink = kShrinkPieceBlocks;
-  pb.cb0_expand = kExpandPieceBlocks;
-  pb.ws_part = static_cast<float *>(workspace);
-  P.nprob = 1;
-  P.T = a.T;
-  P.K = a.K;
-  P.num_experts = a.num_experts;
-  P.weights_per_slot = a.num_experts;
-  P.x_row = a.x_row;
-  P.pair_weight = a.pair_weight;
-  P.x_rows = a.x_rows;
+  int cb_s = 0, cb_e = 0, cb_widest = 0;
+  for (int i = 0; i < nprob; ++i) {
+    const MoEArgs &a = args[i];
+    StreamProblem &pb = P.prob[i];
+    pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
+    pb.ldx = a.ldx; pb.ldy = a.ldy;
+    pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
+    cb_s += kShrinkPieceBlocks;
+    cb_e += kExpandPieceBlocks;
+    pb.cb0_shrink = cb_s;
+    pb.cb0_expand = cb_e;
+    cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
+    cb_widest = std::max(cb_widest, kShrinkPieceBlocks + (a.d + kShrinkBlock - 1) / kShrinkBlock);
+    cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
+    pb.ws_part = static_cast<float *>(workspaces[i]);
+  }
+  P.nprob = nprob;
+  P.T = a0.T;
+  P.K = a0.K;
+  P.num_experts = a0.num_experts;
+  P.weights_per_slot = a0.num_experts;
+  P.x_row = a0.x_row;
+  P.pair_weight = a0.pair_weight;
+  P.x_rows = a0.x_rows;
   P.lanes = lanes;
-  P.cb_shrink = kShrinkPieceBlocks + (a.d + kShrinkBlock - 1) / kShrinkBlock;
-  P.cb_expand = kExpandPieceBlocks + (a.n + kExpandBlock - 1) / kExpandBlock;
-  P.cb_shrink_widest = P.cb_shrink;
+  P.cb_shrink = cb_s;
+  P.cb_expand = cb_e;
+  P.cb_shrink_widest = cb_widest;
   P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
-  P.status = a.status;
+  P.status = a0.status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, pairs, key_space);
 
@@ -1301,7 +1313,6 @@ int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void
   cfg.dynamicSmemBytes = kRingsBytes;
   cfg.stream = s;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
   // the first apply after a plan or a bind waits for that kernel in full: it reads the plan at once
   cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
   st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<true>, P), "shrink_stream (packed) launch");

@@ -257,8 +257,9 @@ struct MoEArgs {
   int32_t *status;
 };
 int32_t mint_launch_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, cudaStream_t s);
-int32_t mint_launch_stream_moe(const MoEArgs &a, const TableDev &tab, const void *plan_dev, void *workspace,
-                               cudaStream_t s);
+// nprob problems that share the plan, the row map and the pair weights (args[0]'s are used)
+int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                               void *const *workspaces, cudaStream_t s);
 
 int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
                                float *slot_scale, int32_t num_slots, cudaStream_t s);

@@ -188,3 +188,54 @@ def test_combine_is_deterministic():
     a, _ = run_combine(case, y0)
     b, _ = run_combine(case, y0)
     np.testing.assert_array_equal(a, b)
+
+
+# ---- grouped call: several projections over the same routed pairs in one launch pair ----
+def run_moe_grouped(cases, weighted, y0_zero=False):
+    from paper_2605_13779_b200 import binding as mb, harness
+    table = harness.upload_table(cases[0].table)
+    devs = [harness.upload_moe(c, table=table) for c in cases]
+    if y0_zero:
+        for dv in devs:
+            dv.y.zero_()
+    d0 = devs[0]
+    plan = mb.mint_lora_plan(table, d0.ids, d0.status, expert_ids=d0.expert_ids, num_experts=cases[0].E)
+    ws = [mb.new_moe_workspace(dv.pool, plan.T, plan.K) for dv in devs]
+    for w in ws:
+        w.fill_(0xFF)   # the workspace needs no initialisation
+    mb.mint_moe_lora_apply_grouped([(dv.pool, dv.x, dv.y, w) for dv, w in zip(devs, ws)], table, plan, d0.status,
+                                   x_row=d0.x_row, pair_weight=d0.pair_weight if weighted else None)
+    torch.cuda.synchronize()
+    return [harness.y_to_f64(dv.y) for dv in devs], d0.status.cpu().numpy()
+
+
+def check_grouped(cases, what):
+    for weighted, y0_zero in ((False, False), (True, False), (False, True)):
+        ys, status = run_moe_grouped(cases, weighted, y0_zero)
+        assert status[0] == 0, status
+        for c, y in zip(cases, ys):
+            y_ref, _ = parity.oracle_moe(c, weighted=weighted, y0=np.zeros_like(c.y0) if y0_zero else None)
+            parity.assert_close(y, y_ref, f"{what} {c.name} weighted={weighted} y0_zero={y0_zero}")
+
+
+@pytest.mark.parametrize("T", [512, 4096])
+def test_config4_gate_and_up_in_one_call(T):
+    """Gate and up read the same hidden rows for the same routed pairs: one grouped call, as
+    the benchmark issues it."""
+    batch = synth.config4_batch(T=T)
+    cases = [synth.config4_projection(batch, "gate"), synth.config4_projection(batch, "up")]
+    assert not np.array_equal(cases[0].A, cases[1].A)
+    check_grouped(cases, f"config4/gate+up/T{T}")
+
+
+def test_grouped_moe_projections_of_different_widths():
+    tag = "gpu/moe/grouped"
+    batch = synth.config4_batch(T=96, E=8, K=2, num_slots=3, rank=8, p_none=0.1, tag=tag)
+    cases = [synth.config4_projection(batch, "gate", d=520, n=264, tag=tag),
+             synth.config4_projection(batch, "up", d=520, n=1024, tag=tag),
+             synth.config4_projection(batch, "gate", d=520, n=72, tag=tag + "/third")]
+    check_grouped(cases, tag)
+    none = np.repeat(batch.ids < 0, batch.K)
+    ys, _ = run_moe_grouped(cases, weighted=True)
+    for c, y in zip(cases, ys):
+        np.testing.assert_array_equal(y[none], synth.bf16_bits_to_f64(c.y0)[none])
