@@ -229,6 +229,8 @@ class DeviceWorkload:
                     pool = mb.Pool(A, B, dv.pool.d, dv.pool.n, dv.pool.r_max, dv.pool.num_slots,
                                    num_experts=dv.pool.num_experts)
                     row.append((pool, dv.x.clone(), dv.y.clone()))
+            if self.moe and len(row) == 3 and np.array_equal(wl["cases"][0].x, wl["cases"][1].x):
+                row[1] = (row[1][0], row[0][1], row[1][2])   # gate and up read the same hidden states
             self.layers.append(row)
         self.ids = self.base[0].ids
         self.status = mb.new_status()

@@ -102,6 +102,8 @@ struct StreamProblem {
   int64_t ldx, ldy;
   int32_t d, n, r_max;
   int32_t cb0_shrink, cb0_expand;  // first virtual column block of this problem
+  int32_t dual;        // packed MoE pools: 1: the shrink pieces of this problem also shrink the next one, which
+                       // reads the same x (gate and up); 2: this problem's v comes from the previous one's pieces
   float *ws_part;      // slots of 32 * r_max floats: slot (tile + lane): that lane's sum, [len][rank] packed;
                        // slot (dense_slot0 + s * tiles_ub + tile): part s of the v of a dense segment's tile
 };
@@ -350,6 +352,7 @@ __device__ __forceinline__ void walk_batch(const StreamParams &P, const Area &ar
     pc.rows = sh.rows + (sh.desc[ti].off - sh.desc[0].off);
     for (int p = 0; p < P.nprob; ++p) {
       const StreamProblem &pb = P.prob[p];
+      if (!kExpand && pb.dual == 2) continue;   // shrunk together with the problem before it
       const int width = kExpand ? pb.n : pb.d;
       const int first = kExpand ? pb.cb0_expand : pb.cb0_shrink;
       const int count = (width + kBlock - 1) / kBlock;
@@ -479,17 +482,22 @@ __device__ __forceinline__ void shrink_mma(const StreamProblem &pb, const Piece 
 // of the block, the same permutation of k that the x fragments use.  A pass covers
 // min(RG, 4) rank groups from rank rh on; segments of rank groups at or beyond
 // the slot's rank are not read.
-template <int XG, int RG>
+// kDual (RG <= 2): the rank groups of a second pool with the same shape follow those of the
+// first (pb2: same x, same d and r_max), so that one pass over x shrinks both.
+template <int XG, int RG, bool kDual = false>
 __device__ __forceinline__ void shrink_mma_packed(const StreamProblem &pb, const Piece &pc, int rh,
-                                                  uint32_t ring_base, float *scratch) {
+                                                  uint32_t ring_base, float *scratch,
+                                                  const StreamProblem *pb2 = nullptr) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  constexpr int NT = RG < 4 ? RG : 4;
+  constexpr int NT = kDual ? 2 * RG : (RG < 4 ? RG : 4);
+  static_assert(!kDual || RG <= 2, "two pools share a pass only up to 16 ranks each");
   constexpr int N = XG + NT;
   constexpr int MT = (XG + 1) / 2;
   Ring<N> ring{ring_base};
   const uint32_t warp_base = ring_base - (uint32_t)lane * 16;
   const uint16_t *A_w = pb.A + (int64_t)pc.slot * pb.d * pb.r_max;
+  const uint16_t *A_w2 = kDual ? pb2->A + (int64_t)pc.slot * pb.d * pb.r_max : nullptr;
   const uint16_t *xsrc[XG];
 #pragma unroll
   for (int i = 0; i < XG; ++i) {
@@ -500,9 +508,12 @@ __device__ __forceinline__ void shrink_mma_packed(const StreamProblem &pb, const
   // this lane's segment of every 512-byte slot of a block of A: where it comes from, where it goes
   int a_off[NT], a_k[NT];
   uint32_t a_dst[NT];
+  bool a_second[NT];
 #pragma unroll
   for (int j = 0; j < NT; ++j) {
-    const int c = j * 32 + lane, k = c / NT, rgl = c % NT, rg = (rh >> 3) + rgl;
+    const int c = j * 32 + lane, k = c / NT, rgl = c % NT;
+    const int rg = kDual ? rgl % RG : (rh >> 3) + rgl;   // rank group inside its pool
+    a_second[j] = kDual && rgl >= RG;
     a_off[j] = k * pb.r_max + rg * 8;
     a_k[j] = rg * 8 < pc.r ? k : (1 << 30);
     const int m = (((k >> 2) & 1) * 2 + ((k >> 1) & 1)) * NT + rgl, jj = 2 * (k >> 3) + (k & 1);
@@ -540,11 +551,12 @@ __device__ __forceinline__ void shrink_mma_packed(const StreamProblem &pb, const
 #pragma unroll
       for (int i = 0; i < XG; ++i) cp_async16(ring.slot(it, i), xsrc[i] ? xsrc[i] + col : pb.A, ok && xsrc[i]);
       const uint16_t *blk = A_w + (int64_t)col * pb.r_max;
+      const uint16_t *blk2 = kDual ? A_w2 + (int64_t)col * pb.r_max : nullptr;
       const uint32_t dst = a_region(it);
 #pragma unroll
       for (int j = 0; j < NT; ++j) {
         const bool ok_a = col + a_k[j] < pb.d;
-        cp_async16(dst + a_dst[j], ok_a ? blk + a_off[j] : pb.A, ok_a);
+        cp_async16(dst + a_dst[j], ok_a ? ((kDual && a_second[j]) ? blk2 : blk) + a_off[j] : pb.A, ok_a);
       }
     }
     cp_async_commit();
@@ -662,6 +674,30 @@ __device__ __forceinline__ void shrink_piece(const StreamParams &P, SmemShrink &
   // the sum over this lane's columns; the expand adds the lanes of a tile in lane order
   float *dst = pb.ws_part + (size_t)(pc.t + blockIdx.x) * slot_floats;
   const bool vec = !kPacked && pc.r == 1 && pc.len <= 8;
+  if (kPacked && pb.dual == 1) {
+    // this problem and the next one (same x, same shape, at most 16 ranks) in one pass over x
+    const StreamProblem &pb2 = P.prob[pc.p + 1];
+    const int rg = pb.r_max >> 3;
+#define MINT_SHRINK_CASE(XG)                                                                    \
+  if (rg == 1) shrink_mma_packed<XG, 1, true>(pb, pc, 0, ring_base, S.scratch, &pb2);          \
+  else shrink_mma_packed<XG, 2, true>(pb, pc, 0, ring_base, S.scratch, &pb2)
+    if (pc.len <= 16) { MINT_SHRINK_CASE(2); }
+    else { MINT_SHRINK_CASE(4); }
+#undef MINT_SHRINK_CASE
+    __syncthreads();
+    float *dst2 = pb2.ws_part + (size_t)(pc.t + blockIdx.x) * slot_floats;
+    for (int i = tid; i < 2 * pc.len * pc.r; i += kThreads) {
+      const int second = i >= pc.len * pc.r, e = second ? i - pc.len * pc.r : i;
+      const int l = e / pc.r, j = e - l * pc.r;
+      const int mt = l >> 4, g = l & 15, nt = second * rg + (j >> 3), cc = j & 7;
+      const int frag = ((g & 7) * 4 + (cc >> 1)) * 4 + (g >> 3) * 2 + (cc & 1);
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) s += S.scratch[((w * 2 + mt) * 4 + nt) * 128 + frag];
+      (second ? dst2 : dst)[l * pc.r + j] = s;
+    }
+    return;
+  }
   for (int rh = 0; rh < pc.r; rh += 32) {
     const int rr = min(32, pc.r - rh);
     // (the bodies wait, right before they write the scratch, until the previous gather has read it)
@@ -1278,14 +1314,27 @@ int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &t
     pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
     pb.ldx = a.ldx; pb.ldy = a.ldy;
     pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
-    cb_s += kShrinkPieceBlocks;
+    pb.ws_part = static_cast<float *>(workspaces[i]);
     cb_e += kExpandPieceBlocks;
-    pb.cb0_shrink = cb_s;
     pb.cb0_expand = cb_e;
+    cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
+    // Two consecutive projections that read the same x through pools of the same shape and at most 16
+    // ranks (gate and up) are shrunk in one pass over x: the second takes no columns of the shrink's
+    // area and finds its parts where the first one's are.
+    const bool follows = i > 0 && P.prob[i - 1].dual == 1;
+    if (follows) {
+      pb.dual = 2;
+      pb.cb0_shrink = P.prob[i - 1].cb0_shrink;
+      continue;
+    }
+    cb_s += kShrinkPieceBlocks;
+    pb.cb0_shrink = cb_s;
     cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
     cb_widest = std::max(cb_widest, kShrinkPieceBlocks + (a.d + kShrinkBlock - 1) / kShrinkBlock);
-    cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
-    pb.ws_part = static_cast<float *>(workspaces[i]);
+    if (i + 1 < nprob) {
+      const MoEArgs &b = args[i + 1];
+      if (b.x == a.x && b.ldx == a.ldx && b.d == a.d && b.r_max == a.r_max && a.r_max <= 16) pb.dual = 1;
+    }
   }
   P.nprob = nprob;
   P.T = a0.T;

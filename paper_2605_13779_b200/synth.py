@@ -368,8 +368,8 @@ def config4_batch(T: int = 4096, E: int = 128, K: int = 8, num_slots: int = 16, 
 
 def config4_projection(batch: MoEBatch, proj: str, d: Optional[int] = None, n: Optional[int] = None,
                        layer: int = 0, tag: str = "config4") -> MoECase:
-    """gate/up read the token's hidden row (x_row[p] = p // K); down reads the
-    per-pair intermediate row (identity)."""
+    """gate/up read the token's hidden row (x_row[p] = p // K), the same hidden
+    states for both; down reads the per-pair intermediate row (identity)."""
     if d is None or n is None:
         d, n = MOE_30B_PROJECTIONS[proj]
     P = batch.T * batch.K
@@ -378,7 +378,7 @@ def config4_projection(batch: MoEBatch, proj: str, d: Optional[int] = None, n: O
         x = normal_bf16(stream(tag, proj, layer, "x"), (P, d), 1.0)
         x_row = None
     else:
-        x = normal_bf16(stream(tag, proj, layer, "x"), (batch.T, d), 1.0)
+        x = normal_bf16(stream(tag, "gate", layer, "x"), (batch.T, d), 1.0)
         x_row = (np.arange(P, dtype=np.int64) // batch.K).astype(np.int32)
     y0 = normal_bf16(stream(tag, proj, layer, "y0"), (P, n), 1.0)
     return MoECase(f"{tag}/{proj}/L{layer}", batch.T, batch.K, batch.E, d, n, batch.r_max,

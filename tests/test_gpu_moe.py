@@ -195,6 +195,9 @@ def run_moe_grouped(cases, weighted, y0_zero=False):
     from paper_2605_13779_b200 import binding as mb, harness
     table = harness.upload_table(cases[0].table)
     devs = [harness.upload_moe(c, table=table) for c in cases]
+    for i in range(1, len(cases)):   # projections with the same hidden states read one tensor
+        if cases[i].x.shape == cases[i - 1].x.shape and np.array_equal(cases[i].x, cases[i - 1].x):
+            devs[i].x = devs[i - 1].x
     if y0_zero:
         for dv in devs:
             dv.y.zero_()
@@ -224,7 +227,7 @@ def test_config4_gate_and_up_in_one_call(T):
     the benchmark issues it."""
     batch = synth.config4_batch(T=T)
     cases = [synth.config4_projection(batch, "gate"), synth.config4_projection(batch, "up")]
-    assert not np.array_equal(cases[0].A, cases[1].A)
+    assert not np.array_equal(cases[0].A, cases[1].A) and np.array_equal(cases[0].x, cases[1].x)
     check_grouped(cases, f"config4/gate+up/T{T}")
 
 
@@ -239,3 +242,17 @@ def test_grouped_moe_projections_of_different_widths():
     ys, _ = run_moe_grouped(cases, weighted=True)
     for c, y in zip(cases, ys):
         np.testing.assert_array_equal(y[none], synth.bf16_bits_to_f64(c.y0)[none])
+
+
+@pytest.mark.parametrize("r_max,ranks", [(16, [16, 1, 9, 8]), (8, [8, 2, 5]), (32, [32, 3, 17])])
+def test_grouped_gate_and_up_share_x_with_mixed_ranks(r_max, ranks):
+    """Gate and up over the same hidden states with slots of different ranks in NaN-padded pools:
+    pools of at most 16 ranks take one pass over x for both, wider ones one pass each."""
+    import dataclasses
+    tag = f"gpu/moe/grouped-mixed/{r_max}"
+    S = len(ranks)
+    batch = synth.config4_batch(T=160, E=4, K=2, num_slots=S, rank=r_max, p_none=0.05, tag=tag)
+    batch = dataclasses.replace(batch, table=synth.identity_table(S, np.asarray(ranks, dtype=np.int32), 2.0))
+    cases = [synth.config4_projection(batch, "gate", d=520, n=264, tag=tag),
+             synth.config4_projection(batch, "up", d=520, n=136, tag=tag)]
+    check_grouped(cases, tag)
