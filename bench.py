@@ -229,8 +229,10 @@ class DeviceWorkload:
                     pool = mb.Pool(A, B, dv.pool.d, dv.pool.n, dv.pool.r_max, dv.pool.num_slots,
                                    num_experts=dv.pool.num_experts)
                     row.append((pool, dv.x.clone(), dv.y.clone()))
-            if self.moe and len(row) == 3 and np.array_equal(wl["cases"][0].x, wl["cases"][1].x):
-                row[1] = (row[1][0], row[0][1], row[1][2])   # gate and up read the same hidden states
+            for i in range(1, len(row)):   # projections with the same input (q, k, v; gate, up) read one tensor
+                ca, cb = wl["cases"][i - 1], wl["cases"][i]
+                if ca.x.shape == cb.x.shape and np.array_equal(ca.x, cb.x):
+                    row[i] = (row[i][0], row[i - 1][1], row[i][2])
             self.layers.append(row)
         self.ids = self.base[0].ids
         self.status = mb.new_status()

@@ -20,6 +20,9 @@ def run_grouped(cases, groups, y0_zero=False, repeat=1):
     from paper_2605_13779_b200 import binding as mb, harness
     table = harness.upload_table(cases[0].table)
     devs = [harness.upload_dense(c, table=table) for c in cases]
+    for i in range(1, len(cases)):   # projections with the same input read one tensor
+        if cases[i].x.shape == cases[i - 1].x.shape and np.array_equal(cases[i].x, cases[i - 1].x):
+            devs[i].x = devs[i - 1].x
     if y0_zero:
         for dv in devs:
             dv.y.zero_()
@@ -77,14 +80,16 @@ def test_config2_layer_call_with_tokens_without_adapter():
     check_groups(cases, [list(range(7))], "layer call with none")
 
 
-def equal_width_cases(count, T, rank, d=2560, n=64, num_slots=1, tag="gpu/equal"):
-    table = synth.identity_table(num_slots, np.full(num_slots, rank, dtype=np.int32), 2.0)
+def equal_width_cases(count, T, rank, d=2560, n=64, num_slots=1, tag="gpu/equal", same_x=1, ranks=None):
+    """same_x: runs of that many consecutive projections read the same x."""
+    ranks = np.full(num_slots, rank, dtype=np.int32) if ranks is None else np.asarray(ranks, dtype=np.int32)
+    table = synth.identity_table(num_slots, ranks, 2.0)
     ids = (np.arange(T) % num_slots).astype(np.int64)
     cases = []
     for i in range(count):
         name = f"{tag}/{count}/{T}/{rank}/{i}"
         A, B = synth.dense_pool(synth.stream(name, "pool"), table, rank, d, n)
-        x = synth.normal_bf16(synth.stream(name, "x"), (T, d), 1.0)
+        x = synth.normal_bf16(synth.stream(f"{tag}/{count}/{T}/{rank}/{i // same_x}", "x"), (T, d), 1.0)
         y0 = synth.normal_bf16(synth.stream(name, "y0"), (T, n), 1.0)
         cases.append(synth.DenseCase(name, T, d, n, rank, table, ids, A, B, x, y0))
     return cases
@@ -114,3 +119,18 @@ def test_grouped_call_twice_on_one_workspace():
         y_ref, _, _ = parity.oracle_dense(c)
         delta = y_ref - synth.bf16_bits_to_f64(c.y0)
         assert np.abs(y - (y_ref + delta)).max() <= 6e-2
+
+
+@pytest.mark.parametrize("count,same_x,T,num_slots,ranks,r_max", [
+    (3, 3, 40, 4, [8, 1, 16, 32], 32),      # q, k, v: three pools, one x
+    (2, 2, 33, 3, [16, 5, 1], 16),          # gate, up
+    (5, 2, 70, 5, [32, 8, 1, 16, 3], 32),   # pairs, then one projection on its own
+    (7, 3, 16, 2, [1, 1], 8),               # rank 1 only: the FMA path of every member
+    (8, 4, 50, 3, [8, 16, 2], 16),          # runs of four: groups of three and one
+])
+def test_projections_that_read_the_same_x(count, same_x, T, num_slots, ranks, r_max):
+    """Items of a grouped call may read the same x tensor (q, k, v; gate, up)."""
+    cases = equal_width_cases(count, T, r_max, d=1032, n=264, num_slots=num_slots, tag="gpu/same-x",
+                              same_x=same_x, ranks=ranks)
+    check_groups(cases, [list(range(count))], f"same x: {count} items in runs of {same_x}")
+
