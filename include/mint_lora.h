@@ -317,6 +317,32 @@ int32_t mint_lora_apply_fused_grouped(const mint_apply_item *items, int32_t coun
                                       const mint_slot_table *table, const void *plan_dev, int32_t T,
                                       int32_t *status_dev, mint_stream_t stream);
 
+/* ---- LoRA backward over padded slots (dense projections) --------------------
+ * The derivative of the update the fused apply performs, for the paper's
+ * time-sliced training over a shared frozen base ("Time-Sliced Multi-LoRA
+ * Training": adapter slots of a configured maximum shape, smaller ranks padded
+ * and masked; kernels that update several adapters in one batch are the
+ * alternative it names).  With A: rank x d and B: rank x n of the token's slot,
+ * u = dy . B^T and v = x . A^T:
+ *   dx[t, :]        += s * u[t, :] . A                      bf16 [T][lddx], one RNE store
+ *   dA[slot][k, :]  += s * sum over the slot's tokens of u[t, k] * x[t, :]
+ *   dB[slot][k, :]  += s * sum over the slot's tokens of v[t, k] * dy[t, :]
+ * dA_dev / dB_dev: fp32, device, shaped like the pool's tensors
+ * ([num_slots][r_max][d], [num_slots][r_max][n]), caller-owned, accumulated
+ * into; rows k >= rank of a slot and slots without tokens are not touched.
+ * Tokens with id -1 (or not resident) contribute nothing and keep their dx row
+ * bit for bit.  dx_dev may be NULL (no input gradient wanted); dA_dev and dB_dev
+ * may both be NULL (frozen adapters).  The sums run in the plan's token order in
+ * fp32: bit-identical from run to run.  x_dev [T][ldx] and dy_dev [T][lddy] are
+ * bf16; plan_dev, workspace rules and errors as for mint_lora_apply_fused, with
+ * mint_lora_backward_workspace_bytes.  Rank-major pools only.                 */
+size_t mint_lora_backward_workspace_bytes(const mint_pool *pool, int32_t T);
+int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                           int32_t T, const void *x_dev, int64_t ldx, const void *dy_dev, int64_t lddy,
+                           void *dx_dev, int64_t lddx, float *dA_dev, float *dB_dev,
+                           void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                           mint_stream_t stream);
+
 /* ---- MoE expert LoRA apply -------------------------------------------------
  * Per-expert LoRA tensors keyed by expert id (paper, "Scale Up", Megatron
  * placement), in the packed layout.  For pair p = t*K + k with expert e and

@@ -45,6 +45,7 @@ EXPORTS = [
     "mint_lora_shrink", "mint_lora_expand",
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
     "mint_lora_apply_fused_static", "mint_selftest_wait_timeout",
+    "mint_lora_backward_workspace_bytes", "mint_lora_backward",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply", "mint_moe_lora_apply_grouped",
     "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
 ]
@@ -130,6 +131,8 @@ def load_library() -> ctypes.CDLL:
         "mint_lora_apply_fused_static": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, vp]),
         "mint_selftest_wait_timeout": (i32, [vp, vp, vp, i32, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
+        "mint_lora_backward_workspace_bytes": (sz, [vp, i32]),
+        "mint_lora_backward": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, i64, vp, vp, vp, sz, vp, vp]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, i32, i64, vp, vp, vp, vp]),
         "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
@@ -437,6 +440,27 @@ class ApplyGroup:
 def mint_lora_apply_fused_grouped(group: ApplyGroup, table: SlotTable, plan: Plan, status: torch.Tensor):
     _check(load_library().mint_lora_apply_fused_grouped(group.array, group.count, table.handle,
                                                         _ptr(plan.blob), plan.T, _ptr(status), _stream()))
+
+
+def new_backward_workspace(pool: Pool, T: int, device="cuda") -> torch.Tensor:
+    """Workspace of the backward for one projection; it needs no initialisation."""
+    nbytes = max(256, int(load_library().mint_lora_backward_workspace_bytes(pool.handle, T)))
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def mint_lora_backward(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, dy: torch.Tensor,
+                       status: torch.Tensor, dx: Optional[torch.Tensor] = None,
+                       dA: Optional[torch.Tensor] = None, dB: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None):
+    """dx (bf16 [T, d]) and dA / dB (fp32, shaped like the pool's tensors) are accumulated into."""
+    for g in (dA, dB):
+        assert g is None or (g.dtype == torch.float32 and g.is_contiguous())
+    if workspace is None:
+        workspace = new_backward_workspace(pool, plan.T, device=x.device)
+    _check(load_library().mint_lora_backward(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(dy), _ld(dy, pool.n),
+        _ptr(dx), _ld(dx, pool.d) if dx is not None else 0, _ptr(dA), _ptr(dB), _ptr(workspace),
+        workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
 
 
 def mint_moe_lora_apply_workspace_bytes(pool: Pool, T: int, K: int) -> int:

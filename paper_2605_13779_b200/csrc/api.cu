@@ -598,6 +598,75 @@ extern "C" int32_t mint_selftest_wait_timeout(const mint_pool *pool, const mint_
 }
 
 // ---------------------------------------------------------------------------
+// backward
+// ---------------------------------------------------------------------------
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// The pool with A and B in each other's place: B's rows (rank rows of n elements) are what the shrink
+// wants of A, A's rows what the expand wants of B, so the forward kernels compute dy . B^T and (.) . A.
+static mint_pool transposed_pool(const mint_pool *pool) {
+  mint_pool t = *pool;
+  t.desc.A_dev = pool->desc.B_dev;
+  t.desc.B_dev = pool->desc.A_dev;
+  t.desc.d = pool->desc.n;
+  t.desc.n = pool->desc.d;
+  return t;
+}
+
+extern "C" size_t mint_lora_backward_workspace_bytes(const mint_pool *pool, int32_t T) {
+  if (!pool || T < 0) return 0;
+  const mint_pool tp = transposed_pool(pool);
+  return 2 * align256((size_t)T * pool->desc.r_max * sizeof(float)) + mint_lora_apply_workspace_bytes(&tp, T);
+}
+
+extern "C" int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                      int32_t T, const void *x_dev, int64_t ldx, const void *dy_dev, int64_t lddy,
+                                      void *dx_dev, int64_t lddx, float *dA_dev, float *dB_dev,
+                                      void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
+                                      mint_stream_t stream) {
+  int32_t st = check_dense(pool, table, plan_dev, T, "backward");
+  if (st) return st;
+  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "backward: null status_dev");
+  if (T == 0) return MINT_OK;
+  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "backward"))) return st;
+  if ((st = check_act(dy_dev, lddy, pool->desc.n, "dy_dev", "backward"))) return st;
+  if (dx_dev && (st = check_act(dx_dev, lddx, pool->desc.d, "dx_dev", "backward"))) return st;
+  if ((dA_dev == nullptr) != (dB_dev == nullptr))
+    return mint_fail(MINT_ERR_INVALID_ARG, "backward: dA_dev and dB_dev come together (both or neither)");
+  if ((dA_dev && !aligned16(dA_dev)) || (dB_dev && !aligned16(dB_dev)))
+    return mint_fail(MINT_ERR_MISALIGNED, "backward: dA_dev and dB_dev must be 16-byte aligned");
+  if ((pool->desc.d & 7) || (pool->desc.n & 7))
+    return mint_fail(MINT_ERR_UNSUPPORTED, "backward: d and n must be multiples of 8");
+  const size_t need = mint_lora_backward_workspace_bytes(pool, T);
+  if (!workspace_dev || workspace_bytes < need)
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "backward: workspace %zu < %zu", workspace_bytes, need);
+  if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u)
+    return mint_fail(MINT_ERR_MISALIGNED, "backward: workspace must be 256-byte aligned");
+  const mint_pool tp = transposed_pool(pool);
+  const size_t vbytes = align256((size_t)T * pool->desc.r_max * sizeof(float));
+  char *ws = static_cast<char *>(workspace_dev);
+  float *u = reinterpret_cast<float *>(ws);            // dy . B^T, [T][r_max]
+  float *v = reinterpret_cast<float *>(ws + vbytes);   // x . A^T
+  void *apply_ws = ws + 2 * vbytes;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (dA_dev) {
+    if ((st = mint_lora_shrink(&tp, table, plan_dev, T, dy_dev, lddy, u, status_dev, stream))) return st;
+    if ((st = mint_lora_shrink(pool, table, plan_dev, T, x_dev, ldx, v, status_dev, stream))) return st;
+    const TableDev tab = table_dev(table);
+    if ((st = mint_launch_grad_weight(u, static_cast<const uint16_t *>(x_dev), ldx, dA_dev, pool->desc.d,
+                                      pool->desc.r_max, T, tab, plan_dev, status_dev, s)))
+      return st;
+    if ((st = mint_launch_grad_weight(v, static_cast<const uint16_t *>(dy_dev), lddy, dB_dev, pool->desc.n,
+                                      pool->desc.r_max, T, tab, plan_dev, status_dev, s)))
+      return st;
+  }
+  if (dx_dev)
+    return mint_lora_apply_fused(&tp, table, plan_dev, T, dy_dev, lddy, dx_dev, lddx, apply_ws,
+                                 workspace_bytes - 2 * vbytes, status_dev, stream);
+  return MINT_OK;
+}
+
+// ---------------------------------------------------------------------------
 // MoE
 // ---------------------------------------------------------------------------
 extern "C" size_t mint_moe_lora_apply_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K) {

@@ -1,0 +1,135 @@
+// LoRA backward over padded slots (dense projections).
+//
+// The paper trains many adapters over one frozen base in time slices and names
+// kernels that update several adapters in one batch as the alternative (section
+// "Time-Sliced Multi-LoRA Training"); workers hold adapters in slots of a
+// configured maximum shape, smaller ranks padded and masked.  This file is that
+// alternative for the update the forward path applies,
+//   y[t, :] += s * (x[t, :] . A^T) . B          (A: rank x d, B: rank x n of the token's slot):
+// for an upstream gradient dy,
+//   u = dy . B^T,  v = x . A^T                               (rank values per token)
+//   dx[t, :] += s * u[t, :] . A
+//   dA[slot][k, :] += s * sum over the slot's tokens of u[t, k] * x[t, :]
+//   dB[slot][k, :] += s * sum over the slot's tokens of v[t, k] * dy[t, :]
+// with rows k >= rank (the padding) and slots without tokens left untouched.
+//
+// dx is the forward apply with the pool's tensors in each other's place (B's
+// rows are rank rows of n contiguous elements, exactly what the shrink wants of
+// A, and A's are what the expand wants of B), u and v are the unfused shrink of
+// the same two pools, so those three steps reuse the forward kernels.  What is
+// new is the weight gradient: one CTA per (segment, 512-column block) walks the
+// segment's tokens in plan order and keeps 16 rank rows x 4 columns of fp32
+// sums per thread; a thread owns its elements of dA / dB outright, so there are
+// no atomics and the sums do not depend on scheduling.
+#include "mint_device.cuh"
+
+using namespace mint;
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kColsPerThread = 4;
+constexpr int kColsPerCta = kThreads * kColsPerThread;   // 512
+constexpr int kRankChunk = 16;
+constexpr int kTokenBatch = 64;
+
+struct GradParams {
+  const float *coef;      // [T][r_max] fp32, token order: u (for dA) or v (for dB)
+  const uint16_t *act;    // [T][ld] bf16: x (for dA) or dy (for dB)
+  int64_t ld;
+  float *out;             // [slots][r_max][width] fp32, accumulated into
+  int32_t width, r_max, T;
+  int32_t *status;
+  TableDev tab;
+  PlanView pv;
+};
+
+__global__ void __launch_bounds__(kThreads) grad_weight_kernel(const GradParams p) {
+  __shared__ int32_t tok[kTokenBatch];
+  __shared__ float cf[kTokenBatch][kRankChunk];
+  const int tid = threadIdx.x;
+  if (!plan_ok(p.pv.header, p.T, 1, p.tab.num_slots, 0, p.tab.gen_lo, p.tab.gen_hi,
+               (blockIdx.x == 0 && blockIdx.y == 0) ? p.status : nullptr))
+    return;
+  const int seg = blockIdx.x;
+  if (seg >= p.pv.header[PH_NUM_SEGMENTS]) return;
+  const int off = p.pv.seg_start[seg], len = p.pv.seg_start[seg + 1] - off;
+  const int slot = p.pv.seg_slot[seg];
+  const int rank = p.tab.slot_rank[slot];
+  const float scale = p.tab.slot_scale[slot];
+  if (rank > p.r_max) {
+    if (tid == 0) report(p.status, MINT_ERR_RANK_TOO_LARGE, slot);
+    return;
+  }
+  const int col = blockIdx.y * kColsPerCta + tid * kColsPerThread;
+  const bool col_ok = col < p.width;   // (widths are multiples of 8, so four columns are in or out together)
+  float *out_slot = p.out + (size_t)slot * p.r_max * p.width;
+  for (int k0 = 0; k0 < rank; k0 += kRankChunk) {
+    const int kc = min(kRankChunk, rank - k0);
+    float acc[kRankChunk][kColsPerThread];
+#pragma unroll
+    for (int k = 0; k < kRankChunk; ++k)
+#pragma unroll
+      for (int e = 0; e < kColsPerThread; ++e) acc[k][e] = 0.f;
+    for (int b0 = 0; b0 < len; b0 += kTokenBatch) {
+      const int nb = min(kTokenBatch, len - b0);
+      __syncthreads();   // the previous batch has been read
+      if (tid < nb) tok[tid] = p.pv.perm[off + b0 + tid];
+      __syncthreads();
+      for (int i = tid; i < nb * kRankChunk; i += kThreads) {
+        const int j = i / kRankChunk, k = i - j * kRankChunk;
+        cf[j][k] = k < kc ? p.coef[(size_t)tok[j] * p.r_max + k0 + k] : 0.f;
+      }
+      __syncthreads();
+      if (col_ok) {
+#pragma unroll 4
+        for (int j = 0; j < nb; ++j) {
+          const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p.act + (int64_t)tok[j] * p.ld + col));
+          const float a[4] = {bf16lo(q.x), bf16hi(q.x), bf16lo(q.y), bf16hi(q.y)};
+#pragma unroll
+          for (int k = 0; k < kRankChunk; ++k) {
+            const float c = cf[j][k];
+#pragma unroll
+            for (int e = 0; e < kColsPerThread; ++e) acc[k][e] = fmaf(c, a[e], acc[k][e]);
+          }
+        }
+      }
+    }
+    if (col_ok) {
+#pragma unroll
+      for (int k = 0; k < kRankChunk; ++k)
+        if (k < kc) {
+          float4 *dst = reinterpret_cast<float4 *>(out_slot + (size_t)(k0 + k) * p.width + col);
+          float4 o = *dst;
+          o.x = fmaf(scale, acc[k][0], o.x);
+          o.y = fmaf(scale, acc[k][1], o.y);
+          o.z = fmaf(scale, acc[k][2], o.z);
+          o.w = fmaf(scale, acc[k][3], o.w);
+          *dst = o;
+        }
+    }
+  }
+}
+
+}  // namespace
+
+int32_t mint_launch_grad_weight(const float *coef, const uint16_t *act, int64_t ld, float *out, int32_t width,
+                                int32_t r_max, int32_t T, const TableDev &tab, const void *plan_dev, int32_t *status,
+                                cudaStream_t s) {
+  if (T == 0) return MINT_OK;
+  GradParams p;
+  p.coef = coef;
+  p.act = act;
+  p.ld = ld;
+  p.out = out;
+  p.width = width;
+  p.r_max = r_max;
+  p.T = T;
+  p.status = status;
+  p.tab = tab;
+  p.pv = mint_plan_view(plan_dev, T, tab.num_slots);
+  const int64_t seg_ub = T < tab.num_slots ? T : tab.num_slots;
+  const dim3 grid((unsigned)seg_ub, (unsigned)((width + kColsPerCta - 1) / kColsPerCta));
+  grad_weight_kernel<<<grid, kThreads, 0, s>>>(p);
+  return mint_check_cuda(cudaGetLastError(), "grad_weight launch");
+}

@@ -239,6 +239,12 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);
 
+// Weight gradient of one pool tensor: out[slot][k][:] += scale_slot * sum over the slot's tokens of coef[t][k] * act[t][:]
+// for the rank rows k of the slot (the padding rows are not touched).
+int32_t mint_launch_grad_weight(const float *coef, const uint16_t *act, int64_t ld, float *out, int32_t width,
+                                int32_t r_max, int32_t T, const TableDev &tab, const void *plan_dev, int32_t *status,
+                                cudaStream_t s);
+
 // MoE apply on the streamed kernels (pool r_max of 8, 16, 32 or 64; bound ranks up to 64).
 bool mint_stream_moe_supported(int32_t r_max, int32_t max_bound_rank);
 size_t mint_stream_moe_workspace_bytes(int64_t pairs, int64_t key_space, int32_t r_max);
