@@ -409,6 +409,74 @@ def measure_side_workload(torch, dist, world, stream, name, peak):
     return res
 
 
+def measure_backward(torch, dist, world, stream, peak, layers=6):
+    """The LoRA backward (dx, dA, dB) of every projection of config 2's layer, device-timed: one plan,
+    then mint_lora_backward per projection and layer; every layer has its own tensors (about 0.4 GB each)."""
+    from oracle import backward as oracle_backward
+    from paper_2605_13779_b200 import accounting, binding as mb, harness, synth
+    wl = build_workload("config2", 0)
+    cases = wl["cases"]
+    base = [harness.upload_dense(c) for c in cases]
+    table, ids, status = base[0].table, base[0].ids, mb.new_status()
+    dys = [synth.normal_bf16(synth.stream("bench/backward", c.name), (c.T, c.n), 1.0) for c in cases]
+    rows = []
+    for li in range(layers):
+        row = []
+        for dv, c, dy in zip(base, cases, dys):
+            pool = dv.pool if li == 0 else mb.Pool(dv.pool.A.clone(), dv.pool.B.clone(), c.d, c.n, c.r_max,
+                                                   dv.pool.num_slots)
+            row.append((pool, dv.x if li == 0 else dv.x.clone(), mb.bf16_from_bits(dy),
+                        torch.zeros(c.T, c.d, dtype=torch.bfloat16, device="cuda"),
+                        torch.zeros(c.A.shape, dtype=torch.float32, device="cuda"),
+                        torch.zeros(c.B.shape, dtype=torch.float32, device="cuda")))
+        rows.append(row)
+    ws = [mb.new_backward_workspace(dv.pool, wl["T"]) for dv in base]
+    plan = mb.Plan(wl["T"], 1, table.num_slots, 0)
+
+    def one_pass():
+        mb.mint_lora_plan(table, ids, status, plan=plan)
+        for row in rows:
+            for (pool, x, dy, dx, dA, dB), w in zip(row, ws):
+                mb.mint_lora_backward(pool, table, plan, x, dy, status, dx=dx, dA=dA, dB=dB, workspace=w)
+
+    one_pass()
+    torch.cuda.synchronize()
+    # parity of the first layer's first call (all outputs started at zero) against the fp64 oracle
+    par = {"max_abs_dx": 0.0, "rel_fro_dx": 0.0, "rel_fro_dA": 0.0, "rel_fro_dB": 0.0}
+    for ci in (0, 6):
+        c, (_, _, _, dx, dA, dB) = cases[ci], rows[0][ci]
+        t = c.table
+        dx_ref, dA_ref, dB_ref, _ = oracle_backward.lora_backward(c.ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                                                  c.A, c.B, c.x, dys[ci])
+        dxg = harness.y_to_f64(dx)
+        par["max_abs_dx"] = max(par["max_abs_dx"], float(np.abs(dxg - dx_ref).max()))
+        par["rel_fro_dx"] = max(par["rel_fro_dx"], float(np.linalg.norm(dxg - dx_ref) / np.linalg.norm(dx_ref)))
+        par["rel_fro_dA"] = max(par["rel_fro_dA"], float(np.linalg.norm(dA.cpu().numpy() - dA_ref) / np.linalg.norm(dA_ref)))
+        par["rel_fro_dB"] = max(par["rel_fro_dB"], float(np.linalg.norm(dB.cpu().numpy() - dB_ref) / np.linalg.norm(dB_ref)))
+    par["within_tolerance"] = bool(par["max_abs_dx"] <= 3e-2 and par["rel_fro_dx"] <= 5e-3 and
+                                   par["rel_fro_dA"] <= 1e-4 and par["rel_fro_dB"] <= 1e-4)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            one_pass()
+    est = time_graph(torch, dist, world, stream, g, 2, 2) / 2
+    steps = int(min(100, max(5, 150.0 / max(est, 1e-3))))
+    ms = time_graph(torch, dist, world, stream, g, steps, 3, name="backward") / steps
+    st = status.cpu().numpy()
+    if st[0] != 0:
+        raise SystemExit(f"device status {mb.status_name(int(st[0]))} after the backward loop")
+    layer_bytes = sum(accounting.algorithmic_bytes_backward(c)["total"] for c in cases)
+    res = {"workload": "config2 layer: dx, dA, dB of the seven projections (one call per projection)",
+           "layers": layers, "us_per_layer": ms * 1e3 / layers, "bytes_per_layer": layer_bytes,
+           "GBps": layer_bytes / (ms * 1e-3 / layers) / 1e9,
+           "roofline_frac": layer_bytes / (ms * 1e-3 / layers) / 1e9 / peak,
+           "tokens_per_s": world * wl["T"] * layers / (ms * 1e-3), "parity": par}
+    del g, rows, base, ws
+    gc.collect()
+    torch.cuda.empty_cache()
+    return res
+
+
 def measure_admission(torch, stream):
     """Admitting one adapter into the three expert projections of a 30B-A3B-shaped layer (128 experts):
     the packed representation (one call per projection) against one copy per tensor."""
@@ -645,6 +713,8 @@ def run_gpu(args):
         for name in ("config5", "config4", "config3"):
             workloads[name] = measure_side_workload(torch, dist, 1, stream, name, peak)
     admission = None if args.no_side_workloads else measure_admission(torch, stream)
+    backward = (measure_backward(torch, dist, 1, stream, peak)
+                if (args.workload == "config2" and not args.no_side_workloads and rank == 0) else None)
     cpu_val, cores, sample = oracle_layer_seconds(wl)
 
     line = {
@@ -666,6 +736,7 @@ def run_gpu(args):
         "schedules": other,
         "workloads": workloads,
         "admission": admission,
+        "backward": backward,
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "layers_per_step": e2e_layers},

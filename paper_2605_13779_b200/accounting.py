@@ -37,6 +37,22 @@ def algorithmic_bytes_dense(case: DenseCase) -> dict:
     return b
 
 
+def algorithmic_bytes_backward(case: DenseCase) -> dict:
+    """Bytes the backward must move: x and dy rows of active tokens once, each touched A and B
+    once, dx read + write (bf16), dA and dB of the touched adapters read + write (fp32, true rank
+    rows), plus ids."""
+    f = algorithmic_bytes_dense(case)
+    b = {
+        "x_dy": 2 * f["t_active"] * (case.d + case.n),
+        "ab": f["ab"],
+        "dx": 4 * f["t_active"] * case.d,
+        "grads": 8 * f["sum_rank"] * (case.d + case.n),
+        "ids": f["ids"],
+    }
+    b["total"] = sum(b.values())
+    return b
+
+
 def algorithmic_bytes_moe(case: MoECase) -> dict:
     """MoE apply: x once per distinct row read, each touched (slot, expert)
     A and B once, y read + write per active pair."""

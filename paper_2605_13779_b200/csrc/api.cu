@@ -616,7 +616,10 @@ static mint_pool transposed_pool(const mint_pool *pool) {
 extern "C" size_t mint_lora_backward_workspace_bytes(const mint_pool *pool, int32_t T) {
   if (!pool || T < 0) return 0;
   const mint_pool tp = transposed_pool(pool);
-  return 2 * align256((size_t)T * pool->desc.r_max * sizeof(float)) + mint_lora_apply_workspace_bytes(&tp, T);
+  // u and v, the workspace of the forward kernels on the exchanged pool (the shrink of dy, then the apply
+  // that makes dx) and the one of the shrink of x on the pool itself
+  return 2 * align256((size_t)T * pool->desc.r_max * sizeof(float)) +
+         align256(mint_lora_apply_workspace_bytes(&tp, T)) + align256(mint_lora_apply_workspace_bytes(pool, T));
 }
 
 extern "C" int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
@@ -648,11 +651,26 @@ extern "C" int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_tab
   float *u = reinterpret_cast<float *>(ws);            // dy . B^T, [T][r_max]
   float *v = reinterpret_cast<float *>(ws + vbytes);   // x . A^T
   void *apply_ws = ws + 2 * vbytes;
+  const size_t apply_ws_bytes = align256(mint_lora_apply_workspace_bytes(&tp, T));
+  void *shrink_ws = ws + 2 * vbytes + apply_ws_bytes;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   if (dA_dev) {
-    if ((st = mint_lora_shrink(&tp, table, plan_dev, T, dy_dev, lddy, u, status_dev, stream))) return st;
-    if ((st = mint_lora_shrink(pool, table, plan_dev, T, x_dev, ldx, v, status_dev, stream))) return st;
     const TableDev tab = table_dev(table);
+    if (mint_stream_supported(table->max_rank)) {
+      // both rank-space tensors from one launch of the streamed shrink: dy through B's rows, x through A's
+      DenseArgs two[2] = {dense_args(&tp, T), dense_args(pool, T)};
+      two[0].x = static_cast<const uint16_t *>(dy_dev);
+      two[0].ldx = lddy;
+      two[1].x = static_cast<const uint16_t *>(x_dev);
+      two[1].ldx = ldx;
+      two[0].status = two[1].status = status_dev;
+      void *wss[2] = {apply_ws, shrink_ws};
+      float *vs[2] = {u, v};
+      if ((st = mint_launch_stream_shrink_v(two, 2, tab, plan_dev, wss, vs, s))) return st;
+    } else {
+      if ((st = mint_lora_shrink(&tp, table, plan_dev, T, dy_dev, lddy, u, status_dev, stream))) return st;
+      if ((st = mint_lora_shrink(pool, table, plan_dev, T, x_dev, ldx, v, status_dev, stream))) return st;
+    }
     if ((st = mint_launch_grad_weight(u, static_cast<const uint16_t *>(x_dev), ldx, dA_dev, pool->desc.d,
                                       pool->desc.r_max, T, tab, plan_dev, status_dev, s)))
       return st;
@@ -661,8 +679,8 @@ extern "C" int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_tab
       return st;
   }
   if (dx_dev)
-    return mint_lora_apply_fused(&tp, table, plan_dev, T, dy_dev, lddy, dx_dev, lddx, apply_ws,
-                                 workspace_bytes - 2 * vbytes, status_dev, stream);
+    return mint_lora_apply_fused(&tp, table, plan_dev, T, dy_dev, lddy, dx_dev, lddx, apply_ws, apply_ws_bytes,
+                                 status_dev, stream);
   return MINT_OK;
 }
 

@@ -1441,6 +1441,121 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
   return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
 }
 
+// ---- v in token order from the streamed shrink ----------------------------------------
+// The backward needs x . A^T (and dy . B^T) of every token as a tensor of its own.  The streamed
+// shrink leaves a tile's v as parts, one per lane that met the tile; this kernel adds them, in lane
+// order as the expand would, and writes row l of a tile to row perm[off + l] of v[T][r_max]
+// (ranks below the slot's rank only).  One CTA per tile, all problems of the call.
+struct GatherV {
+  float *v[kMaxProblems];
+};
+
+__global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constant__ StreamParams P, const GatherV out) {
+  __shared__ int32_t part_first[16];
+  __shared__ int32_t part_count[16];
+  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi, nullptr)) return;
+  if (P.pv.header[PH_LANES] != P.lanes) return;
+  const int t = blockIdx.x;
+  if (t >= P.pv.header[PH_NCHUNK1]) return;
+  const TileDesc d = P.pv.tile_desc[t];
+  if (!d.dense) {
+    const Area shrink_area = make_area<false>(P);
+    const int item = threadIdx.x >> 3;
+    int first, count;
+    shrink_parts(P, shrink_area, d, item, item < P.nprob, first, count);
+    if (item < P.nprob && (threadIdx.x & 7) == 0) {
+      part_first[item] = first;
+      part_count[item] = count;
+    }
+  }
+  __syncthreads();
+  const int nel = d.len * d.rank;
+  for (int p = 0; p < P.nprob; ++p) {
+    const StreamProblem &pb = P.prob[p];
+    const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
+    // dense segments: the tensor-core shrink left one part per share of d in slots of their own
+    const int count = d.dense ? mint_dense_splits(pb.d) : part_count[p];
+    const size_t stride = d.dense ? (size_t)(P.dense_slot0 - MINT_MAX_LANES) * slot_floats : slot_floats;
+    const float *part0 = pb.ws_part + (size_t)(t + (d.dense ? P.dense_slot0 : part_first[p])) * slot_floats;
+    for (int i = threadIdx.x; i < nel; i += kThreads) {
+      float s = 0.f;
+      for (int k0 = 0; k0 < count; k0 += 4) {
+        float part[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) part[k] = k0 + k < count ? __ldcg(part0 + (size_t)(k0 + k) * stride + i) : 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) s += part[k];
+      }
+      const int l = i / d.rank, j = i - l * d.rank;
+      out.v[p][(size_t)P.pv.perm[d.off + l] * pb.r_max + j] = s;
+    }
+  }
+}
+
+// x . A^T of every problem into v_out[i] ([T][r_max] fp32, token order; rows of tokens without an adapter
+// and ranks at or above the slot's rank are not written): the streamed shrink, the tensor-core shrink of
+// dense segments, then the kernel above.  Workspaces as for mint_launch_stream.
+int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                    void *const *workspaces, float *const *v_out, cudaStream_t s) {
+  if (nprob < 1 || nprob > kMaxProblems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "grouped shrink: 1..%d problems", kMaxProblems);
+  int32_t lanes = 0;
+  int32_t st = mint_device_lanes(&lanes);
+  if (st) return st;
+  if ((st = stream_kernel_attributes())) return st;
+  const int32_t T = args[0].T;
+  const int64_t tiles = mint_tile_upper_bound(1, T, tab.num_slots);
+  if (tiles == 0) return MINT_OK;
+  StreamParams P = {};
+  GatherV out = {};
+  int cb_s = 0, cb_widest = 0;
+  for (int i = 0; i < nprob; ++i) {
+    const DenseArgs &a = args[i];
+    StreamProblem &pb = P.prob[i];
+    pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
+    pb.ldx = a.ldx; pb.ldy = a.ldy;
+    pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
+    cb_s += kShrinkPieceBlocks;
+    pb.cb0_shrink = cb_s;
+    cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
+    cb_widest = std::max(cb_widest, (a.d + kShrinkBlock - 1) / kShrinkBlock);
+    pb.ws_part = static_cast<float *>(workspaces[i]);
+    out.v[i] = v_out[i];
+  }
+  P.nprob = nprob;
+  P.T = T;
+  P.K = 1;
+  P.weights_per_slot = 1;
+  P.lanes = lanes;
+  P.cb_shrink = cb_s;
+  P.cb_expand = 1;
+  P.cb_shrink_widest = cb_widest;
+  P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
+  P.status = args[0].status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
+
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)lanes);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kRingsBytes;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
+  if (st) return st;
+  if (T >= MINT_DENSE_MIN_BATCH) {
+    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
+    if (st) return st;
+  }
+  // (an ordinary launch: it starts when the shrink kernels are complete)
+  gather_v_kernel<<<(unsigned)tiles, kThreads, 0, s>>>(P, out);
+  return mint_check_cuda(cudaGetLastError(), "gather_v launch");
+}
+
 // ---- fused apply without a caller-provided workspace -------------------------------
 // The workspace of the fused apply, held by the library itself so that a caller
 // that cannot allocate device memory needs none: MINT_STATIC_WORKSPACE_BYTES of

@@ -245,6 +245,12 @@ int32_t mint_launch_grad_weight(const float *coef, const uint16_t *act, int64_t 
                                 int32_t r_max, int32_t T, const TableDev &tab, const void *plan_dev, int32_t *status,
                                 cudaStream_t s);
 
+// x . A^T of up to 8 problems as tensors v_out[i] ([T][r_max] fp32, token order) through the streamed shrink
+// (bound ranks up to 64).  Entries of tokens without an adapter and of ranks at or above a slot's rank are
+// not written.
+int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                    void *const *workspaces, float *const *v_out, cudaStream_t s);
+
 // MoE apply on the streamed kernels (pool r_max of 8, 16, 32 or 64; bound ranks up to 64).
 bool mint_stream_moe_supported(int32_t r_max, int32_t max_bound_rank);
 size_t mint_stream_moe_workspace_bytes(int64_t pairs, int64_t key_space, int32_t r_max);
