@@ -433,11 +433,13 @@ def measure_backward(torch, dist, world, stream, peak, layers=6):
     ws = [mb.new_backward_workspace(dv.pool, wl["T"]) for dv in base]
     plan = mb.Plan(wl["T"], 1, table.num_slots, 0)
 
+    groups = [mb.BackwardGroup([(pool, x, dy, dx, dA, dB, w) for (pool, x, dy, dx, dA, dB), w in zip(row, ws)])
+              for row in rows]
+
     def one_pass():
         mb.mint_lora_plan(table, ids, status, plan=plan)
-        for row in rows:
-            for (pool, x, dy, dx, dA, dB), w in zip(row, ws):
-                mb.mint_lora_backward(pool, table, plan, x, dy, status, dx=dx, dA=dA, dB=dB, workspace=w)
+        for grp in groups:
+            mb.mint_lora_backward_grouped(grp, table, plan, status)
 
     one_pass()
     torch.cuda.synchronize()
@@ -466,12 +468,12 @@ def measure_backward(torch, dist, world, stream, peak, layers=6):
     if st[0] != 0:
         raise SystemExit(f"device status {mb.status_name(int(st[0]))} after the backward loop")
     layer_bytes = sum(accounting.algorithmic_bytes_backward(c)["total"] for c in cases)
-    res = {"workload": "config2 layer: dx, dA, dB of the seven projections (one call per projection)",
+    res = {"workload": "config2 layer: dx, dA, dB of the seven projections (one grouped call per layer)",
            "layers": layers, "us_per_layer": ms * 1e3 / layers, "bytes_per_layer": layer_bytes,
            "GBps": layer_bytes / (ms * 1e-3 / layers) / 1e9,
            "roofline_frac": layer_bytes / (ms * 1e-3 / layers) / 1e9 / peak,
            "tokens_per_s": world * wl["T"] * layers / (ms * 1e-3), "parity": par}
-    del g, rows, base, ws
+    del g, groups, rows, base, ws
     gc.collect()
     torch.cuda.empty_cache()
     return res

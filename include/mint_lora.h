@@ -342,6 +342,26 @@ int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_table *table, 
                            void *dx_dev, int64_t lddx, float *dA_dev, float *dB_dev,
                            void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
                            mint_stream_t stream);
+/* Grouped form: the backward of up to MINT_MAX_GROUP projections that share one
+ * plan (the projections of a layer) with a handful of launches for all of them.
+ * Each item has its own pool, tensors and workspace (rules as above); items
+ * must not alias each other's dx, dA or dB.                                   */
+typedef struct {
+  const mint_pool *pool;
+  const void *x_dev;
+  int64_t ldx;
+  const void *dy_dev;
+  int64_t lddy;
+  void *dx_dev;        /* may be NULL */
+  int64_t lddx;
+  float *dA_dev;       /* both NULL or both given */
+  float *dB_dev;
+  void *workspace_dev;
+  size_t workspace_bytes;
+} mint_backward_item;
+int32_t mint_lora_backward_grouped(const mint_backward_item *items, int32_t count,
+                                   const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                   int32_t *status_dev, mint_stream_t stream);
 
 /* ---- MoE expert LoRA apply -------------------------------------------------
  * Per-expert LoRA tensors keyed by expert id (paper, "Scale Up", Megatron

@@ -45,7 +45,7 @@ EXPORTS = [
     "mint_lora_shrink", "mint_lora_expand",
     "mint_lora_apply_workspace_bytes", "mint_lora_apply_fused", "mint_lora_apply_fused_grouped",
     "mint_lora_apply_fused_static", "mint_selftest_wait_timeout",
-    "mint_lora_backward_workspace_bytes", "mint_lora_backward",
+    "mint_lora_backward_workspace_bytes", "mint_lora_backward", "mint_lora_backward_grouped",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply", "mint_moe_lora_apply_grouped",
     "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
 ]
@@ -67,6 +67,13 @@ class ApplyItem(ctypes.Structure):
     _fields_ = [("pool", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("ldx", ctypes.c_int64),
                 ("y_dev", ctypes.c_void_p), ("ldy", ctypes.c_int64), ("workspace_dev", ctypes.c_void_p),
                 ("workspace_bytes", ctypes.c_size_t)]
+
+
+class BackwardItem(ctypes.Structure):
+    _fields_ = [("pool", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("ldx", ctypes.c_int64),
+                ("dy_dev", ctypes.c_void_p), ("lddy", ctypes.c_int64), ("dx_dev", ctypes.c_void_p),
+                ("lddx", ctypes.c_int64), ("dA_dev", ctypes.c_void_p), ("dB_dev", ctypes.c_void_p),
+                ("workspace_dev", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
 MINT_MAX_GROUP = 8
@@ -133,6 +140,7 @@ def load_library() -> ctypes.CDLL:
         "mint_moe_lora_apply_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_lora_backward_workspace_bytes": (sz, [vp, i32]),
         "mint_lora_backward": (i32, [vp, vp, vp, i32, vp, i64, vp, i64, vp, i64, vp, vp, vp, sz, vp, vp]),
+        "mint_lora_backward_grouped": (i32, [ctypes.POINTER(BackwardItem), i32, vp, vp, i32, vp, vp]),
         "mint_moe_lora_apply": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
         "mint_moe_lora_apply_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, i32, i64, vp, vp, vp, vp]),
         "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
@@ -461,6 +469,29 @@ def mint_lora_backward(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor
         pool.handle, table.handle, _ptr(plan.blob), plan.T, _ptr(x), _ld(x, pool.d), _ptr(dy), _ld(dy, pool.n),
         _ptr(dx), _ld(dx, pool.d) if dx is not None else 0, _ptr(dA), _ptr(dB), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
+
+
+class BackwardGroup:
+    """Up to MINT_MAX_GROUP (pool, x, dy, dx, dA, dB, workspace) items sharing one plan, marshalled once;
+    dx, or dA and dB together, may be None."""
+
+    def __init__(self, items):
+        assert 1 <= len(items) <= MINT_MAX_GROUP
+        self.keep = items
+        arr = (BackwardItem * len(items))()
+        for i, (pool, x, dy, dx, dA, dB, ws) in enumerate(items):
+            for g in (dA, dB):
+                assert g is None or (g.dtype == torch.float32 and g.is_contiguous())
+            arr[i] = BackwardItem(pool.handle, _ptr(x), _ld(x, pool.d), _ptr(dy), _ld(dy, pool.n), _ptr(dx),
+                                  _ld(dx, pool.d) if dx is not None else 0, _ptr(dA), _ptr(dB), _ptr(ws),
+                                  ws.numel() * ws.element_size())
+        self.array = arr
+        self.count = len(items)
+
+
+def mint_lora_backward_grouped(group: BackwardGroup, table: SlotTable, plan: Plan, status: torch.Tensor):
+    _check(load_library().mint_lora_backward_grouped(group.array, group.count, table.handle, _ptr(plan.blob),
+                                                     plan.T, _ptr(status), _stream()))
 
 
 def mint_moe_lora_apply_workspace_bytes(pool: Pool, T: int, K: int) -> int:

@@ -627,60 +627,126 @@ extern "C" int32_t mint_lora_backward(const mint_pool *pool, const mint_slot_tab
                                       void *dx_dev, int64_t lddx, float *dA_dev, float *dB_dev,
                                       void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
                                       mint_stream_t stream) {
-  int32_t st = check_dense(pool, table, plan_dev, T, "backward");
-  if (st) return st;
-  if (!status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "backward: null status_dev");
-  if (T == 0) return MINT_OK;
-  if ((st = check_act(x_dev, ldx, pool->desc.d, "x_dev", "backward"))) return st;
-  if ((st = check_act(dy_dev, lddy, pool->desc.n, "dy_dev", "backward"))) return st;
-  if (dx_dev && (st = check_act(dx_dev, lddx, pool->desc.d, "dx_dev", "backward"))) return st;
-  if ((dA_dev == nullptr) != (dB_dev == nullptr))
-    return mint_fail(MINT_ERR_INVALID_ARG, "backward: dA_dev and dB_dev come together (both or neither)");
-  if ((dA_dev && !aligned16(dA_dev)) || (dB_dev && !aligned16(dB_dev)))
-    return mint_fail(MINT_ERR_MISALIGNED, "backward: dA_dev and dB_dev must be 16-byte aligned");
-  if ((pool->desc.d & 7) || (pool->desc.n & 7))
-    return mint_fail(MINT_ERR_UNSUPPORTED, "backward: d and n must be multiples of 8");
-  const size_t need = mint_lora_backward_workspace_bytes(pool, T);
-  if (!workspace_dev || workspace_bytes < need)
-    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "backward: workspace %zu < %zu", workspace_bytes, need);
-  if (reinterpret_cast<uintptr_t>(workspace_dev) & 255u)
-    return mint_fail(MINT_ERR_MISALIGNED, "backward: workspace must be 256-byte aligned");
-  const mint_pool tp = transposed_pool(pool);
-  const size_t vbytes = align256((size_t)T * pool->desc.r_max * sizeof(float));
-  char *ws = static_cast<char *>(workspace_dev);
-  float *u = reinterpret_cast<float *>(ws);            // dy . B^T, [T][r_max]
-  float *v = reinterpret_cast<float *>(ws + vbytes);   // x . A^T
-  void *apply_ws = ws + 2 * vbytes;
-  const size_t apply_ws_bytes = align256(mint_lora_apply_workspace_bytes(&tp, T));
-  void *shrink_ws = ws + 2 * vbytes + apply_ws_bytes;
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (dA_dev) {
-    const TableDev tab = table_dev(table);
-    if (mint_stream_supported(table->max_rank)) {
-      // both rank-space tensors from one launch of the streamed shrink: dy through B's rows, x through A's
-      DenseArgs two[2] = {dense_args(&tp, T), dense_args(pool, T)};
-      two[0].x = static_cast<const uint16_t *>(dy_dev);
-      two[0].ldx = lddy;
-      two[1].x = static_cast<const uint16_t *>(x_dev);
-      two[1].ldx = ldx;
-      two[0].status = two[1].status = status_dev;
-      void *wss[2] = {apply_ws, shrink_ws};
-      float *vs[2] = {u, v};
-      if ((st = mint_launch_stream_shrink_v(two, 2, tab, plan_dev, wss, vs, s))) return st;
-    } else {
-      if ((st = mint_lora_shrink(&tp, table, plan_dev, T, dy_dev, lddy, u, status_dev, stream))) return st;
-      if ((st = mint_lora_shrink(pool, table, plan_dev, T, x_dev, ldx, v, status_dev, stream))) return st;
-    }
-    if ((st = mint_launch_grad_weight(u, static_cast<const uint16_t *>(x_dev), ldx, dA_dev, pool->desc.d,
-                                      pool->desc.r_max, T, tab, plan_dev, status_dev, s)))
-      return st;
-    if ((st = mint_launch_grad_weight(v, static_cast<const uint16_t *>(dy_dev), lddy, dB_dev, pool->desc.n,
-                                      pool->desc.r_max, T, tab, plan_dev, status_dev, s)))
-      return st;
+  mint_backward_item it;
+  it.pool = pool;
+  it.x_dev = x_dev;
+  it.ldx = ldx;
+  it.dy_dev = dy_dev;
+  it.lddy = lddy;
+  it.dx_dev = dx_dev;
+  it.lddx = lddx;
+  it.dA_dev = dA_dev;
+  it.dB_dev = dB_dev;
+  it.workspace_dev = workspace_dev;
+  it.workspace_bytes = workspace_bytes;
+  return mint_lora_backward_grouped(&it, 1, table, plan_dev, T, status_dev, stream);
+}
+
+extern "C" int32_t mint_lora_backward_grouped(const mint_backward_item *items, int32_t count,
+                                              const mint_slot_table *table, const void *plan_dev, int32_t T,
+                                              int32_t *status_dev, mint_stream_t stream) {
+  if (!items || count < 1 || count > MINT_MAX_GROUP)
+    return mint_fail(MINT_ERR_INVALID_ARG, "backward: count=%d (1..%d)", count, MINT_MAX_GROUP);
+  if (!table || !status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "backward: null argument");
+  int32_t st;
+  mint_pool tp[MINT_MAX_GROUP];
+  for (int i = 0; i < count; ++i) {
+    const mint_backward_item &it = items[i];
+    if ((st = check_dense(it.pool, table, plan_dev, T, "backward"))) return st;
+    if (T == 0) continue;
+    if ((st = check_act(it.x_dev, it.ldx, it.pool->desc.d, "x_dev", "backward"))) return st;
+    if ((st = check_act(it.dy_dev, it.lddy, it.pool->desc.n, "dy_dev", "backward"))) return st;
+    if (it.dx_dev && (st = check_act(it.dx_dev, it.lddx, it.pool->desc.d, "dx_dev", "backward"))) return st;
+    if ((it.dA_dev == nullptr) != (it.dB_dev == nullptr))
+      return mint_fail(MINT_ERR_INVALID_ARG, "backward: dA_dev and dB_dev come together (both or neither)");
+    if ((it.dA_dev && !aligned16(it.dA_dev)) || (it.dB_dev && !aligned16(it.dB_dev)))
+      return mint_fail(MINT_ERR_MISALIGNED, "backward: dA_dev and dB_dev must be 16-byte aligned");
+    if ((it.pool->desc.d & 7) || (it.pool->desc.n & 7))
+      return mint_fail(MINT_ERR_UNSUPPORTED, "backward: d and n must be multiples of 8");
+    const size_t need = mint_lora_backward_workspace_bytes(it.pool, T);
+    if (!it.workspace_dev || it.workspace_bytes < need)
+      return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "backward: workspace %zu < %zu", it.workspace_bytes, need);
+    if (reinterpret_cast<uintptr_t>(it.workspace_dev) & 255u)
+      return mint_fail(MINT_ERR_MISALIGNED, "backward: workspace must be 256-byte aligned");
+    tp[i] = transposed_pool(it.pool);
   }
-  if (dx_dev)
-    return mint_lora_apply_fused(&tp, table, plan_dev, T, dy_dev, lddy, dx_dev, lddx, apply_ws, apply_ws_bytes,
-                                 status_dev, stream);
+  if (T == 0) return MINT_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const TableDev tab = table_dev(table);
+  // every item's workspace: u, v, the workspace of the kernels on the exchanged pool, the one of the shrink of x
+  float *u[MINT_MAX_GROUP], *v[MINT_MAX_GROUP];
+  void *ws_t[MINT_MAX_GROUP], *ws_n[MINT_MAX_GROUP];
+  size_t ws_t_bytes[MINT_MAX_GROUP];
+  for (int i = 0; i < count; ++i) {
+    const size_t vbytes = align256((size_t)T * items[i].pool->desc.r_max * sizeof(float));
+    char *ws = static_cast<char *>(items[i].workspace_dev);
+    u[i] = reinterpret_cast<float *>(ws);
+    v[i] = reinterpret_cast<float *>(ws + vbytes);
+    ws_t[i] = ws + 2 * vbytes;
+    ws_t_bytes[i] = align256(mint_lora_apply_workspace_bytes(&tp[i], T));
+    ws_n[i] = ws + 2 * vbytes + ws_t_bytes[i];
+  }
+  // 1. the rank-space tensors u = dy . B^T and v = x . A^T of every item whose adapters are trained
+  DenseArgs probs[2 * MINT_MAX_GROUP];
+  void *pws[2 * MINT_MAX_GROUP];
+  float *pv[2 * MINT_MAX_GROUP];
+  GradJobHost jobs[2 * MINT_MAX_GROUP];
+  int np = 0;
+  for (int i = 0; i < count; ++i) {
+    const mint_backward_item &it = items[i];
+    if (!it.dA_dev) continue;
+    probs[np] = dense_args(&tp[i], T);
+    probs[np].x = static_cast<const uint16_t *>(it.dy_dev);
+    probs[np].ldx = it.lddy;
+    probs[np].status = status_dev;
+    pws[np] = ws_t[i];
+    pv[np] = u[i];
+    jobs[np] = GradJobHost{u[i], static_cast<const uint16_t *>(it.x_dev), it.ldx, it.dA_dev, it.pool->desc.d,
+                           it.pool->desc.r_max};
+    ++np;
+    probs[np] = dense_args(it.pool, T);
+    probs[np].x = static_cast<const uint16_t *>(it.x_dev);
+    probs[np].ldx = it.ldx;
+    probs[np].status = status_dev;
+    pws[np] = ws_n[i];
+    pv[np] = v[i];
+    jobs[np] = GradJobHost{v[i], static_cast<const uint16_t *>(it.dy_dev), it.lddy, it.dB_dev, it.pool->desc.n,
+                           it.pool->desc.r_max};
+    ++np;
+  }
+  if (np > 0) {
+    if (mint_stream_supported(table->max_rank)) {
+      for (int p0 = 0; p0 < np; p0 += MINT_MAX_GROUP) {   // the streamed shrink takes eight problems a launch
+        const int m = np - p0 < MINT_MAX_GROUP ? np - p0 : MINT_MAX_GROUP;
+        if ((st = mint_launch_stream_shrink_v(probs + p0, m, tab, plan_dev, pws + p0, pv + p0, s))) return st;
+      }
+    } else {
+      for (int i = 0; i < count; ++i) {
+        const mint_backward_item &it = items[i];
+        if (!it.dA_dev) continue;
+        if ((st = mint_lora_shrink(&tp[i], table, plan_dev, T, it.dy_dev, it.lddy, u[i], status_dev, stream))) return st;
+        if ((st = mint_lora_shrink(it.pool, table, plan_dev, T, it.x_dev, it.ldx, v[i], status_dev, stream))) return st;
+      }
+    }
+    // 2. dA and dB of all items in one launch
+    if ((st = mint_launch_grad_weights(jobs, np, T, tab, plan_dev, status_dev, s))) return st;
+  }
+  // 3. dx of all items: the fused apply on the exchanged pools
+  mint_apply_item ax[MINT_MAX_GROUP];
+  int nx = 0;
+  for (int i = 0; i < count; ++i) {
+    const mint_backward_item &it = items[i];
+    if (!it.dx_dev) continue;
+    ax[nx].pool = &tp[i];
+    ax[nx].x_dev = it.dy_dev;
+    ax[nx].ldx = it.lddy;
+    ax[nx].y_dev = it.dx_dev;
+    ax[nx].ldy = it.lddx;
+    ax[nx].workspace_dev = ws_t[i];
+    ax[nx].workspace_bytes = ws_t_bytes[i];
+    ++nx;
+  }
+  if (nx > 0) return mint_lora_apply_fused_grouped(ax, nx, table, plan_dev, T, status_dev, stream);
   return MINT_OK;
 }
 

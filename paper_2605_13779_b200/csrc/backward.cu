@@ -33,35 +33,47 @@ constexpr int kColsPerCta = kThreads * kColsPerThread;   // 512
 constexpr int kRankChunk = 16;
 constexpr int kTokenBatch = 64;
 
-struct GradParams {
+constexpr int kMaxJobs = 2 * MINT_MAX_GROUP;   // dA and dB of every projection of a grouped call
+
+struct GradJob {
   const float *coef;      // [T][r_max] fp32, token order: u (for dA) or v (for dB)
   const uint16_t *act;    // [T][ld] bf16: x (for dA) or dy (for dB)
   int64_t ld;
   float *out;             // [slots][r_max][width] fp32, accumulated into
-  int32_t width, r_max, T;
+  int32_t width, r_max;
+  int32_t block0;         // first of its 512-column blocks in the grid's second dimension
+  int32_t pad;
+};
+
+struct GradParams {
+  GradJob job[kMaxJobs];
+  int32_t njobs, T;
   int32_t *status;
   TableDev tab;
   PlanView pv;
 };
 
-__global__ void __launch_bounds__(kThreads) grad_weight_kernel(const GradParams p) {
+__global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_constant__ GradParams P) {
   __shared__ int32_t tok[kTokenBatch];
   __shared__ float cf[kTokenBatch][kRankChunk];
   const int tid = threadIdx.x;
-  if (!plan_ok(p.pv.header, p.T, 1, p.tab.num_slots, 0, p.tab.gen_lo, p.tab.gen_hi,
-               (blockIdx.x == 0 && blockIdx.y == 0) ? p.status : nullptr))
+  if (!plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi,
+               (blockIdx.x == 0 && blockIdx.y == 0) ? P.status : nullptr))
     return;
+  int ji = 0;   // the job this column block belongs to
+  while (ji + 1 < P.njobs && (int)blockIdx.y >= P.job[ji + 1].block0) ++ji;
+  const GradJob &p = P.job[ji];
   const int seg = blockIdx.x;
-  if (seg >= p.pv.header[PH_NUM_SEGMENTS]) return;
-  const int off = p.pv.seg_start[seg], len = p.pv.seg_start[seg + 1] - off;
-  const int slot = p.pv.seg_slot[seg];
-  const int rank = p.tab.slot_rank[slot];
-  const float scale = p.tab.slot_scale[slot];
+  if (seg >= P.pv.header[PH_NUM_SEGMENTS]) return;
+  const int off = P.pv.seg_start[seg], len = P.pv.seg_start[seg + 1] - off;
+  const int slot = P.pv.seg_slot[seg];
+  const int rank = P.tab.slot_rank[slot];
+  const float scale = P.tab.slot_scale[slot];
   if (rank > p.r_max) {
-    if (tid == 0) report(p.status, MINT_ERR_RANK_TOO_LARGE, slot);
+    if (tid == 0) report(P.status, MINT_ERR_RANK_TOO_LARGE, slot);
     return;
   }
-  const int col = blockIdx.y * kColsPerCta + tid * kColsPerThread;
+  const int col = ((int)blockIdx.y - p.block0) * kColsPerCta + tid * kColsPerThread;
   const bool col_ok = col < p.width;   // (widths are multiples of 8, so four columns are in or out together)
   float *out_slot = p.out + (size_t)slot * p.r_max * p.width;
   for (int k0 = 0; k0 < rank; k0 += kRankChunk) {
@@ -74,7 +86,7 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const GradParams 
     for (int b0 = 0; b0 < len; b0 += kTokenBatch) {
       const int nb = min(kTokenBatch, len - b0);
       __syncthreads();   // the previous batch has been read
-      if (tid < nb) tok[tid] = p.pv.perm[off + b0 + tid];
+      if (tid < nb) tok[tid] = P.pv.perm[off + b0 + tid];
       __syncthreads();
       for (int i = tid; i < nb * kRankChunk; i += kThreads) {
         const int j = i / kRankChunk, k = i - j * kRankChunk;
@@ -113,23 +125,30 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const GradParams 
 
 }  // namespace
 
-int32_t mint_launch_grad_weight(const float *coef, const uint16_t *act, int64_t ld, float *out, int32_t width,
-                                int32_t r_max, int32_t T, const TableDev &tab, const void *plan_dev, int32_t *status,
-                                cudaStream_t s) {
-  if (T == 0) return MINT_OK;
-  GradParams p;
-  p.coef = coef;
-  p.act = act;
-  p.ld = ld;
-  p.out = out;
-  p.width = width;
-  p.r_max = r_max;
-  p.T = T;
-  p.status = status;
-  p.tab = tab;
-  p.pv = mint_plan_view(plan_dev, T, tab.num_slots);
+int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, const TableDev &tab,
+                                 const void *plan_dev, int32_t *status, cudaStream_t s) {
+  if (T == 0 || njobs == 0) return MINT_OK;
+  if (njobs > kMaxJobs) return mint_fail(MINT_ERR_INVALID_ARG, "weight gradients: at most %d tensors per launch", kMaxJobs);
+  GradParams P = {};
+  int blocks = 0;
+  for (int i = 0; i < njobs; ++i) {
+    GradJob &j = P.job[i];
+    j.coef = jobs[i].coef;
+    j.act = jobs[i].act;
+    j.ld = jobs[i].ld;
+    j.out = jobs[i].out;
+    j.width = jobs[i].width;
+    j.r_max = jobs[i].r_max;
+    j.block0 = blocks;
+    blocks += (jobs[i].width + kColsPerCta - 1) / kColsPerCta;
+  }
+  P.njobs = njobs;
+  P.T = T;
+  P.status = status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
   const int64_t seg_ub = T < tab.num_slots ? T : tab.num_slots;
-  const dim3 grid((unsigned)seg_ub, (unsigned)((width + kColsPerCta - 1) / kColsPerCta));
-  grad_weight_kernel<<<grid, kThreads, 0, s>>>(p);
+  const dim3 grid((unsigned)seg_ub, (unsigned)blocks);
+  grad_weight_kernel<<<grid, kThreads, 0, s>>>(P);
   return mint_check_cuda(cudaGetLastError(), "grad_weight launch");
 }

@@ -239,11 +239,18 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
 int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                            void *const *workspaces, cudaStream_t s);
 
-// Weight gradient of one pool tensor: out[slot][k][:] += scale_slot * sum over the slot's tokens of coef[t][k] * act[t][:]
+// Weight gradients of up to 16 pool tensors in one launch:
+//   out[slot][k][:] += scale_slot * sum over the slot's tokens of coef[t][k] * act[t][:]
 // for the rank rows k of the slot (the padding rows are not touched).
-int32_t mint_launch_grad_weight(const float *coef, const uint16_t *act, int64_t ld, float *out, int32_t width,
-                                int32_t r_max, int32_t T, const TableDev &tab, const void *plan_dev, int32_t *status,
-                                cudaStream_t s);
+struct GradJobHost {
+  const float *coef;      // [T][r_max] fp32, token order
+  const uint16_t *act;    // [T][ld] bf16
+  int64_t ld;
+  float *out;             // [slots][r_max][width] fp32
+  int32_t width, r_max;
+};
+int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, const TableDev &tab,
+                                 const void *plan_dev, int32_t *status, cudaStream_t s);
 
 // x . A^T of up to 8 problems as tensors v_out[i] ([T][r_max] fp32, token order) through the streamed shrink
 // (bound ranks up to 64).  Entries of tokens without an adapter and of ranks at or above a slot's rank are

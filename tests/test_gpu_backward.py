@@ -137,3 +137,39 @@ def test_backward_is_deterministic_and_accumulates():
     # two calls add the gradient twice
     np.testing.assert_allclose(twice["dA"] - a["dA0"], 2 * (dA_ref - a["dA0"]), rtol=2e-4, atol=1e-5)
     np.testing.assert_allclose(twice["dB"] - a["dB0"], 2 * (dB_ref - a["dB0"]), rtol=2e-4, atol=1e-5)
+
+
+def test_grouped_backward_of_a_whole_layer():
+    """The seven projections of the 4B-dense decode layer in one grouped call (as the benchmark issues it);
+    one of them with frozen adapters, one without an input gradient."""
+    from paper_2605_13779_b200 import binding as mb, harness
+    batch = synth.config2_batch()
+    cases = [synth.config2_projection(batch, p) for p in synth.QWEN3_4B_PROJECTIONS]
+    table = harness.upload_table(cases[0].table)
+    devs = [harness.upload_dense(c, table=table) for c in cases]
+    status = devs[0].status
+    plan = mb.mint_lora_plan(table, devs[0].ids, status)
+    items, keep = [], []
+    for i, (c, dv) in enumerate(zip(cases, devs)):
+        dy = synth.normal_bf16(synth.stream(c.name, "dy"), (c.T, c.n), 1.0)
+        dx0 = synth.normal_bf16(synth.stream(c.name, "dx0"), c.x.shape, 1.0)
+        dx = None if i == 2 else mb.bf16_from_bits(dx0)
+        frozen = i == 4
+        dA = None if frozen else torch.zeros(c.A.shape, dtype=torch.float32, device="cuda")
+        dB = None if frozen else torch.zeros(c.B.shape, dtype=torch.float32, device="cuda")
+        ws = mb.new_backward_workspace(dv.pool, c.T)
+        ws.fill_(0xFF)
+        items.append((dv.pool, dv.x, mb.bf16_from_bits(dy), dx, dA, dB, ws))
+        keep.append((dy, dx0))
+    mb.mint_lora_backward_grouped(mb.BackwardGroup(items), table, plan, status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    for c, (pool, x, dyd, dx, dA, dB, ws), (dy, dx0) in zip(cases, items, keep):
+        dx_ref, dA_ref, dB_ref, _ = oracle_backward(c, dy, dx0, None, None)
+        if dx is not None:
+            parity.assert_close(harness.y_to_f64(dx), dx_ref, f"grouped {c.name} dx")
+        if dA is not None:
+            zero = np.zeros(c.A.shape, dtype=np.float32)
+            check_grads(dA.cpu().numpy().astype(np.float64), dA_ref, zero, c, f"grouped {c.name} dA")
+            check_grads(dB.cpu().numpy().astype(np.float64), dB_ref, np.zeros(c.B.shape, dtype=np.float32), c,
+                        f"grouped {c.name} dB")
