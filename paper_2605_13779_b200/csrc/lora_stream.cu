@@ -1445,50 +1445,46 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
 // The backward needs x . A^T (and dy . B^T) of every token as a tensor of its own.  The streamed
 // shrink leaves a tile's v as parts, one per lane that met the tile; this kernel adds them, in lane
 // order as the expand would, and writes row l of a tile to row perm[off + l] of v[T][r_max]
-// (ranks below the slot's rank only).  One CTA per tile, all problems of the call.
+// (ranks below the slot's rank only).  One CTA per (tile, problem).
 struct GatherV {
   float *v[kMaxProblems];
 };
 
 __global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constant__ StreamParams P, const GatherV out) {
-  __shared__ int32_t part_first[16];
-  __shared__ int32_t part_count[16];
+  __shared__ int32_t part_first, part_count;
   if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi, nullptr)) return;
   if (P.pv.header[PH_LANES] != P.lanes) return;
-  const int t = blockIdx.x;
+  const int t = blockIdx.x, p = blockIdx.y;
   if (t >= P.pv.header[PH_NCHUNK1]) return;
   const TileDesc d = P.pv.tile_desc[t];
   if (!d.dense) {
     const Area shrink_area = make_area<false>(P);
-    const int item = threadIdx.x >> 3;
     int first, count;
-    shrink_parts(P, shrink_area, d, item, item < P.nprob, first, count);
-    if (item < P.nprob && (threadIdx.x & 7) == 0) {
-      part_first[item] = first;
-      part_count[item] = count;
+    shrink_parts(P, shrink_area, d, p, threadIdx.x < 8, first, count);   // (eight threads look per item)
+    if (threadIdx.x == 0) {
+      part_first = first;
+      part_count = count;
     }
   }
   __syncthreads();
   const int nel = d.len * d.rank;
-  for (int p = 0; p < P.nprob; ++p) {
-    const StreamProblem &pb = P.prob[p];
-    const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
-    // dense segments: the tensor-core shrink left one part per share of d in slots of their own
-    const int count = d.dense ? mint_dense_splits(pb.d) : part_count[p];
-    const size_t stride = d.dense ? (size_t)(P.dense_slot0 - MINT_MAX_LANES) * slot_floats : slot_floats;
-    const float *part0 = pb.ws_part + (size_t)(t + (d.dense ? P.dense_slot0 : part_first[p])) * slot_floats;
-    for (int i = threadIdx.x; i < nel; i += kThreads) {
-      float s = 0.f;
-      for (int k0 = 0; k0 < count; k0 += 4) {
-        float part[4];
+  const StreamProblem &pb = P.prob[p];
+  const size_t slot_floats = (size_t)kTileRowsMax * pb.r_max;
+  // dense segments: the tensor-core shrink left one part per share of d in slots of their own
+  const int count = d.dense ? mint_dense_splits(pb.d) : part_count;
+  const size_t stride = d.dense ? (size_t)(P.dense_slot0 - MINT_MAX_LANES) * slot_floats : slot_floats;
+  const float *part0 = pb.ws_part + (size_t)(t + (d.dense ? P.dense_slot0 : part_first)) * slot_floats;
+  for (int i = threadIdx.x; i < nel; i += kThreads) {
+    float s = 0.f;
+    for (int k0 = 0; k0 < count; k0 += 4) {
+      float part[4];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) part[k] = k0 + k < count ? __ldcg(part0 + (size_t)(k0 + k) * stride + i) : 0.f;
+      for (int k = 0; k < 4; ++k) part[k] = k0 + k < count ? __ldcg(part0 + (size_t)(k0 + k) * stride + i) : 0.f;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) s += part[k];
-      }
-      const int l = i / d.rank, j = i - l * d.rank;
-      out.v[p][(size_t)P.pv.perm[d.off + l] * pb.r_max + j] = s;
+      for (int k = 0; k < 4; ++k) s += part[k];
     }
+    const int l = i / d.rank, j = i - l * d.rank;
+    out.v[p][(size_t)P.pv.perm[d.off + l] * pb.r_max + j] = s;
   }
 }
 
@@ -1552,7 +1548,7 @@ int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const Tabl
     if (st) return st;
   }
   // (an ordinary launch: it starts when the shrink kernels are complete)
-  gather_v_kernel<<<(unsigned)tiles, kThreads, 0, s>>>(P, out);
+  gather_v_kernel<<<dim3((unsigned)tiles, (unsigned)nprob), kThreads, 0, s>>>(P, out);
   return mint_check_cuda(cudaGetLastError(), "gather_v launch");
 }
 
