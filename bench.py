@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-adapter LoRA apply on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3|config1]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3|config1|backward]
     python bench.py --impl reference ...        # the fp64 CPU oracle, timed on the host cores
 
 A step is a fixed number of passes of the whole hot path over one batch: each
@@ -409,7 +409,7 @@ def measure_side_workload(torch, dist, world, stream, name, peak):
     return res
 
 
-def measure_backward(torch, dist, world, stream, peak, layers=6):
+def measure_backward(torch, dist, world, stream, peak, layers=6, short=False):
     """The LoRA backward (dx, dA, dB) of every projection of config 2's layer, device-timed: one plan,
     then mint_lora_backward per projection and layer; every layer has its own tensors (about 0.4 GB each)."""
     from oracle import backward as oracle_backward
@@ -462,7 +462,7 @@ def measure_backward(torch, dist, world, stream, peak, layers=6):
         with torch.cuda.graph(g, stream=stream):
             one_pass()
     est = time_graph(torch, dist, world, stream, g, 2, 2) / 2
-    steps = int(min(100, max(5, 150.0 / max(est, 1e-3))))
+    steps = 2 if short else int(min(100, max(5, 150.0 / max(est, 1e-3))))
     ms = time_graph(torch, dist, world, stream, g, steps, 3, name="backward") / steps
     st = status.cpu().numpy()
     if st[0] != 0:
@@ -537,6 +537,12 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     mb.load_library()
     peak, peak_src = hbm_peak()
+    if args.workload == "backward":   # the backward alone (the command profilers wrap): its own JSON line
+        res = measure_backward(torch, dist, 1, torch.cuda.Stream(), peak, layers=args.layers or 6,
+                               short=args.profile)
+        if rank == 0:
+            print(json.dumps(res))
+        return
 
     wl = build_workload(args.workload, args.layers)
     dw = DeviceWorkload(wl, wl["layers"])
