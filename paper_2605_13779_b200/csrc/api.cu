@@ -686,6 +686,35 @@ extern "C" int32_t mint_lora_backward_grouped(const mint_backward_item *items, i
     ws_t_bytes[i] = align256(mint_lora_apply_workspace_bytes(&tp[i], T));
     ws_n[i] = ws + 2 * vbytes + ws_t_bytes[i];
   }
+  // The usual training step wants everything of every item: then the shrink of dy through B's rows serves
+  // twice, as u for dA and as the first half of the apply that makes dx (its parts stay in the workspace).
+  bool everything = mint_stream_supported(table->max_rank);
+  for (int i = 0; i < count; ++i) everything = everything && items[i].dx_dev && items[i].dA_dev;
+  if (everything) {
+    DenseArgs pu[MINT_MAX_GROUP], pv_[MINT_MAX_GROUP];
+    GradJobHost jobs[2 * MINT_MAX_GROUP];
+    for (int i = 0; i < count; ++i) {
+      const mint_backward_item &it = items[i];
+      pu[i] = dense_args(&tp[i], T);
+      pu[i].x = static_cast<const uint16_t *>(it.dy_dev);
+      pu[i].ldx = it.lddy;
+      pu[i].y = static_cast<uint16_t *>(it.dx_dev);
+      pu[i].ldy = it.lddx;
+      pu[i].status = status_dev;
+      pv_[i] = dense_args(it.pool, T);
+      pv_[i].x = static_cast<const uint16_t *>(it.x_dev);
+      pv_[i].ldx = it.ldx;
+      pv_[i].status = status_dev;
+      jobs[2 * i] = GradJobHost{u[i], static_cast<const uint16_t *>(it.x_dev), it.ldx, it.dA_dev, it.pool->desc.d,
+                                it.pool->desc.r_max};
+      jobs[2 * i + 1] = GradJobHost{v[i], static_cast<const uint16_t *>(it.dy_dev), it.lddy, it.dB_dev,
+                                    it.pool->desc.n, it.pool->desc.r_max};
+    }
+    if ((st = mint_launch_stream_phases(pu, count, tab, plan_dev, ws_t, s, 1, u))) return st;
+    if ((st = mint_launch_stream_phases(pv_, count, tab, plan_dev, ws_n, s, 1, v))) return st;
+    if ((st = mint_launch_grad_weights(jobs, 2 * count, T, tab, plan_dev, status_dev, s))) return st;
+    return mint_launch_stream_phases(pu, count, tab, plan_dev, ws_t, s, 2, nullptr);
+  }
   // 1. the rank-space tensors u = dy . B^T and v = x . A^T of every item whose adapters are trained
   DenseArgs probs[2 * MINT_MAX_GROUP];
   void *pws[2 * MINT_MAX_GROUP];

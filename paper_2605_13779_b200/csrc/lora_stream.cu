@@ -1374,73 +1374,6 @@ size_t mint_stream_workspace_bytes(int32_t T, int32_t num_slots, int32_t r_max) 
   return workspace_bytes(mint_tile_upper_bound(1, T, num_slots), r_max, T >= MINT_DENSE_MIN_BATCH);
 }
 
-int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                           void *const *workspaces, cudaStream_t s) {
-  if (nprob < 1 || nprob > kMaxProblems)
-    return mint_fail(MINT_ERR_INVALID_ARG, "grouped apply: 1..%d problems", kMaxProblems);
-  int32_t lanes = 0;
-  int32_t st = mint_device_lanes(&lanes);
-  if (st) return st;
-  if ((st = stream_kernel_attributes())) return st;
-  const int32_t T = args[0].T;
-  const int64_t tiles = mint_tile_upper_bound(1, T, tab.num_slots);
-  if (tiles == 0) return MINT_OK;
-  StreamParams P = {};
-  int cb_s = 0, cb_e = 0, cb_widest = 0;
-  for (int i = 0; i < nprob; ++i) {
-    const DenseArgs &a = args[i];
-    StreamProblem &pb = P.prob[i];
-    pb.A = a.A; pb.B = a.B; pb.x = a.x; pb.y = a.y;
-    pb.ldx = a.ldx; pb.ldy = a.ldy;
-    pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
-    cb_s += kShrinkPieceBlocks;
-    cb_e += kExpandPieceBlocks;
-    pb.cb0_shrink = cb_s;
-    pb.cb0_expand = cb_e;
-    cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
-    cb_widest = std::max(cb_widest, (a.d + kShrinkBlock - 1) / kShrinkBlock);
-    cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
-    pb.ws_part = static_cast<float *>(workspaces[i]);
-  }
-  P.nprob = nprob;
-  P.T = T;
-  P.K = 1;
-  P.num_experts = 0;
-  P.weights_per_slot = 1;
-  P.lanes = lanes;
-  P.cb_shrink = cb_s;
-  P.cb_expand = cb_e;
-  P.cb_shrink_widest = cb_widest;
-  P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
-  P.status = args[0].status;
-  P.tab = tab;
-  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
-
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)lanes);
-  cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = kRingsBytes;
-  cfg.stream = s;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  // the first apply after a plan or a bind waits for that kernel in full: it reads the plan at once
-  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
-  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
-  if (st) return st;
-  cfg.numAttrs = 1;
-  const bool dense = T >= MINT_DENSE_MIN_BATCH;   // the plan may have given dense segments to the tensor-core kernels
-  if (dense) {
-    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
-    if (st) return st;
-  }
-  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
-  if (st || !dense) return st;
-  return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
-}
-
 // ---- v in token order from the streamed shrink ----------------------------------------
 // The backward needs x . A^T (and dy . B^T) of every token as a tensor of its own.  The streamed
 // shrink leaves a tile's v as parts, one per lane that met the tile; this kernel adds them, in lane
@@ -1488,13 +1421,14 @@ __global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constan
   }
 }
 
-// x . A^T of every problem into v_out[i] ([T][r_max] fp32, token order; rows of tokens without an adapter
-// and ranks at or above the slot's rank are not written): the streamed shrink, the tensor-core shrink of
-// dense segments, then the kernel above.  Workspaces as for mint_launch_stream.
-int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                                    void *const *workspaces, float *const *v_out, cudaStream_t s) {
+// The streamed fused apply of up to eight problems.  phases: bit 0 = the shrink (and the tensor-core
+// shrink of dense segments), bit 1 = the expand (and theirs).  v_out, when given, receives x . A^T of
+// every problem in token order ([T][r_max] fp32) right after the shrink.  A call with the expand alone
+// relies on the parts an earlier call with the same problems, plan and workspaces left behind.
+int32_t mint_launch_stream_phases(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                  void *const *workspaces, cudaStream_t s, int phases, float *const *v_out) {
   if (nprob < 1 || nprob > kMaxProblems)
-    return mint_fail(MINT_ERR_INVALID_ARG, "grouped shrink: 1..%d problems", kMaxProblems);
+    return mint_fail(MINT_ERR_INVALID_ARG, "grouped apply: 1..%d problems", kMaxProblems);
   int32_t lanes = 0;
   int32_t st = mint_device_lanes(&lanes);
   if (st) return st;
@@ -1504,7 +1438,7 @@ int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const Tabl
   if (tiles == 0) return MINT_OK;
   StreamParams P = {};
   GatherV out = {};
-  int cb_s = 0, cb_widest = 0;
+  int cb_s = 0, cb_e = 0, cb_widest = 0;
   for (int i = 0; i < nprob; ++i) {
     const DenseArgs &a = args[i];
     StreamProblem &pb = P.prob[i];
@@ -1512,19 +1446,23 @@ int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const Tabl
     pb.ldx = a.ldx; pb.ldy = a.ldy;
     pb.d = a.d; pb.n = a.n; pb.r_max = a.r_max;
     cb_s += kShrinkPieceBlocks;
+    cb_e += kExpandPieceBlocks;
     pb.cb0_shrink = cb_s;
+    pb.cb0_expand = cb_e;
     cb_s += (a.d + kShrinkBlock - 1) / kShrinkBlock;
     cb_widest = std::max(cb_widest, (a.d + kShrinkBlock - 1) / kShrinkBlock);
+    cb_e += (a.n + kExpandBlock - 1) / kExpandBlock;
     pb.ws_part = static_cast<float *>(workspaces[i]);
-    out.v[i] = v_out[i];
+    if (v_out) out.v[i] = v_out[i];
   }
   P.nprob = nprob;
   P.T = T;
   P.K = 1;
+  P.num_experts = 0;
   P.weights_per_slot = 1;
   P.lanes = lanes;
   P.cb_shrink = cb_s;
-  P.cb_expand = 1;
+  P.cb_expand = cb_e;
   P.cb_shrink_widest = cb_widest;
   P.dense_slot0 = (int32_t)(tiles + MINT_MAX_LANES);
   P.status = args[0].status;
@@ -1540,16 +1478,38 @@ int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const Tabl
   cfg.dynamicSmemBytes = kRingsBytes;
   cfg.stream = s;
   cfg.attrs = attr;
-  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
-  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
-  if (st) return st;
-  if (T >= MINT_DENSE_MIN_BATCH) {
-    st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
+  const bool dense = T >= MINT_DENSE_MIN_BATCH;   // the plan may have given dense segments to the tensor-core kernels
+  if (phases & 1) {
+    // the first apply after a plan or a bind waits for that kernel in full: it reads the plan at once
+    cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+    st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
     if (st) return st;
+    if (dense) {
+      st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
+      if (st) return st;
+    }
+    if (v_out) {   // (an ordinary launch: it starts when the shrink kernels are complete)
+      gather_v_kernel<<<dim3((unsigned)tiles, (unsigned)nprob), kThreads, 0, s>>>(P, out);
+      if ((st = mint_check_cuda(cudaGetLastError(), "gather_v launch"))) return st;
+    }
   }
-  // (an ordinary launch: it starts when the shrink kernels are complete)
-  gather_v_kernel<<<dim3((unsigned)tiles, (unsigned)nprob), kThreads, 0, s>>>(P, out);
-  return mint_check_cuda(cudaGetLastError(), "gather_v launch");
+  if (!(phases & 2)) return MINT_OK;
+  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+  st = mint_check_cuda(cudaLaunchKernelEx(&cfg, expand_stream_kernel, P), "expand_stream launch");
+  if (st || !dense) return st;
+  return mint_launch_dense_expand(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
+}
+
+int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                           void *const *workspaces, cudaStream_t s) {
+  return mint_launch_stream_phases(args, nprob, tab, plan_dev, workspaces, s, 3, nullptr);
+}
+
+// x . A^T of every problem into v_out[i] ([T][r_max] fp32, token order; rows of tokens without an adapter
+// and ranks at or above the slot's rank are not written).  Workspaces as for mint_launch_stream.
+int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                    void *const *workspaces, float *const *v_out, cudaStream_t s) {
+  return mint_launch_stream_phases(args, nprob, tab, plan_dev, workspaces, s, 1, v_out);
 }
 
 // ---- fused apply without a caller-provided workspace -------------------------------

@@ -257,6 +257,11 @@ int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, 
 // not written.
 int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                     void *const *workspaces, float *const *v_out, cudaStream_t s);
+// The same launcher by phases: bit 0 of `phases` = the shrink (v_out, when given, receives x . A^T in token
+// order), bit 1 = the expand.  The expand alone relies on the parts that an earlier shrink-only call with
+// the same problems, plan and workspaces left in the workspaces.
+int32_t mint_launch_stream_phases(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                  void *const *workspaces, cudaStream_t s, int phases, float *const *v_out);
 
 // MoE apply on the streamed kernels (pool r_max of 8, 16, 32 or 64; bound ranks up to 64).
 bool mint_stream_moe_supported(int32_t r_max, int32_t max_bound_rank);

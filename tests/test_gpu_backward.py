@@ -121,8 +121,14 @@ def test_frozen_adapters_and_no_input_gradient():
     only_dx = run_backward(case, dy, want_grads=False)
     only_w = run_backward(case, dy, want_dx=False)
     np.testing.assert_array_equal(only_dx["dx"], full["dx"])
-    np.testing.assert_array_equal(only_w["dA"], full["dA"])
-    np.testing.assert_array_equal(only_w["dB"], full["dB"])
+    # (a call that wants everything shares the shrink of dy between dA and dx, so its lanes cut the columns
+    # elsewhere than those of a call for the weight gradients alone: equal up to fp32 summation order)
+    np.testing.assert_allclose(only_w["dA"] - full["dA0"], full["dA"] - full["dA0"], rtol=1e-4, atol=1e-5)
+    np.testing.assert_allclose(only_w["dB"] - full["dB0"], full["dB"] - full["dB0"], rtol=1e-4, atol=1e-5)
+    dy_ref = oracle_backward(case, dy, full["dx0"], full["dA0"], full["dB0"])
+    check_grads(only_w["dA"], dy_ref[1], full["dA0"], case, "weights only dA")
+    check_grads(only_w["dB"], dy_ref[2], full["dB0"], case, "weights only dB")
+    parity.assert_close(only_dx["dx"], dy_ref[0], "dx only")
 
 
 def test_backward_is_deterministic_and_accumulates():
