@@ -176,3 +176,46 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable()
     assert status[0].item() == 0
     y_ref, _, _ = parity.oracle_dense(case)
     parity.assert_close(harness.y_to_f64(dev.y), y_ref, "apply after a timed-out wait")
+
+
+def test_host_side_argument_checks_of_the_backward_and_the_grouped_moe_call():
+    from paper_2605_13779_b200 import binding as mb, harness
+    case = synth.random_dense_case("gpu/args-bwd", 16, 64, 64, 3, [2, 2, 2], 2, p_none=0.0)
+    dev = harness.upload_dense(case)
+    plan = mb.mint_lora_plan(dev.table, dev.ids, dev.status)
+    dy = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    dx = torch.zeros(16, 64, dtype=torch.bfloat16, device="cuda")
+    dA = torch.zeros(3, 2, 64, dtype=torch.float32, device="cuda")
+    dB = torch.zeros(3, 2, 64, dtype=torch.float32, device="cuda")
+    with pytest.raises(mb.MintError) as e:      # the weight gradients come together
+        mb.mint_lora_backward(dev.pool, dev.table, plan, dev.x, dy, dev.status, dx=dx, dA=dA, dB=None)
+    assert e.value.status == mb.MINT_ERR_INVALID_ARG
+    with pytest.raises(mb.MintError) as e:      # a workspace that is too small
+        mb.mint_lora_backward(dev.pool, dev.table, plan, dev.x, dy, dev.status, dx=dx, dA=dA, dB=dB,
+                              workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == mb.MINT_ERR_WORKSPACE_TOO_SMALL
+    moe_pool = mb.Pool(dev.pool.A, dev.pool.B, 64, 64, 2, 3, num_experts=1)
+    with pytest.raises(mb.MintError) as e:      # the backward takes rank-major pools only
+        mb.mint_lora_backward(moe_pool, dev.table, plan, dev.x, dy, dev.status, dx=dx, dA=dA, dB=dB)
+    assert e.value.status == mb.MINT_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert float(dA.abs().sum()) == 0.0 and float(dx.float().abs().sum()) == 0.0   # none of the refused calls ran
+
+    # grouped MoE call: pools with different expert counts, a dense pool among the items
+    batch = synth.config4_batch(T=8, E=4, K=2, num_slots=2, rank=8, tag="gpu/args-moe")
+    mcase = synth.config4_projection(batch, "gate", d=64, n=64, tag="gpu/args-moe")
+    mdev = harness.upload_moe(mcase)
+    mplan = mb.mint_lora_plan(mdev.table, mdev.ids, mdev.status, expert_ids=mdev.expert_ids, num_experts=4)
+    ws = mb.new_moe_workspace(mdev.pool, 8, 2)
+    fewer = mb.Pool(mdev.pool.A, mdev.pool.B, 64, 64, 8, 2, num_experts=2)
+    with pytest.raises(mb.MintError) as e:
+        mb.mint_moe_lora_apply_grouped([(mdev.pool, mdev.x, mdev.y, ws), (fewer, mdev.x, mdev.y, ws)], mdev.table,
+                                       mplan, mdev.status, x_row=mdev.x_row)
+    assert e.value.status == mb.MINT_ERR_SHAPE_MISMATCH
+    dense_pool = mb.Pool(mdev.pool.A, mdev.pool.B, 64, 64, 8, 2)
+    with pytest.raises(mb.MintError) as e:
+        mb.mint_moe_lora_apply_grouped([(dense_pool, mdev.x, mdev.y, ws)], mdev.table, mplan, mdev.status,
+                                       x_row=mdev.x_row)
+    assert e.value.status == mb.MINT_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(mb.bits_from_bf16(mdev.y), mcase.y0)
