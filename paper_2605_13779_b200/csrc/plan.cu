@@ -70,6 +70,31 @@ __device__ int block_exclusive_scan(int val, int *warp_tot /*[kWarps + 1]*/, int
   return warp_tot[warp] + inc - val;
 }
 
+// Ordered compaction over positions 0 .. n-1 walked 1024 at a time (coalesced): pass A stores, per
+// (chunk, warp), how many positions of the warp are flagged; scan_counts turns the counts into exclusive
+// prefix sums (and returns the total); pass B then gives every flagged position its rank as
+// cnt[chunk * 32 + warp] + the flagged lanes below it.  cnt holds chunks * 32 <= kCompactMax entries.
+constexpr int kCompactMax = kWarps * 256;   // the radix sort's histogram array, free once the sort is done
+__device__ int scan_counts(int32_t *cnt, int n_cnt, int *warp_tot) {
+  constexpr int kPer = kCompactMax / kThreads;   // 8 consecutive entries per thread
+  const int base = threadIdx.x * kPer;
+  int v[kPer], sum = 0;
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    v[q] = base + q < n_cnt ? cnt[base + q] : 0;
+    sum += v[q];
+  }
+  int total;
+  int run = block_exclusive_scan(sum, warp_tot, total);
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    if (base + q < n_cnt) cnt[base + q] = run;
+    run += v[q];
+  }
+  __syncthreads();
+  return total;
+}
+
 __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   __shared__ int32_t hist[kWarps][256];
   __shared__ int32_t bin_base[256];
@@ -200,12 +225,89 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   const int32_t *skey = (p.npass & 1) ? key_b : key_a;  // keys in sorted order
   const int n_active = P - counters[0];
 
-  // ---- segments: one per distinct key among the active prefix ----------------
+  // ---- segments and tile lists ------------------------------------------------------
   const int run_len = (P + kThreads - 1) / kThreads;
   const int r_begin = min(n_active, tid * run_len), r_end = min(n_active, (tid + 1) * run_len);
+  int S;
+  int tile_total[MINT_NUM_TILE_LISTS];
+  // dense segments (segmented prefill): dense plans of large batches only
+  const bool dense_plan = p.expert_ids == nullptr && P >= MINT_DENSE_MIN_BATCH;
+  auto tile_len = [&](int g, int sg) {   // the run length list g cuts segment sg into
+    const bool dense_seg = dense_plan && seg_start[sg + 1] - seg_start[sg] >= MINT_DENSE_MIN_SEGMENT;
+    return (p.tab.slot_rank[seg_slot[sg]] == 1 && !dense_seg) ? mint_tile_tokens_rank1(g) : mint_tile_tokens(g);
+  };
+  const int chunks = (n_active + kThreads - 1) / kThreads;
+  if (chunks * kWarps <= kCompactMax) {
+    // Coalesced walks (every batch of up to 262 144 items): a position is a segment head when its key
+    // differs from the one before it, and a tile head of list g when its offset in its segment is a
+    // multiple of the segment's run length.  Ordered compaction gives each head its index.
+    int32_t *cnt = &hist[0][0];
+    int32_t *seg_of = idx_a;   // segment of every position (the sort's scratch is free)
+    int32_t *seg_run = idx_b;  // per segment: run length of list 0 | run length of list 1 << 8
+    const unsigned below = (1u << lane) - 1u;
+    auto is_head = [&](int i) { return i < n_active && (i == 0 || skey[i] != skey[i - 1]); };
+    for (int c = 0; c < chunks; ++c) {
+      const unsigned b = __ballot_sync(0xffffffffu, is_head(c * kThreads + tid));
+      if (lane == 0) cnt[c * kWarps + warp] = __popc(b);
+    }
+    __syncthreads();
+    S = scan_counts(cnt, chunks * kWarps, warp_tot);
+    for (int c = 0; c < chunks; ++c) {
+      const int i = c * kThreads + tid;
+      const bool f = is_head(i);
+      const unsigned b = __ballot_sync(0xffffffffu, f);
+      const int seg = cnt[c * kWarps + warp] + __popc(b & below) + (f ? 1 : 0) - 1;   // heads at or before i, less one
+      if (i < n_active) seg_of[i] = seg;
+      if (f) {
+        const int32_t k = skey[i];
+        seg_start[seg] = i;
+        seg_key[seg] = k;
+        seg_slot[seg] = k % p.tab.num_slots;
+        seg_expert[seg] = k / p.tab.num_slots;
+      }
+    }
+    if (tid == 0) seg_start[S] = n_active;
+    __syncthreads();
+    for (int sg = tid; sg < S; sg += kThreads) {
+      atomicMax(&counters[5], seg_start[sg + 1] - seg_start[sg]);
+      atomicAdd(&counters[6], p.tab.slot_rank[seg_slot[sg]]);
+      seg_run[sg] = tile_len(0, sg) | (tile_len(1, sg) << 8);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
+      int32_t *tseg = reinterpret_cast<int32_t *>(p.blob + p.off.tile_seg[g]);
+      int32_t *toff = reinterpret_cast<int32_t *>(p.blob + p.off.tile_off[g]);
+      auto tile_head = [&](int i, int &sg) {
+        if (i >= n_active) return false;
+        sg = seg_of[i];
+        const int G = (seg_run[sg] >> (8 * g)) & 255;
+        return ((i - seg_start[sg]) % G) == 0;
+      };
+      for (int c = 0; c < chunks; ++c) {
+        int sg = 0;
+        const unsigned b = __ballot_sync(0xffffffffu, tile_head(c * kThreads + tid, sg));
+        if (lane == 0) cnt[c * kWarps + warp] = __popc(b);
+      }
+      __syncthreads();
+      tile_total[g] = scan_counts(cnt, chunks * kWarps, warp_tot);
+      for (int c = 0; c < chunks; ++c) {
+        const int i = c * kThreads + tid;
+        int sg = 0;
+        const bool f = tile_head(i, sg);
+        const unsigned b = __ballot_sync(0xffffffffu, f);
+        if (f) {
+          const int pos = cnt[c * kWarps + warp] + __popc(b & below);
+          tseg[pos] = sg;
+          toff[pos] = i;
+        }
+      }
+      __syncthreads();   // cnt is rewritten for the next list
+    }
+  } else {
+  // (larger batches: every thread walks a contiguous run of positions)
   int heads = 0;
   for (int i = r_begin; i < r_end; ++i) heads += (i == 0 || skey[i] != skey[i - 1]);
-  int S;
   int seg = block_exclusive_scan(heads, warp_tot, S);
   for (int i = r_begin; i < r_end; ++i) {
     const int32_t k = skey[i];
@@ -225,7 +327,6 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     atomicAdd(&counters[6], p.tab.slot_rank[seg_slot[s]]);
   }
 
-  // ---- derived tile lists: every segment cut into runs of at most G items ----
   // Position i starts a tile of list g when (i - start of its segment) % G == 0.
   int s0 = 0;
   if (r_begin < r_end) {  // segment containing r_begin: last s with seg_start[s] <= r_begin
@@ -236,13 +337,6 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     }
     s0 = lo;
   }
-  int tile_total[MINT_NUM_TILE_LISTS];
-  // dense segments (segmented prefill): dense plans of large batches only
-  const bool dense_plan = p.expert_ids == nullptr && P >= MINT_DENSE_MIN_BATCH;
-  auto tile_len = [&](int g, int sg) {   // the run length list g cuts segment sg into
-    const bool dense_seg = dense_plan && seg_start[sg + 1] - seg_start[sg] >= MINT_DENSE_MIN_SEGMENT;
-    return (p.tab.slot_rank[seg_slot[sg]] == 1 && !dense_seg) ? mint_tile_tokens_rank1(g) : mint_tile_tokens(g);
-  };
 #pragma unroll
   for (int g = 0; g < MINT_NUM_TILE_LISTS; ++g) {
     int cnt = 0, s = s0;
@@ -270,6 +364,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
         ++pos;
       }
     }
+  }
   }
   __syncthreads();
 
