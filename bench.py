@@ -401,6 +401,20 @@ def measure_side_workload(torch, dist, world, stream, name, peak):
            "roofline_frac": dw.layer_bytes / (ms_a * 1e-3 / dw.L) / 1e9 / peak,
            "roofline_frac_with_plan": dw.layer_bytes / (ms * 1e-3 / dw.L) / 1e9 / peak,
            "replay_footprint_MB": dw.layer_bytes * dw.L / 1e6}
+    if dw.moe:
+        # Routing differs from layer to layer of a MoE model, so a served layer needs a plan of its own:
+        # the same pass with one plan before every layer.
+        def plan_every_layer():
+            for li in range(dw.L):
+                dw.enqueue_plan()
+                dw.enqueue_layer(li, "layer")
+
+        gp = dw.capture(stream, plan_every_layer)
+        ms_p = time_graph(torch, dist, world, stream, gp, steps, 2) / steps
+        dw.check_status(name)
+        res["us_per_layer_plan_every_layer"] = ms_p * 1e3 / dw.L
+        res["roofline_frac_plan_every_layer"] = dw.layer_bytes / (ms_p * 1e-3 / dw.L) / 1e9 / peak
+        del gp
     if name != "config3":
         res["parity"] = parity_of_first_layer(dw, "layer")
     del g, ga, dw
