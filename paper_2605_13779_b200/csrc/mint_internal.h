@@ -134,8 +134,14 @@ struct PlanOffsets {
   int64_t lane_shrink; // LaneStart[MINT_MAX_LANES + 1]  start of cost lane j in the shrink rows
   int64_t lane_expand; // LaneStart[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
+  int64_t cta_hist;    // int32[16 + (ctas + 1) * (key_space + 1)]  counters, per-CTA key counts and key starts of the grid-wide sort
+                       // (only when mint_plan_presort_ctas(P, key_space) > 0)
   int64_t total;
 };
+// Batches of many items over a small key space are sorted by a counting sort that runs on one CTA per
+// 1024 items (three short kernels) before the single-CTA plan kernel derives the rest; returns the
+// number of those CTAs, or 0 when the plan kernel sorts by itself.
+int32_t mint_plan_presort_ctas(int64_t P, int64_t key_space);
 PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space);
 // Upper bound on the number of tiles of list g, computable without reading the plan.
 int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space);

@@ -37,6 +37,7 @@ struct PlanParams {
   int32_t npass;
   int32_t digit_bits;
   int32_t lanes;       // cost lanes G of the lane tables
+  int32_t presort_ctas;   // > 0: the grid-wide counting sort has left sorted keys in key_b and the order in perm
   PlanOffsets off;
   char *blob;
   int32_t *status;
@@ -95,6 +96,134 @@ __device__ int scan_counts(int32_t *cnt, int n_cnt, int *warp_tot) {
   return total;
 }
 
+// Key of item i (key_space: no adapter, or an error that is counted in cnt: 0 inactive, 1 not
+// resident, 2 first missing token, 3 bad expert, 4 first bad item).  kFromZero: the counters started
+// at zero (a memset), so the two minima are kept as maxima of 0x7fffffff - index.
+template <bool kFromZero>
+__device__ __forceinline__ int32_t item_key(const PlanParams &p, int i, int32_t *cnt) {
+  const int t = i / p.K;
+  const int64_t id = p.ids[t];
+  int32_t key = p.key_space;
+  if (id != -1) {
+    int32_t slot = -1;
+    if (id >= 0 && id < p.tab.catalog_size) slot = p.tab.id_to_slot[id];
+    if (slot < 0 || slot >= p.tab.num_slots) {
+      if (i == t * p.K) {
+        atomicAdd(&cnt[1], 1);
+        if (kFromZero) atomicMax(&cnt[2], 0x7fffffff - t); else atomicMin(&cnt[2], t);
+      }
+    } else if (p.expert_ids != nullptr) {
+      const int32_t e = p.expert_ids[i];
+      if (e < 0 || e >= p.E) {
+        atomicAdd(&cnt[3], 1);
+        if (kFromZero) atomicMax(&cnt[4], 0x7fffffff - i); else atomicMin(&cnt[4], i);
+      } else {
+        key = e * p.tab.num_slots + slot;
+      }
+    } else {
+      key = slot;
+    }
+  }
+  if (key == p.key_space) atomicAdd(&cnt[0], 1);
+  return key;
+}
+
+// ---- grid-wide stable counting sort (many items, small key space) ---------------
+// CTA c owns items [1024 c, 1024 c + 1024).  (1) keys and per-CTA key counts; (2) one CTA turns the
+// counts into start positions, key-major and CTA-minor; (3) every CTA places its items: the warps
+// take turns in warp order, and inside a warp an item's rank among equal keys is the number of
+// lower lanes with that key, so equal keys keep their item order whatever the scheduling.
+static_assert((mint_tile_tokens(0) & (mint_tile_tokens(0) - 1)) == 0 && (mint_tile_tokens(1) & (mint_tile_tokens(1) - 1)) == 0 &&
+                  mint_tile_tokens_rank1(0) == mint_tile_tokens(0) && (mint_tile_tokens_rank1(1) & (mint_tile_tokens_rank1(1) - 1)) == 0,
+              "the tile walks take run lengths as powers of two, and list 0 as one length");
+constexpr int kPresortMaxKeys = 4096;   // key_space of the counting sort (bins = key_space + 1)
+
+__global__ void __launch_bounds__(kThreads) presort_count_kernel(const PlanParams p) {
+  __shared__ int32_t bins[kPresortMaxKeys + 1];
+  int32_t *g = reinterpret_cast<int32_t *>(p.blob + p.off.cta_hist);
+  int32_t *key_a = reinterpret_cast<int32_t *>(p.blob + p.off.key_a);
+  const int nb = p.key_space + 1;
+  for (int b = threadIdx.x; b < nb; b += kThreads) bins[b] = 0;
+  __syncthreads();
+  const int i = blockIdx.x * kThreads + threadIdx.x;
+  if (i < p.P) {
+    const int32_t key = item_key<true>(p, i, g);
+    key_a[i] = key;
+    atomicAdd(&bins[key], 1);
+  }
+  __syncthreads();
+  int32_t *row = g + 16 + (size_t)blockIdx.x * nb;
+  for (int b = threadIdx.x; b < nb; b += kThreads) row[b] = bins[b];
+}
+
+__global__ void __launch_bounds__(kThreads) presort_scan_kernel(const PlanParams p) {
+  __shared__ int32_t base[kPresortMaxKeys + 1 + 8];
+  __shared__ int warp_tot[kWarps + 1];
+  int32_t *hist = reinterpret_cast<int32_t *>(p.blob + p.off.cta_hist) + 16;
+  const int nb = p.key_space + 1, C = p.presort_ctas;
+  for (int b = threadIdx.x; b < nb; b += kThreads) {   // counts -> offsets inside the key, CTA-minor
+    int run = 0;
+    for (int c0 = 0; c0 < C; c0 += 16) {   // (sixteen loads go out together)
+      int v[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) v[q] = c0 + q < C ? __ldcg(hist + (size_t)(c0 + q) * nb + b) : 0;
+#pragma unroll
+      for (int q = 0; q < 16; ++q) {
+        if (c0 + q < C) hist[(size_t)(c0 + q) * nb + b] = run;
+        run += v[q];
+      }
+    }
+    base[b] = run;
+  }
+  __syncthreads();
+  constexpr int kPer = (kPresortMaxKeys + 1 + kThreads - 1) / kThreads;   // consecutive keys per thread
+  const int b0 = threadIdx.x * kPer;
+  int v[kPer], sum = 0;
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    v[q] = b0 + q < nb ? base[b0 + q] : 0;
+    sum += v[q];
+  }
+  int total;
+  int run = block_exclusive_scan(sum, warp_tot, total);
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    if (b0 + q < nb) base[b0 + q] = run;
+    run += v[q];
+  }
+  __syncthreads();
+  // row C of the table: where every key starts; the placing CTAs add it to their own row
+  for (int b = threadIdx.x; b < nb; b += kThreads) hist[(size_t)C * nb + b] = base[b];
+}
+
+__global__ void __launch_bounds__(kThreads) presort_place_kernel(const PlanParams p) {
+  __shared__ int32_t next[kPresortMaxKeys + 1];
+  const int32_t *hist = reinterpret_cast<const int32_t *>(p.blob + p.off.cta_hist) + 16;
+  const int32_t *key_a = reinterpret_cast<const int32_t *>(p.blob + p.off.key_a);
+  int32_t *key_b = reinterpret_cast<int32_t *>(p.blob + p.off.key_b);
+  int32_t *perm = reinterpret_cast<int32_t *>(p.blob + p.off.perm);
+  const int nb = p.key_space + 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b = threadIdx.x; b < nb; b += kThreads)
+    next[b] = hist[(size_t)blockIdx.x * nb + b] + hist[(size_t)p.presort_ctas * nb + b];
+  const int i = blockIdx.x * kThreads + threadIdx.x;
+  const bool live = i < p.P;
+  const int32_t key = live ? key_a[i] : -1;
+  const uint32_t grp = __match_any_sync(0xffffffffu, key);
+  const int rank = __popc(grp & ((1u << lane) - 1u));
+  __syncthreads();
+  for (int w = 0; w < kWarps; ++w) {
+    if (warp == w && live) {
+      const int pos = next[key] + rank;
+      key_b[pos] = key;
+      perm[pos] = i;
+    }
+    __syncwarp();
+    if (warp == w && live && rank == 0) next[key] += __popc(grp);
+    __syncthreads();
+  }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   __shared__ int32_t hist[kWarps][256];
   __shared__ int32_t bin_base[256];
@@ -120,32 +249,11 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   __syncthreads();
 
   // ---- keys: id -> slot through the table, (expert, slot) -> key ----------
-  for (int i = tid; i < P; i += kThreads) {
-    const int t = i / p.K;
-    const int64_t id = p.ids[t];
-    int32_t key = p.key_space;
-    if (id != -1) {
-      int32_t slot = -1;
-      if (id >= 0 && id < p.tab.catalog_size) slot = p.tab.id_to_slot[id];
-      if (slot < 0 || slot >= p.tab.num_slots) {
-        if (i == t * p.K) {
-          atomicAdd(&counters[1], 1);
-          atomicMin(&counters[2], t);
-        }
-      } else if (p.expert_ids != nullptr) {
-        const int32_t e = p.expert_ids[i];
-        if (e < 0 || e >= p.E) {
-          atomicAdd(&counters[3], 1);
-          atomicMin(&counters[4], i);
-        } else {
-          key = e * p.tab.num_slots + slot;
-        }
-      } else {
-        key = slot;
-      }
-    }
-    if (key == p.key_space) atomicAdd(&counters[0], 1);
-    key_a[i] = key;
+  if (p.presort_ctas > 0) {   // done by the grid-wide sort, with its counters
+    const int32_t *g = reinterpret_cast<const int32_t *>(p.blob + p.off.cta_hist);
+    if (tid < 5) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff - g[tid] : g[tid];
+  } else {
+    for (int i = tid; i < P; i += kThreads) key_a[i] = item_key<false>(p, i, counters);
   }
   __syncthreads();
 
@@ -153,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   const int R = (((P + kWarps - 1) / kWarps + 31) / 32) * 32;  // items per warp, multiple of 32
   const int w_begin = min(P, warp * R), w_end = min(P, (warp + 1) * R);
   const int nbins = 1 << p.digit_bits;
-  for (int pass = 0; pass < p.npass; ++pass) {
+  for (int pass = 0; pass < (p.presort_ctas > 0 ? 0 : p.npass); ++pass) {
     const int32_t *kin = (pass & 1) ? key_b : key_a;
     int32_t *kout = (pass & 1) ? key_a : key_b;
     const int32_t *iin = (pass & 1) ? idx_b : idx_a;  // unused in pass 0 (index = position)
@@ -222,7 +330,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     }
     __syncthreads();
   }
-  const int32_t *skey = (p.npass & 1) ? key_b : key_a;  // keys in sorted order
+  const int32_t *skey = (p.presort_ctas > 0 || (p.npass & 1)) ? key_b : key_a;  // keys in sorted order
   const int n_active = P - counters[0];
 
   // ---- segments and tile lists ------------------------------------------------------
@@ -246,24 +354,44 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     int32_t *seg_run = idx_b;  // per segment: run length of list 0 | run length of list 1 << 8
     const unsigned below = (1u << lane) - 1u;
     auto is_head = [&](int i) { return i < n_active && (i == 0 || skey[i] != skey[i - 1]); };
-    for (int c = 0; c < chunks; ++c) {
-      const unsigned b = __ballot_sync(0xffffffffu, is_head(c * kThreads + tid));
-      if (lane == 0) cnt[c * kWarps + warp] = __popc(b);
+    // (kU chunks per step: the loads that decide their flags go out together)
+    constexpr int kU = 4;
+    for (int c0 = 0; c0 < chunks; c0 += kU) {
+      bool f[kU];
+#pragma unroll
+      for (int q = 0; q < kU; ++q) f[q] = is_head((c0 + q) * kThreads + tid);
+#pragma unroll
+      for (int q = 0; q < kU; ++q) {
+        const unsigned b = __ballot_sync(0xffffffffu, f[q]);
+        if (lane == 0 && c0 + q < chunks) cnt[(c0 + q) * kWarps + warp] = __popc(b);
+      }
     }
     __syncthreads();
     S = scan_counts(cnt, chunks * kWarps, warp_tot);
-    for (int c = 0; c < chunks; ++c) {
-      const int i = c * kThreads + tid;
-      const bool f = is_head(i);
-      const unsigned b = __ballot_sync(0xffffffffu, f);
-      const int seg = cnt[c * kWarps + warp] + __popc(b & below) + (f ? 1 : 0) - 1;   // heads at or before i, less one
-      if (i < n_active) seg_of[i] = seg;
-      if (f) {
-        const int32_t k = skey[i];
-        seg_start[seg] = i;
-        seg_key[seg] = k;
-        seg_slot[seg] = k % p.tab.num_slots;
-        seg_expert[seg] = k / p.tab.num_slots;
+    for (int c0 = 0; c0 < chunks; c0 += kU) {
+      bool f[kU];
+      int32_t k[kU];
+#pragma unroll
+      for (int q = 0; q < kU; ++q) {
+        const int i = (c0 + q) * kThreads + tid;
+        f[q] = is_head(i);
+        k[q] = i < n_active ? skey[i] : 0;
+      }
+#pragma unroll
+      for (int q = 0; q < kU; ++q) {
+        const int i = (c0 + q) * kThreads + tid;
+        const unsigned b = __ballot_sync(0xffffffffu, f[q]);
+        if (i < n_active) {
+          // heads at or before i, less one
+          const int seg = cnt[(c0 + q) * kWarps + warp] + __popc(b & below) + (f[q] ? 1 : 0) - 1;
+          seg_of[i] = seg;
+          if (f[q]) {
+            seg_start[seg] = i;
+            seg_key[seg] = k[q];
+            seg_slot[seg] = k[q] % p.tab.num_slots;
+            seg_expert[seg] = k[q] / p.tab.num_slots;
+          }
+        }
       }
     }
     if (tid == 0) seg_start[S] = n_active;
@@ -281,25 +409,41 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
       auto tile_head = [&](int i, int &sg) {
         if (i >= n_active) return false;
         sg = seg_of[i];
-        const int G = (seg_run[sg] >> (8 * g)) & 255;
-        return ((i - seg_start[sg]) % G) == 0;
+        // (run lengths are powers of two; list 0 cuts every segment alike)
+        const int G = g == 0 ? mint_tile_tokens(0) : (seg_run[sg] >> 8) & 255;
+        return ((i - seg_start[sg]) & (G - 1)) == 0;
       };
-      for (int c = 0; c < chunks; ++c) {
-        int sg = 0;
-        const unsigned b = __ballot_sync(0xffffffffu, tile_head(c * kThreads + tid, sg));
-        if (lane == 0) cnt[c * kWarps + warp] = __popc(b);
+      for (int c0 = 0; c0 < chunks; c0 += kU) {
+        bool f[kU];
+#pragma unroll
+        for (int q = 0; q < kU; ++q) {
+          int sg = 0;
+          f[q] = tile_head((c0 + q) * kThreads + tid, sg);
+        }
+#pragma unroll
+        for (int q = 0; q < kU; ++q) {
+          const unsigned b = __ballot_sync(0xffffffffu, f[q]);
+          if (lane == 0 && c0 + q < chunks) cnt[(c0 + q) * kWarps + warp] = __popc(b);
+        }
       }
       __syncthreads();
       tile_total[g] = scan_counts(cnt, chunks * kWarps, warp_tot);
-      for (int c = 0; c < chunks; ++c) {
-        const int i = c * kThreads + tid;
-        int sg = 0;
-        const bool f = tile_head(i, sg);
-        const unsigned b = __ballot_sync(0xffffffffu, f);
-        if (f) {
-          const int pos = cnt[c * kWarps + warp] + __popc(b & below);
-          tseg[pos] = sg;
-          toff[pos] = i;
+      for (int c0 = 0; c0 < chunks; c0 += kU) {
+        bool f[kU];
+        int sg[kU];
+#pragma unroll
+        for (int q = 0; q < kU; ++q) {
+          sg[q] = 0;
+          f[q] = tile_head((c0 + q) * kThreads + tid, sg[q]);
+        }
+#pragma unroll
+        for (int q = 0; q < kU; ++q) {
+          const unsigned b = __ballot_sync(0xffffffffu, f[q]);
+          if (f[q]) {
+            const int pos = cnt[(c0 + q) * kWarps + warp] + __popc(b & below);
+            tseg[pos] = sg[q];
+            toff[pos] = (c0 + q) * kThreads + tid;
+          }
         }
       }
       __syncthreads();   // cnt is rewritten for the next list
@@ -533,8 +677,16 @@ PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
   o.key_b = take(n);
   o.idx_a = take(n);
   o.idx_b = take(n);
+  o.cta_hist = cur;
+  const int64_t ctas = mint_plan_presort_ctas(P, key_space);
+  if (ctas > 0) o.cta_hist = take(16 + (ctas + 1) * (key_space + 1));
   o.total = cur;
   return o;
+}
+
+int32_t mint_plan_presort_ctas(int64_t P, int64_t key_space) {
+  if (P < 4096 || P > 256 * (int64_t)kThreads || key_space > kPresortMaxKeys) return 0;
+  return (int32_t)((P + kThreads - 1) / kThreads);
 }
 
 int64_t mint_tile_upper_bound(int g, int64_t P, int64_t key_space) {
@@ -586,6 +738,15 @@ int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, con
   p.off = mint_plan_offsets(p.P, p.key_space);
   p.blob = static_cast<char *>(plan_dev);
   p.status = status;
+  p.presort_ctas = mint_plan_presort_ctas(p.P, p.key_space);
+  if (p.presort_ctas > 0) {
+    int32_t st = mint_check_cuda(cudaMemsetAsync(p.blob + p.off.cta_hist, 0, 64, stream), "plan counters");
+    if (st) return st;
+    presort_count_kernel<<<p.presort_ctas, kThreads, 0, stream>>>(p);
+    presort_scan_kernel<<<1, kThreads, 0, stream>>>(p);
+    presort_place_kernel<<<p.presort_ctas, kThreads, 0, stream>>>(p);
+    if ((st = mint_check_cuda(cudaGetLastError(), "plan sort launch"))) return st;
+  }
   plan_kernel<<<1, kThreads, 0, stream>>>(p);
   return mint_check_cuda(cudaGetLastError(), "plan kernel launch");
 }
