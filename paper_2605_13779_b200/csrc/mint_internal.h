@@ -134,7 +134,7 @@ struct PlanOffsets {
   int64_t lane_shrink; // LaneStart[MINT_MAX_LANES + 1]  start of cost lane j in the shrink rows
   int64_t lane_expand; // LaneStart[MINT_MAX_LANES + 1]  same for the expand rows
   int64_t key_a, key_b, idx_a, idx_b;     // int32[P]  radix-sort ping-pong scratch
-  int64_t cta_hist;    // int32[16 + (ctas + 1) * (key_space + 1)]  counters, per-CTA key counts and key starts of the grid-wide sort
+  int64_t cta_hist;    // int32[16 + (ctas + 4) * (key_space + 1)]  counters, per-CTA key counts and per-key starts, segment and first tiles of the grid-wide sort
                        // (only when mint_plan_presort_ctas(P, key_space) > 0)
   int64_t total;
 };

@@ -194,6 +194,62 @@ __global__ void __launch_bounds__(kThreads) presort_scan_kernel(const PlanParams
   __syncthreads();
   // row C of the table: where every key starts; the placing CTAs add it to their own row
   for (int b = threadIdx.x; b < nb; b += kThreads) hist[(size_t)C * nb + b] = base[b];
+
+  // A key that has items is a segment, and its tiles follow from its item count: segments, and per
+  // key the segment index and the first tile of either list (rows C + 1 .. C + 3; the placing CTAs
+  // write the tile lists from them).  v[q] still holds the item count of key b0 + q.
+  int32_t *g = reinterpret_cast<int32_t *>(p.blob + p.off.cta_hist);
+  int32_t *seg_start = reinterpret_cast<int32_t *>(p.blob + p.off.seg_start);
+  int32_t *seg_key = reinterpret_cast<int32_t *>(p.blob + p.off.seg_key);
+  int32_t *seg_slot = reinterpret_cast<int32_t *>(p.blob + p.off.seg_slot);
+  int32_t *seg_expert = reinterpret_cast<int32_t *>(p.blob + p.off.seg_expert);
+  const bool dense_plan = p.expert_ids == nullptr && p.P >= MINT_DENSE_MIN_BATCH;
+  int run1[kPer], n0 = 0, n1 = 0, ns = 0, max_seg = 0, sum_rank = 0;
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    run1[q] = mint_tile_tokens(1);
+    if (b0 + q >= p.key_space || v[q] == 0) {   // (the last bin holds the items without an adapter)
+      v[q] = 0;
+      continue;
+    }
+    const int rank = p.tab.slot_rank[(b0 + q) % p.tab.num_slots];
+    const bool dense_seg = dense_plan && v[q] >= MINT_DENSE_MIN_SEGMENT;
+    if (rank == 1 && !dense_seg) run1[q] = mint_tile_tokens_rank1(1);
+    ns += 1;
+    n0 += (v[q] + mint_tile_tokens(0) - 1) / mint_tile_tokens(0);
+    n1 += (v[q] + run1[q] - 1) / run1[q];
+    max_seg = max(max_seg, v[q]);
+    sum_rank += rank;
+  }
+  int S, T0, T1;
+  int seg = block_exclusive_scan(ns, warp_tot, S);
+  int t0 = block_exclusive_scan(n0, warp_tot, T0);
+  int t1 = block_exclusive_scan(n1, warp_tot, T1);
+  int32_t *row_seg = hist + (size_t)(C + 1) * nb, *row_t0 = hist + (size_t)(C + 2) * nb,
+          *row_t1 = hist + (size_t)(C + 3) * nb;
+#pragma unroll
+  for (int q = 0; q < kPer; ++q) {
+    if (v[q] == 0) continue;
+    const int b = b0 + q;
+    row_seg[b] = seg;
+    row_t0[b] = t0;
+    row_t1[b] = t1 | (run1[q] << 24);
+    seg_start[seg] = base[b];
+    seg_key[seg] = b;
+    seg_slot[seg] = b % p.tab.num_slots;
+    seg_expert[seg] = b / p.tab.num_slots;
+    seg += 1;
+    t0 += (v[q] + mint_tile_tokens(0) - 1) / mint_tile_tokens(0);
+    t1 += (v[q] + run1[q] - 1) / run1[q];
+  }
+  if (max_seg > 0) atomicMax(&g[5], max_seg);
+  if (sum_rank > 0) atomicAdd(&g[6], sum_rank);
+  if (threadIdx.x == 0) {
+    seg_start[S] = base[p.key_space];   // the active items
+    g[7] = S;
+    g[8] = T0;
+    g[9] = T1;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads) presort_place_kernel(const PlanParams p) {
@@ -202,6 +258,10 @@ __global__ void __launch_bounds__(kThreads) presort_place_kernel(const PlanParam
   const int32_t *key_a = reinterpret_cast<const int32_t *>(p.blob + p.off.key_a);
   int32_t *key_b = reinterpret_cast<int32_t *>(p.blob + p.off.key_b);
   int32_t *perm = reinterpret_cast<int32_t *>(p.blob + p.off.perm);
+  int32_t *tseg0 = reinterpret_cast<int32_t *>(p.blob + p.off.tile_seg[0]);
+  int32_t *toff0 = reinterpret_cast<int32_t *>(p.blob + p.off.tile_off[0]);
+  int32_t *tseg1 = reinterpret_cast<int32_t *>(p.blob + p.off.tile_seg[1]);
+  int32_t *toff1 = reinterpret_cast<int32_t *>(p.blob + p.off.tile_off[1]);
   const int nb = p.key_space + 1;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int b = threadIdx.x; b < nb; b += kThreads)
@@ -212,15 +272,32 @@ __global__ void __launch_bounds__(kThreads) presort_place_kernel(const PlanParam
   const uint32_t grp = __match_any_sync(0xffffffffu, key);
   const int rank = __popc(grp & ((1u << lane) - 1u));
   __syncthreads();
+  // the warps take their positions in warp order (shared memory only); the stores follow, all at once
+  int pos = 0;
   for (int w = 0; w < kWarps; ++w) {
-    if (warp == w && live) {
-      const int pos = next[key] + rank;
-      key_b[pos] = key;
-      perm[pos] = i;
-    }
+    if (warp == w && live) pos = next[key] + rank;
     __syncwarp();
     if (warp == w && live && rank == 0) next[key] += __popc(grp);
     __syncthreads();
+  }
+  if (!live) return;
+  key_b[pos] = key;
+  perm[pos] = i;
+  if (key < p.key_space) {   // the first item of a tile lists the tile
+    const int32_t *rows = hist + (size_t)p.presort_ctas * nb + key;   // start, segment, first tiles of the key
+    const int off = pos - __ldg(rows);
+    const int seg = __ldg(rows + nb), c0 = __ldg(rows + 2 * (size_t)nb), w1 = __ldg(rows + 3 * (size_t)nb);
+    const int run1 = w1 >> 24;
+    if ((off & (mint_tile_tokens(0) - 1)) == 0) {
+      const int c = c0 + off / mint_tile_tokens(0);
+      tseg0[c] = seg;
+      toff0[c] = pos;
+    }
+    if ((off & (run1 - 1)) == 0) {
+      const int c = (w1 & 0xffffff) + (off >> (31 - __clz(run1)));
+      tseg1[c] = seg;
+      toff1[c] = pos;
+    }
   }
 }
 
@@ -251,7 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
   // ---- keys: id -> slot through the table, (expert, slot) -> key ----------
   if (p.presort_ctas > 0) {   // done by the grid-wide sort, with its counters
     const int32_t *g = reinterpret_cast<const int32_t *>(p.blob + p.off.cta_hist);
-    if (tid < 5) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff - g[tid] : g[tid];
+    if (tid < 5) counters[tid] = (tid == 2 || tid == 4) ? 0x7fffffff - g[tid] : g[tid];   // (5, 6: further down)
   } else {
     for (int i = tid; i < P; i += kThreads) key_a[i] = item_key<false>(p, i, counters);
   }
@@ -345,7 +422,17 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
     return (p.tab.slot_rank[seg_slot[sg]] == 1 && !dense_seg) ? mint_tile_tokens_rank1(g) : mint_tile_tokens(g);
   };
   const int chunks = (n_active + kThreads - 1) / kThreads;
-  if (chunks * kWarps <= kCompactMax) {
+  if (p.presort_ctas > 0) {
+    // the grid-wide sort has also written the segments and both tile lists (a key with items is a segment)
+    const int32_t *g = reinterpret_cast<const int32_t *>(p.blob + p.off.cta_hist);
+    S = g[7];
+    tile_total[0] = g[8];
+    tile_total[1] = g[9];
+    if (tid == 0) {
+      counters[5] = g[5];
+      counters[6] = g[6];
+    }
+  } else if (chunks * kWarps <= kCompactMax) {
     // Coalesced walks (every batch of up to 262 144 items): a position is a segment head when its key
     // differs from the one before it, and a tile head of list g when its offset in its segment is a
     // multiple of the segment's run length.  Ordered compaction gives each head its index.
@@ -679,7 +766,7 @@ PlanOffsets mint_plan_offsets(int64_t P, int64_t key_space) {
   o.idx_b = take(n);
   o.cta_hist = cur;
   const int64_t ctas = mint_plan_presort_ctas(P, key_space);
-  if (ctas > 0) o.cta_hist = take(16 + (ctas + 1) * (key_space + 1));
+  if (ctas > 0) o.cta_hist = take(16 + (ctas + 4) * (key_space + 1));
   o.total = cur;
   return o;
 }

@@ -116,3 +116,33 @@ def test_plan_is_deterministic():
     a2, _ = gpu_plan(b.ids, b.table, b.expert_ids, b.E)
     for k in ("perm", "seg_start", "seg_key"):
         np.testing.assert_array_equal(a1[k], a2[k])
+
+
+@pytest.mark.parametrize("T,K,E,num_slots", [(4096, 1, 0, 7), (5000, 1, 0, 4096), (18439, 1, 0, 32), (600, 8, 128, 16),
+                                              (4096, 8, 128, 32), (1111, 6, 60, 64), (262144, 1, 0, 3)])
+def test_plans_of_the_grid_wide_sort(T, K, E, num_slots):
+    """Batches of 4096 .. 262 144 items over at most 4096 keys are sorted by the counting sort that
+    runs on one CTA per 1024 items: tokens without an adapter, ids that are not resident, expert ids
+    out of range, ranks 1 and above side by side, and a segment long enough for the dense tiles."""
+    from paper_2605_13779_b200 import binding as mb
+    rng = synth.stream("gpu/plan/grid", T, K, E, num_slots)
+    ids = rng.integers(0, num_slots, size=T).astype(np.int64)
+    ids[rng.random(T) < 0.3] = 0                       # one long segment
+    ids[rng.random(T) < 0.05] = -1
+    ranks = rng.choice(np.array([1, 8, 16], dtype=np.int32), size=num_slots)
+    table = synth.identity_table(num_slots, ranks)
+    table.id_to_slot = rng.permutation(num_slots).astype(np.int32)
+    if num_slots > 4:
+        table.id_to_slot[rng.integers(0, num_slots, size=2)] = -1      # two catalog ids without a slot
+    ex = None
+    if E:
+        ex = np.stack([rng.permutation(E)[:K] for _ in range(T)]).astype(np.int32)
+        ex[T // 3, K - 1] = E + 5
+        ex[T // 2, 0] = -1
+    got, ref, status = check(ids, table, ex, E)
+    assert got["sum_rank"] == int(ranks[ref["seg_key"] % num_slots].sum())
+    if ref["n_not_resident"]:
+        assert status[0] == mb.MINT_ERR_NOT_RESIDENT and status[1] == ref["n_not_resident"]
+        assert status[2] == int(np.nonzero((ids >= 0) & (table.id_to_slot[np.maximum(ids, 0)] < 0))[0][0])
+    elif E:
+        assert status[0] == mb.MINT_ERR_BAD_INDEX and got["n_bad_expert"] == 2
