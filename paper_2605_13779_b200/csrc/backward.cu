@@ -39,6 +39,12 @@ constexpr int kBlocksPerCta = 1;      // 512-column blocks of one tensor per CTA
 
 constexpr int kMaxJobs = 2 * MINT_MAX_GROUP;   // dA and dB of every projection of a grouped call
 
+// Programmatic dependent launch: the next kernel of the stream may become resident at once; data of
+// earlier kernels is touched only after the wait, which every CTA executes (completion stays
+// transitive along the stream).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 struct GradJob {
   const float *coef;      // [T][r_max] fp32, token order: u (for dA) or v (for dB)
   const uint16_t *act;    // [T][ld] bf16: x (for dA) or dy (for dB)
@@ -61,19 +67,27 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
   __shared__ int32_t tok[kTokenBatch];
   __shared__ float cf[kTokenBatch][kRankChunk];
   const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  // (before the wait: the plan and the slot table, complete before this call's first kernel started)
   if (!plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi,
-               (blockIdx.x == 0 && blockIdx.y == 0) ? P.status : nullptr))
+               (blockIdx.x == 0 && blockIdx.y == 0) ? P.status : nullptr)) {
+    pdl_wait();
     return;
+  }
   int ji = 0;   // the job this column block belongs to
   while (ji + 1 < P.njobs && (int)blockIdx.y >= P.job[ji + 1].block0) ++ji;
   const GradJob &p = P.job[ji];
   const int seg = blockIdx.x;
-  if (seg >= P.pv.header[PH_NUM_SEGMENTS]) return;
+  if (seg >= P.pv.header[PH_NUM_SEGMENTS]) {
+    pdl_wait();
+    return;
+  }
   const int off = P.pv.seg_start[seg], len = P.pv.seg_start[seg + 1] - off;
   const int slot = P.pv.seg_slot[seg];
   const int rank = P.tab.slot_rank[slot];
   const float scale = P.tab.slot_scale[slot];
   if (rank > p.r_max) {
+    pdl_wait();
     if (tid == 0) report(P.status, MINT_ERR_RANK_TOO_LARGE, slot);
     return;
   }
@@ -97,6 +111,7 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
       for (int k = 0; k < rank; ++k)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(out_slot + (size_t)k * p.width + col));
   }
+  pdl_wait();   // the coefficients, the activations and the gradients belong to earlier kernels until here
   for (int k0 = 0; k0 < rank; k0 += kRankChunk) {
     const int kc = min(kRankChunk, rank - k0);
     if (one_batch) stage(0, len, k0, kc);
@@ -169,6 +184,15 @@ int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, 
   P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
   const int64_t seg_ub = T < tab.num_slots ? T : tab.num_slots;
   const dim3 grid((unsigned)seg_ub, (unsigned)blocks);
-  grad_weight_kernel<<<grid, kThreads, 0, s>>>(P);
-  return mint_check_cuda(cudaGetLastError(), "grad_weight launch");
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cfg.attrs = attr;
+  // right after a plan or a bind kernel it waits for that kernel in full: it reads the plan at once
+  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, grad_weight_kernel, P), "grad_weight launch");
 }

@@ -1385,10 +1385,14 @@ struct GatherV {
 
 __global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constant__ StreamParams P, const GatherV out) {
   __shared__ int32_t part_first, part_count;
-  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi, nullptr)) return;
-  if (P.pv.header[PH_LANES] != P.lanes) return;
+  pdl_launch_dependents();
+  // (before the wait: only the plan, complete before the shrink kernel of this call started)
   const int t = blockIdx.x, p = blockIdx.y;
-  if (t >= P.pv.header[PH_NCHUNK1]) return;
+  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.num_experts, P.tab.gen_lo, P.tab.gen_hi, nullptr) ||
+      P.pv.header[PH_LANES] != P.lanes || t >= P.pv.header[PH_NCHUNK1]) {
+    pdl_wait();
+    return;
+  }
   const TileDesc d = P.pv.tile_desc[t];
   if (!d.dense) {
     const Area shrink_area = make_area<false>(P);
@@ -1399,6 +1403,7 @@ __global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constan
       part_count = count;
     }
   }
+  pdl_wait();   // the shrink kernels have completed: the parts are final
   __syncthreads();
   const int nel = d.len * d.rank;
   const StreamProblem &pb = P.prob[p];
@@ -1488,9 +1493,12 @@ int32_t mint_launch_stream_phases(const DenseArgs *args, int nprob, const TableD
       st = mint_launch_dense_shrink(args, nprob, tab, plan_dev, workspaces, lanes, P.dense_slot0, (int32_t)tiles, s);
       if (st) return st;
     }
-    if (v_out) {   // (an ordinary launch: it starts when the shrink kernels are complete)
-      gather_v_kernel<<<dim3((unsigned)tiles, (unsigned)nprob), kThreads, 0, s>>>(P, out);
-      if ((st = mint_check_cuda(cudaGetLastError(), "gather_v launch"))) return st;
+    if (v_out) {
+      cudaLaunchConfig_t gcfg = cfg;   // (it follows a shrink kernel of this call: programmatic launch)
+      gcfg.gridDim = dim3((unsigned)tiles, (unsigned)nprob);
+      gcfg.dynamicSmemBytes = 0;
+      gcfg.numAttrs = 1;
+      if ((st = mint_check_cuda(cudaLaunchKernelEx(&gcfg, gather_v_kernel, P, out), "gather_v launch"))) return st;
     }
   }
   if (!(phases & 2)) return MINT_OK;
