@@ -128,6 +128,11 @@ __device__ __forceinline__ int32_t item_key(const PlanParams &p, int i, int32_t 
   return key;
 }
 
+// Programmatic dependent launch between the kernels of one plan: a kernel lets its successor become
+// resident at once, and touches nothing before its own wait (which every CTA executes).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- grid-wide stable counting sort (many items, small key space) ---------------
 // CTA c owns items [1024 c, 1024 c + 1024).  (1) keys and per-CTA key counts; (2) one CTA turns the
 // counts into start positions, key-major and CTA-minor; (3) every CTA places its items: the warps
@@ -140,6 +145,8 @@ constexpr int kPresortMaxKeys = 4096;   // key_space of the counting sort (bins 
 
 __global__ void __launch_bounds__(kThreads) presort_count_kernel(const PlanParams p) {
   __shared__ int32_t bins[kPresortMaxKeys + 1];
+  pdl_launch_dependents();
+  pdl_wait();
   int32_t *g = reinterpret_cast<int32_t *>(p.blob + p.off.cta_hist);
   int32_t *key_a = reinterpret_cast<int32_t *>(p.blob + p.off.key_a);
   const int nb = p.key_space + 1;
@@ -159,6 +166,8 @@ __global__ void __launch_bounds__(kThreads) presort_count_kernel(const PlanParam
 __global__ void __launch_bounds__(kThreads) presort_scan_kernel(const PlanParams p) {
   __shared__ int32_t base[kPresortMaxKeys + 1 + 8];
   __shared__ int warp_tot[kWarps + 1];
+  pdl_launch_dependents();
+  pdl_wait();
   int32_t *hist = reinterpret_cast<int32_t *>(p.blob + p.off.cta_hist) + 16;
   const int nb = p.key_space + 1, C = p.presort_ctas;
   for (int b = threadIdx.x; b < nb; b += kThreads) {   // counts -> offsets inside the key, CTA-minor
@@ -254,6 +263,8 @@ __global__ void __launch_bounds__(kThreads) presort_scan_kernel(const PlanParams
 
 __global__ void __launch_bounds__(kThreads) presort_place_kernel(const PlanParams p) {
   __shared__ int32_t next[kPresortMaxKeys + 1];
+  pdl_launch_dependents();
+  pdl_wait();
   const int32_t *hist = reinterpret_cast<const int32_t *>(p.blob + p.off.cta_hist) + 16;
   const int32_t *key_a = reinterpret_cast<const int32_t *>(p.blob + p.off.key_a);
   int32_t *key_b = reinterpret_cast<int32_t *>(p.blob + p.off.key_b);
@@ -311,6 +322,7 @@ __global__ void __launch_bounds__(kThreads, 1) plan_kernel(const PlanParams p) {
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int P = p.P;
+  pdl_wait();   // (launched programmatically behind the grid-wide sort; otherwise returns at once)
   int32_t *hdr = reinterpret_cast<int32_t *>(p.blob + p.off.header);
   int32_t *perm = reinterpret_cast<int32_t *>(p.blob + p.off.perm);
   int32_t *seg_start = reinterpret_cast<int32_t *>(p.blob + p.off.seg_start);
@@ -829,10 +841,22 @@ int32_t mint_launch_plan(const TableDev &tab, const int64_t *ids, int32_t T, con
   if (p.presort_ctas > 0) {
     int32_t st = mint_check_cuda(cudaMemsetAsync(p.blob + p.off.cta_hist, 0, 64, stream), "plan counters");
     if (st) return st;
-    presort_count_kernel<<<p.presort_ctas, kThreads, 0, stream>>>(p);
-    presort_scan_kernel<<<1, kThreads, 0, stream>>>(p);
-    presort_place_kernel<<<p.presort_ctas, kThreads, 0, stream>>>(p);
-    if ((st = mint_check_cuda(cudaGetLastError(), "plan sort launch"))) return st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kThreads);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3((unsigned)p.presort_ctas);
+    if ((st = mint_check_cuda(cudaLaunchKernelEx(&cfg, presort_count_kernel, p), "plan sort (count) launch"))) return st;
+    cfg.gridDim = dim3(1);
+    if ((st = mint_check_cuda(cudaLaunchKernelEx(&cfg, presort_scan_kernel, p), "plan sort (scan) launch"))) return st;
+    cfg.gridDim = dim3((unsigned)p.presort_ctas);
+    if ((st = mint_check_cuda(cudaLaunchKernelEx(&cfg, presort_place_kernel, p), "plan sort (place) launch"))) return st;
+    cfg.gridDim = dim3(1);
+    return mint_check_cuda(cudaLaunchKernelEx(&cfg, plan_kernel, p), "plan kernel launch");
   }
   plan_kernel<<<1, kThreads, 0, stream>>>(p);
   return mint_check_cuda(cudaGetLastError(), "plan kernel launch");
