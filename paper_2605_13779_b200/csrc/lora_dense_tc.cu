@@ -567,13 +567,14 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
 // 128-byte-swizzled layout.  B is used as it lies in memory (columns contiguous): its
 // shared-memory descriptor names the MN-major layout, so nothing is transposed.  One
 // thread issues the MMAs of a chunk as soon as its B has landed, into one of two
-// accumulators in tensor memory.  Four warps add the accumulator to the y tile in shared
-// memory (tcgen05.ld, one row per thread) and hand the tile to a tensor-map store (full
-// tiles) or store its rows themselves (a segment's last, shorter tile: the rows beyond it
-// belong to another CTA).  Three buffers of B and y, two accumulators: the loads and the MMAs of chunk
+// accumulators in tensor memory.  Eight warps add the accumulator to the y tile in shared
+// memory (tcgen05.ld, one row x 64 columns per thread) and store its rows themselves when the
+// tile is a segment's last, shorter one (the rows beyond it belong to another CTA); a thread
+// of a warp of its own hands full tiles to a tensor-map store and returns the buffer when the
+// copy engine has read it, so the epilogue warps never wait for a store.  Three buffers of B and y, two accumulators: the loads and the MMAs of chunk
 // kc + 1 run under the epilogue of chunk kc.  Every wait is bounded.
 constexpr int kEpiThreads = 256;                   // 8 epilogue warps: warp w takes rows 32 (w % 4) .., columns 64 (w / 4) .. of a chunk
-constexpr int kTmaThreads = kEpiThreads + 64;      // + the producer's warp and the MMA warp
+constexpr int kTmaThreads = kEpiThreads + 96;      // + the producer's warp, the MMA warp and the warp that stores
 constexpr int kBHalfBytes = kMaxRank * 128;        // 64 ranks x 64 columns
 constexpr int kBBufBytes = 2 * kBHalfBytes;        // 16 KB
 constexpr int kYHalfBytes = kTileRows * 128;       // 128 rows x 64 columns
@@ -727,6 +728,30 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
       mbar_wait(&drain, 0);
     }
     __syncwarp();
+  } else if (warp == kEpiThreads / 32 + 2) {
+    // ---- storing thread: a finished y tile goes back through the tensor map, and its buffer is handed
+    // back once the copy engine has read it (the epilogue warps are on the next chunk meanwhile) ----
+    if (lane == 0) {
+      for (int kc = 0; kc < nchunks; ++kc) {
+        const int b = kc % kBufs;
+        const uint32_t par = (kc / kBufs) & 1u;
+        if (!mbar_wait(&y_written[b], par)) {
+          failed = 1;
+          break;
+        }
+        if (full_tile) {   // (columns beyond n are clipped by the tensor map; short tiles were stored row by row)
+          const int col0 = col_begin + kc * kExpChunk;
+          const uint32_t yb = y_buf + (uint32_t)(b * kYBufBytes);
+          tma_store_2d(&pb.y_map, col0, row0, yb);
+          tma_store_2d(&pb.y_map, col0 + 64, row0, yb + (uint32_t)kYHalfBytes);
+          bulk_commit();
+          bulk_wait_read();   // the tile has been read: the buffer may be refilled
+        }
+        mbar_arrive(&y_free[b]);
+      }
+      bulk_wait_all();   // the stores are complete before the kernel ends
+    }
+    __syncwarp();
   } else {
     // ---- epilogue warps; first v, scaled, as head and remainder (consecutive threads: consecutive rank pairs of a row) ----
     {
@@ -821,23 +846,9 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
           }
         }
       }
-      fence_async_smem();   // this thread's writes to the tile are visible to the store below
+      fence_async_smem();   // this thread's writes to the tile are visible to the store of the storing warp
       mbar_arrive(&y_written[b]);
-      if (tid == 0) {
-        if (!mbar_wait(&y_written[b], par)) {
-          failed = 1;
-          break;
-        }
-        if (full_tile) {   // (columns beyond n are clipped by the tensor map)
-          tma_store_2d(&pb.y_map, col0, row0, yb);
-          tma_store_2d(&pb.y_map, col0 + 64, row0, yb + (uint32_t)kYHalfBytes);
-          bulk_commit();
-          bulk_wait_read();   // the tile has been read: the buffer may be refilled
-        }
-        mbar_arrive(&y_free[b]);
-      }
     }
-    if (tid == 0) bulk_wait_all();   // the stores are complete before the kernel ends
   }
   __syncthreads();
   if (failed && tid == 0) report(P.status, MINT_ERR_TIMEOUT, m);
