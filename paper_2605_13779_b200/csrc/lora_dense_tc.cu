@@ -57,6 +57,7 @@ struct DenseProblem {
 
 struct DenseParams {
   DenseProblem prob[kMaxProblems];
+  int32_t nprob;
   int32_t T;
   int32_t lanes;
   int32_t dense_slot0;   // part s of the v of dense tile t goes to workspace slot dense_slot0 + s * dense_stride + t
@@ -78,8 +79,10 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_
   __shared__ int32_t rows[kTileRows];
   __shared__ volatile int32_t failed;   // written after a wait that ran out; read only after a CTA barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const DenseProblem &pb = P.prob[blockIdx.y / MINT_DENSE_SPLIT_MAX];
-  const int split = blockIdx.y % MINT_DENSE_SPLIT_MAX;
+  // the grid's second dimension runs over the shares of d of all problems laid end to end
+  int split = blockIdx.y, z = 0;
+  while (z + 1 < P.nprob && split >= P.prob[z].splits) split -= P.prob[z++].splits;
+  const DenseProblem &pb = P.prob[z];
 
   pdl_launch_dependents();
   // The plan and the pool weights were complete before this call's kernels
@@ -311,6 +314,7 @@ struct DenseExpandProblem {
 };
 struct DenseExpandParams {
   DenseExpandProblem prob[kMaxProblems];
+  int32_t nprob;
   int32_t T;
   int32_t lanes;
   int32_t dense_slot0;
@@ -319,6 +323,20 @@ struct DenseExpandParams {
   TableDev tab;
   PlanView pv;
 };
+
+// The grid's second dimension runs over the column ranges of all problems laid end to end (a
+// narrow problem then brings no CTAs that only exit): problem and first column of range y.
+__device__ __forceinline__ int expand_range(const DenseExpandParams &P, int y, int &col_begin) {
+  int z = 0;
+  while (z + 1 < P.nprob) {
+    const int ranges = (P.prob[z].n + kColsPerCta - 1) / kColsPerCta;
+    if (y < ranges) break;
+    y -= ranges;
+    ++z;
+  }
+  col_begin = y * kColsPerCta;
+  return z;
+}
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -350,13 +368,13 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
   __shared__ int32_t rows[kTileRows];
   __shared__ volatile int32_t failed;   // written after a wait that ran out; read only after a CTA barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const DenseExpandProblem &pb = P.prob[blockIdx.z];
+  int col_begin;
+  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin)];
 
   pdl_launch_dependents();
   const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
                   P.pv.header[PH_LANES] == P.lanes;
   const int m = blockIdx.x;
-  const int col_begin = blockIdx.y * kColsPerCta;
   // (with tensor maps this kernel is left the tiles whose tokens are scattered: usually none)
   if (!ok || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n ||
       (pb.use_tma && P.pv.header[PH_NUM_SCATTERED] == 0)) {
@@ -579,7 +597,7 @@ constexpr int kBHalfBytes = kMaxRank * 128;        // 64 ranks x 64 columns
 constexpr int kBBufBytes = 2 * kBHalfBytes;        // 16 KB
 constexpr int kYHalfBytes = kTileRows * 128;       // 128 rows x 64 columns
 constexpr int kYBufBytes = 2 * kYHalfBytes;        // 32 KB
-constexpr int kBufs = 3;                            // chunks whose B and y tiles are in shared memory at a time
+constexpr int kBufs = 4;                            // chunks whose B and y tiles are in shared memory at a time
 constexpr size_t kTmaDynSmem = 2 * kVBytes + kBufs * kBBufBytes + kBufs * kYBufBytes + 1024;
 constexpr int kTmaTmemCols = 256;                  // two accumulators of 128 columns
 
@@ -594,13 +612,13 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile int32_t failed;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const DenseExpandProblem &pb = P.prob[blockIdx.z];
+  int col_begin;
+  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin)];
 
   pdl_launch_dependents();
   const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
                   P.pv.header[PH_LANES] == P.lanes;
   const int m = blockIdx.x;
-  const int col_begin = blockIdx.y * kColsPerCta;
   if (!ok || !pb.use_tma || m >= P.pv.header[PH_NUM_DENSE] || col_begin >= pb.n) {
     pdl_wait();
     return;
@@ -872,6 +890,7 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
   const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
   if (tiles == 0) return MINT_OK;
   DenseParams P = {};
+  int32_t shares = 0;
   for (int i = 0; i < nprob; ++i) {
     DenseProblem &pb = P.prob[i];
     pb.A = args[i].A;
@@ -880,11 +899,13 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
     pb.d = args[i].d;
     pb.r_max = args[i].r_max;
     pb.splits = mint_dense_splits(args[i].d);
+    shares += pb.splits;
     pb.ws_part = static_cast<float *>(workspaces[i]);
     pb.use_tma = make_map_2d(&pb.x_map, args[i].x, (uint64_t)T, (uint64_t)args[i].d, (uint64_t)args[i].ldx, kTileRows) &&
                  make_map_2d(&pb.a_map, args[i].A, (uint64_t)args[i].num_slots * args[i].r_max, (uint64_t)args[i].d,
                              (uint64_t)args[i].d, kMaxRank);
   }
+  P.nprob = nprob;
   P.T = T;
   P.lanes = lanes;
   P.dense_slot0 = dense_slot0;
@@ -898,7 +919,7 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)tiles, (unsigned)(nprob * MINT_DENSE_SPLIT_MAX));
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)shares);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kDynSmem;
   cfg.stream = s;
@@ -925,7 +946,7 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
   const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
   if (tiles == 0) return MINT_OK;
   DenseExpandParams P = {};
-  int32_t n_max = 0;
+  int32_t ranges = 0;
   bool any_tma = false;
   for (int i = 0; i < nprob; ++i) {
     DenseExpandProblem &pb = P.prob[i];
@@ -940,8 +961,9 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
                              (uint64_t)args[i].n, kMaxRank) &&
                  make_map_2d(&pb.y_map, args[i].y, (uint64_t)T, (uint64_t)args[i].n, (uint64_t)args[i].ldy, kTileRows);
     any_tma = any_tma || pb.use_tma;
-    n_max = pb.n > n_max ? pb.n : n_max;
+    ranges += (pb.n + kColsPerCta - 1) / kColsPerCta;
   }
+  P.nprob = nprob;
   P.T = T;
   P.lanes = lanes;
   P.dense_slot0 = dense_slot0;
@@ -953,7 +975,7 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)tiles, (unsigned)((n_max + kColsPerCta - 1) / kColsPerCta), (unsigned)nprob);
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)ranges);
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kExpDynSmem;
   cfg.stream = s;
