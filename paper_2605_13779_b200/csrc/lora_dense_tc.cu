@@ -24,6 +24,8 @@
 //
 // Every wait on an mbarrier is bounded; a wait that runs out records
 // MINT_ERR_TIMEOUT, and the CTA still frees its tensor memory before it returns.
+#include <algorithm>
+
 #include "mint_tc.cuh"
 
 using namespace mint;
@@ -291,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_
 // of the speed.)  B is read once per 128 tokens; the streamed expand reads it
 // once per 32.  Waits are bounded as in the shrink.
 constexpr int kExpChunk = 128;                 // columns of n per MMA (N)
-constexpr int kColsPerCta = 4096;
+constexpr int kColsPerCta = 8192;
 constexpr int kStageRowBytes = kExpChunk * 2 + 16;   // padded: rows of a transposing 8x8 load fall into different banks
 constexpr int kBStageBytes = kMaxRank * kStageRowBytes;          // 17408
 constexpr int kYRowBytes = kExpChunk * 2 + 16;                   // padded: a warp's 16-byte accesses to 8 rows do not collide
@@ -325,16 +327,20 @@ struct DenseExpandParams {
 };
 
 // The grid's second dimension runs over the column ranges of all problems laid end to end (a
-// narrow problem then brings no CTAs that only exit): problem and first column of range y.
-__device__ __forceinline__ int expand_range(const DenseExpandParams &P, int y, int &col_begin) {
-  int z = 0;
-  while (z + 1 < P.nprob) {
-    const int ranges = (P.prob[z].n + kColsPerCta - 1) / kColsPerCta;
-    if (y < ranges) break;
+// narrow problem then brings no CTAs that only exit).  A problem of n columns has
+// ceil(n / kColsPerCta) ranges of equal width (a multiple of the 128-column chunk): returns the
+// problem of range y and its columns [col_begin, col_end).
+__device__ __forceinline__ int expand_range(const DenseExpandParams &P, int y, int &col_begin, int &col_end) {
+  int z = 0, ranges = 1;
+  for (;; ++z) {
+    ranges = (P.prob[z].n + kColsPerCta - 1) / kColsPerCta;
+    if (y < ranges || z + 1 >= P.nprob) break;
     y -= ranges;
-    ++z;
   }
-  col_begin = y * kColsPerCta;
+  const int n = P.prob[z].n;
+  const int per = ((n + ranges - 1) / ranges + kExpChunk - 1) / kExpChunk * kExpChunk;
+  col_begin = y * per;
+  col_end = min(n, col_begin + per);
   return z;
 }
 
@@ -368,8 +374,8 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
   __shared__ int32_t rows[kTileRows];
   __shared__ volatile int32_t failed;   // written after a wait that ran out; read only after a CTA barrier
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int col_begin;
-  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin)];
+  int col_begin, col_end;
+  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin, col_end)];
 
   pdl_launch_dependents();
   const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
@@ -381,7 +387,6 @@ __global__ void __launch_bounds__(kThreads, 2) dense_expand_kernel(const __grid_
     pdl_wait();
     return;
   }
-  const int col_end = min(pb.n, col_begin + kColsPerCta);
   const int ntiles = P.pv.header[PH_NCHUNK1];
   const int listed = P.pv.dense_tile[m];
   if (pb.use_tma && listed >= 0) {   // a tile of consecutive tokens is the tensor-map kernel's
@@ -612,8 +617,8 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile int32_t failed;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int col_begin;
-  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin)];
+  int col_begin, col_end;
+  const DenseExpandProblem &pb = P.prob[expand_range(P, (int)blockIdx.y, col_begin, col_end)];
 
   pdl_launch_dependents();
   const bool ok = plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi, nullptr) &&
@@ -623,7 +628,6 @@ __global__ void __launch_bounds__(kTmaThreads, 1) dense_expand_tma_kernel(const 
     pdl_wait();
     return;
   }
-  const int col_end = min(pb.n, col_begin + kColsPerCta);
   const int ntiles = P.pv.header[PH_NCHUNK1];
   const int t0 = P.pv.dense_tile[m];
   if (t0 < 0) {   // its tokens are scattered: the other kernel's
@@ -887,7 +891,10 @@ int32_t mint_launch_dense_shrink(const DenseArgs *args, int nprob, const TableDe
     attr_set = true;
   }
   const int32_t T = args[0].T;
-  const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
+  // 128-row tiles of dense segments: a segment of len tokens has at most len / 128 + 1, and there are at
+  // most min(slots, T / 128) dense segments
+  const int64_t tiles = (int64_t)(T / MINT_DENSE_MIN_SEGMENT) +
+                        std::min<int64_t>(tab.num_slots, T / MINT_DENSE_MIN_SEGMENT);
   if (tiles == 0) return MINT_OK;
   DenseParams P = {};
   int32_t shares = 0;
@@ -943,7 +950,10 @@ int32_t mint_launch_dense_expand(const DenseArgs *args, int nprob, const TableDe
     attr_set = true;
   }
   const int32_t T = args[0].T;
-  const int64_t tiles = 2 * (int64_t)(T / MINT_DENSE_MIN_SEGMENT);   // full and ragged 128-row tiles of dense segments
+  // 128-row tiles of dense segments: a segment of len tokens has at most len / 128 + 1, and there are at
+  // most min(slots, T / 128) dense segments
+  const int64_t tiles = (int64_t)(T / MINT_DENSE_MIN_SEGMENT) +
+                        std::min<int64_t>(tab.num_slots, T / MINT_DENSE_MIN_SEGMENT);
   if (tiles == 0) return MINT_OK;
   DenseExpandParams P = {};
   int32_t ranges = 0;
