@@ -293,7 +293,7 @@ __global__ void __launch_bounds__(kThreads, 2) dense_shrink_kernel(const __grid_
 // of the speed.)  B is read once per 128 tokens; the streamed expand reads it
 // once per 32.  Waits are bounded as in the shrink.
 constexpr int kExpChunk = 128;                 // columns of n per MMA (N)
-constexpr int kColsPerCta = 8192;
+constexpr int kColsPerCta = 16384;
 constexpr int kStageRowBytes = kExpChunk * 2 + 16;   // padded: rows of a transposing 8x8 load fall into different banks
 constexpr int kBStageBytes = kMaxRank * kStageRowBytes;          // 17408
 constexpr int kYRowBytes = kExpChunk * 2 + 16;                   // padded: a warp's 16-byte accesses to 8 rows do not collide
