@@ -224,8 +224,8 @@ def test_dense_segments_take_the_tensor_core_kernels():
 def test_dense_segments_grouped_projections_of_different_widths():
     """Two projections of different widths in one grouped call over a batch with
     dense segments: both take one range of columns per 128-row tile in the
-    tensor-core expand, the wide one with a ragged last 128-column chunk (n = 2184),
-    and the narrow one leaves part of the grid without work.  (Several column
+    tensor-core expand, the wide one with a ragged last 128-column chunk (n = 2184);
+    the ranges of the two lie end to end in the grid.  (Several column
     ranges per tile: test_dense_segments_wide_output_takes_several_column_ranges.)"""
     from paper_2605_13779_b200 import binding as mb, harness
     lengths = [900, 128, 257, 60, 1100, 131, 2, 640, 512, 400]
@@ -295,10 +295,12 @@ def test_dense_segments_wide_input_is_split_over_several_ctas(d, parts):
     check_case(case, f"dense segments d={d} ({parts} parts)")
 
 
-@pytest.mark.parametrize("n", [25600, 24584])
+@pytest.mark.parametrize("n", [25600, 24584, 40968])
 def test_dense_segments_wide_output_takes_several_column_ranges(n):
-    """n = 25600: seven ranges of 4096 columns per 128-row tile in the tensor-core
-    expand; n = 24584 ends with a range of 8 columns (a ragged last chunk)."""
+    """The tensor-core expand gives a 128-row tile one CTA per range of at most 16384
+    columns, the ranges of a projection equally wide: n = 25600 is two ranges of 12800,
+    n = 24584 two of 12416 and 12168 columns, n = 40968 three, and the last 128-column
+    chunk of the last two holds 8 columns (a ragged chunk)."""
     case = dense_segment_case(f"gpu/dense-tc/wide-n/{n}", SPLIT_LENGTHS, SPLIT_ADAPTERS, SPLIT_RANKS,
                               d=520, n=n, r_max=64)
     y_ref, _, _ = parity.oracle_dense(case)
