@@ -161,3 +161,137 @@ def test_not_resident_tokens_are_counted_and_skipped():
     dx, dA, dB, missing = backward.lora_backward(case.ids, table, t.slot_rank, t.slot_scale, case.A, case.B, case.x, dy)
     assert missing == int((case.ids == victim).sum())
     np.testing.assert_array_equal(dx[case.ids == victim], 0.0)
+
+
+# ---- per-expert LoRA tensors (packed MoE layout) --------------------------------------
+def moe_case(tag="bwd-moe-pin", T=9, K=3, E=5, num_slots=3, rank=3, d=10, n=6, proj="gate", p_none=0.2):
+    batch = synth.config4_batch(T=T, E=E, K=K, num_slots=num_slots, rank=rank, p_none=p_none, tag=tag)
+    return synth.config4_projection(batch, proj, d=d, n=n, tag=tag)
+
+
+def run_moe_backward(c, dy, **kw):
+    t = c.table
+    kw.setdefault("x_row", c.x_row)
+    kw.setdefault("pair_weight", c.pair_weight)
+    return backward.moe_lora_backward(c.ids, c.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B, c.x,
+                                      dy, **kw)
+
+
+def moe_forward_loss(c, dy, x=None, A=None, B=None):
+    t = c.table
+    zero = np.zeros((c.T * c.K, c.n), dtype=np.uint16)
+    y, _ = oracle.moe_lora_apply(c.ids, c.expert_ids, t.id_to_slot, t.slot_rank, t.slot_scale,
+                                 c.A if A is None else A, c.B if B is None else B, c.x if x is None else x, zero,
+                                 x_row=c.x_row, pair_weight=c.pair_weight)
+    return float((y * f64(dy)).sum())
+
+
+def test_moe_backward_hand_worked_pair():
+    """One pair, d = 2, rank 1, n = 2, scale 2, routing weight 0.5: A = [[1], [2]], B = [[3, -1]],
+    x = [1, 1] so v = 3; dy = [1, 2] so u = 3 - 2 = 1; w s = 1:
+    dx = A u = [1, 2], dA = x u = [[1], [1]], dB = v dy = [[3, 6]]."""
+    A = bits(np.array([[[[1.0], [2.0]]]]))          # [slot, expert, d, r]
+    B = bits(np.array([[[[3.0, -1.0]]]]))           # [slot, expert, r, n]
+    dx, dA, dB, missing = backward.moe_lora_backward(
+        [0], np.array([[0]], np.int32), [0], [1], [2.0], A, B, bits([[1.0, 1.0]]), bits([[1.0, 2.0]]),
+        pair_weight=np.array([0.5], np.float32))
+    assert missing == 0
+    np.testing.assert_array_equal(dx, [[1.0, 2.0]])
+    np.testing.assert_array_equal(dA, [[[[1.0], [1.0]]]])
+    np.testing.assert_array_equal(dB, [[[[3.0, 6.0]]]])
+
+
+@pytest.mark.parametrize("proj", ["gate", "down"])
+def test_moe_backward_central_differences_of_the_forward_oracle(proj):
+    """As for the dense backward: L = <y, dy> through the forward MoE oracle (the C program) is linear
+    in each of x, A and B, so central differences around 0 are exact.  For gate, several pairs read
+    one x row: dL/dx of that row is the sum of the pairs' dx rows."""
+    c = moe_case(proj=proj)
+    P = c.T * c.K
+    dy = synth.normal_bf16(synth.stream(c.name, "dy"), (P, c.n), 1.0)
+    dx, dA, dB, _ = run_moe_backward(c, dy)
+    rows = np.arange(P) if c.x_row is None else c.x_row
+    rng = np.random.default_rng(11)
+    h = 0.5
+    for _ in range(10):
+        row, col = int(rng.integers(c.x.shape[0])), int(rng.integers(c.d))
+        xp, xm = c.x.copy(), c.x.copy()
+        xp[row, col], xm[row, col] = bits(h).item(), bits(-h).item()
+        fd = (moe_forward_loss(c, dy, x=xp) - moe_forward_loss(c, dy, x=xm)) / (2 * h)
+        assert fd == pytest.approx(dx[rows == row, col].sum(), rel=1e-9, abs=1e-9)
+    t = c.table
+    active = [(tt, k) for tt in range(c.T) for k in range(c.K) if c.ids[tt] >= 0]
+    for _ in range(12):
+        tt, k = active[int(rng.integers(len(active)))]
+        slot, e = int(t.id_to_slot[c.ids[tt]]), int(c.expert_ids[tt, k])
+        rk = int(rng.integers(t.slot_rank[slot]))
+        col = int(rng.integers(c.d))
+        Ap, Am = c.A.copy(), c.A.copy()
+        Ap[slot, e, col, rk], Am[slot, e, col, rk] = bits(h).item(), bits(-h).item()
+        fd = (moe_forward_loss(c, dy, A=Ap) - moe_forward_loss(c, dy, A=Am)) / (2 * h)
+        assert fd == pytest.approx(dA[slot, e, col, rk], rel=1e-9, abs=1e-9)
+        j = int(rng.integers(c.n))
+        Bp, Bm = c.B.copy(), c.B.copy()
+        Bp[slot, e, rk, j], Bm[slot, e, rk, j] = bits(h).item(), bits(-h).item()
+        fd = (moe_forward_loss(c, dy, B=Bp) - moe_forward_loss(c, dy, B=Bm)) / (2 * h)
+        assert fd == pytest.approx(dB[slot, e, rk, j], rel=1e-9, abs=1e-9)
+
+
+def test_moe_backward_one_expert_one_route_is_the_dense_backward():
+    """E = K = 1 with unit weights: the packed tensors are the dense ones with A transposed."""
+    case = small_case("bwd-moe-dense", p_none=0.1)
+    dy = upstream(case)
+    dx, dA, dB, _ = run_backward(case, dy)
+    t = case.table
+    A_moe = np.ascontiguousarray(case.A.transpose(0, 2, 1))[:, None]        # [slots, 1, d, r_max]
+    B_moe = case.B[:, None]                                                   # [slots, 1, r_max, n]
+    mdx, mdA, mdB, _ = backward.moe_lora_backward(case.ids, np.zeros((case.T, 1), np.int32), t.id_to_slot,
+                                                  t.slot_rank, t.slot_scale, A_moe, B_moe, case.x, dy)
+    np.testing.assert_allclose(mdx, dx, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(mdA[:, 0].transpose(0, 2, 1), dA, rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(mdB[:, 0], dB, rtol=1e-12, atol=1e-12)
+
+
+def test_moe_backward_masks_and_weights():
+    """Ranks at or above the slot's rank and (slot, expert) blocks without pairs keep their starting
+    values bit for bit; pairs of tokens without an adapter and of expert ids out of
+    range keep their dx row; a constant routing weight c is the scale times c."""
+    c = moe_case(tag="bwd-moe-mask", rank=2, p_none=0.3)
+    P = c.T * c.K
+    dy = synth.normal_bf16(synth.stream(c.name, "dy"), (P, c.n), 1.0)
+    ex = c.expert_ids.copy()
+    live = np.nonzero(c.ids >= 0)[0]
+    ex[live[0], 0] = c.E + 3                                     # dropped pair
+    t = c.table
+    t.slot_rank = t.slot_rank.copy()
+    t.slot_rank[0] = 1                                           # a slot padded up to r_max
+    r_max = c.A.shape[3]
+    used = np.zeros((t.num_slots, c.E), bool)
+    for tt in live:
+        for k in range(c.K):
+            if 0 <= ex[tt, k] < c.E:
+                used[t.id_to_slot[c.ids[tt]], ex[tt, k]] = True
+    dA0 = np.full(c.A.shape, 7.0)
+    dB0 = np.full(c.B.shape, -3.0)
+    touch_a = np.zeros(c.A.shape, bool)
+    touch_b = np.zeros(c.B.shape, bool)
+    for s_ in range(t.num_slots):
+        touch_a[s_, used[s_], :, :t.slot_rank[s_]] = True
+        touch_b[s_, used[s_], :t.slot_rank[s_], :] = True
+    dx0 = synth.normal_bf16(synth.stream(c.name, "dx0"), (P, c.d), 1.0)
+    dx, dA, dB, _ = backward.moe_lora_backward(c.ids, ex, t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B, c.x, dy,
+                                               x_row=c.x_row, pair_weight=c.pair_weight, dx0=dx0, dA0=dA0, dB0=dB0)
+    assert t.slot_rank.min() < r_max and not used.all()        # there is padding and there are idle blocks
+    assert (dA[~touch_a] == 7.0).all() and (dB[~touch_b] == -3.0).all()
+    assert (dA[touch_a] != 7.0).mean() > 0.99 and (dB[touch_b] != -3.0).mean() > 0.99
+    dead = np.repeat(c.ids < 0, c.K)
+    dead[live[0] * c.K] = True
+    np.testing.assert_array_equal(dx[dead], f64(dx0)[dead])
+    assert np.abs(dx[~dead] - f64(dx0)[~dead]).max() > 0
+    const = np.full(P, 0.25, np.float32)
+    a = backward.moe_lora_backward(c.ids, ex, t.id_to_slot, t.slot_rank, t.slot_scale, c.A, c.B, c.x, dy,
+                                   x_row=c.x_row, pair_weight=const)
+    b = backward.moe_lora_backward(c.ids, ex, t.id_to_slot, t.slot_rank, t.slot_scale * np.float32(0.25), c.A, c.B,
+                                   c.x, dy, x_row=c.x_row)
+    for u_, v_ in zip(a[:3], b[:3]):
+        np.testing.assert_allclose(u_, v_, rtol=1e-12, atol=1e-15)
