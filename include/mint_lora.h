@@ -420,6 +420,34 @@ int32_t mint_moe_lora_apply_combine(const mint_pool *pool, const mint_slot_table
                                     void *workspace_dev, size_t workspace_bytes, int32_t *status_dev,
                                     mint_stream_t stream);
 
+/* Backward of the MoE expert LoRA apply (paper, "Scale Up": per-expert LoRA tensors
+ * keyed by expert id; "Time-Sliced Multi-LoRA Training": adapters padded to the
+ * slot's shape and masked).  For pair p = t*K + k with expert e, slot sigma, routing
+ * weight w_p and an upstream gradient dy_dev (bf16 [T*K][lddy], one row per pair),
+ * with u = B[sigma][e] . dy[p] and v = X[row(p)] . A[sigma][e]:
+ *   dx[p, :]             += w_p * s * A[sigma][e] . u          bf16 [T*K][lddx], one row per PAIR, one RNE
+ *                                                              store; the rows of the pairs that read one x
+ *                                                              row (gate, up: row(p) = t) are the caller's to add
+ *   dA[sigma][e][:, k]   += w_p * s * u[k] * X[row(p), :]      fp32 [num_slots][E][d][r_max]
+ *   dB[sigma][e][k, :]   += w_p * s * v[k] * dy[p, :]          fp32 [num_slots][E][r_max][n]
+ * dA_dev / dB_dev are caller-owned, shaped like the pool's tensors, accumulated into;
+ * ranks k >= rank of a slot and (slot, expert) blocks without pairs are not touched;
+ * pairs of tokens without a resident adapter, of expert ids out of range (both already
+ * reported by the plan) or whose x row is out of range (reported as BAD_INDEX) contribute
+ * nothing and keep their dx row.  The routing weights are constants: no gradient with
+ * respect to them.  dx_dev may be NULL; dA_dev and dB_dev may both be NULL.  Sums over a
+ * block's pairs run in the plan's order in fp32: bit-identical from run to run.
+ * Pools of r_max 8, 16, 32 or 64 only (UNSUPPORTED otherwise).  workspace_dev: device,
+ * 256-byte aligned, at least mint_moe_lora_backward_workspace_bytes(pool, T, K) bytes,
+ * uninitialised.  Other arguments and errors as for mint_moe_lora_apply.           */
+size_t mint_moe_lora_backward_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K);
+int32_t mint_moe_lora_backward(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                               int32_t T, int32_t K, const void *x_dev, int64_t ldx, int64_t x_rows,
+                               const int32_t *x_row_dev, const float *pair_weight_dev,
+                               const void *dy_dev, int64_t lddy, void *dx_dev, int64_t lddx,
+                               float *dA_dev, float *dB_dev, void *workspace_dev, size_t workspace_bytes,
+                               int32_t *status_dev, mint_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

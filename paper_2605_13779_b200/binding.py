@@ -48,6 +48,7 @@ EXPORTS = [
     "mint_lora_backward_workspace_bytes", "mint_lora_backward", "mint_lora_backward_grouped",
     "mint_moe_lora_apply_workspace_bytes", "mint_moe_lora_apply", "mint_moe_lora_apply_grouped",
     "mint_moe_lora_apply_combine_workspace_bytes", "mint_moe_lora_apply_combine",
+    "mint_moe_lora_backward_workspace_bytes", "mint_moe_lora_backward",
 ]
 
 
@@ -145,6 +146,9 @@ def load_library() -> ctypes.CDLL:
         "mint_moe_lora_apply_grouped": (i32, [ctypes.POINTER(ApplyItem), i32, vp, vp, i32, i32, i64, vp, vp, vp, vp]),
         "mint_moe_lora_apply_combine_workspace_bytes": (sz, [vp, i32, i32]),
         "mint_moe_lora_apply_combine": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, sz, vp, vp]),
+        "mint_moe_lora_backward_workspace_bytes": (sz, [vp, i32, i32]),
+        "mint_moe_lora_backward": (i32, [vp, vp, vp, i32, i32, vp, i64, i64, vp, vp, vp, i64, vp, i64, vp, vp, vp, sz,
+                                         vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -558,3 +562,27 @@ def mint_moe_lora_apply_combine(pool: Pool, table: SlotTable, plan: Plan, x: tor
         _ptr(x_row), _ptr(pair_weight), _ptr(y), y.stride(0), _ptr(workspace),
         workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
     return y
+
+
+def mint_moe_lora_backward(pool: Pool, table: SlotTable, plan: Plan, x: torch.Tensor, dy: torch.Tensor,
+                           status: torch.Tensor, dx: Optional[torch.Tensor] = None,
+                           dA: Optional[torch.Tensor] = None, dB: Optional[torch.Tensor] = None,
+                           x_row: Optional[torch.Tensor] = None, pair_weight: Optional[torch.Tensor] = None,
+                           workspace: Optional[torch.Tensor] = None):
+    """dx (bf16 [T*K, d], one row per pair) and dA / dB (fp32, shaped like the pool's packed tensors)
+    are accumulated into; dy is bf16 [T*K, n]."""
+    if x_row is not None:
+        assert x_row.dtype == torch.int32 and x_row.is_contiguous()
+    if pair_weight is not None:
+        assert pair_weight.dtype == torch.float32 and pair_weight.is_contiguous()
+    for g in (dA, dB):
+        assert g is None or (g.dtype == torch.float32 and g.is_contiguous())
+    lib = load_library()
+    if workspace is None:
+        nbytes = max(256, int(lib.mint_moe_lora_backward_workspace_bytes(pool.handle, plan.T, plan.K)))
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=dy.device)
+    _check(lib.mint_moe_lora_backward(
+        pool.handle, table.handle, _ptr(plan.blob), plan.T, plan.K, _ptr(x), x.stride(0), x.shape[0],
+        _ptr(x_row), _ptr(pair_weight), _ptr(dy), dy.stride(0), _ptr(dx), dx.stride(0) if dx is not None else 0,
+        _ptr(dA), _ptr(dB), _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status), _stream()))
+    return dx, dA, dB

@@ -892,3 +892,88 @@ extern "C" int32_t mint_moe_lora_apply_grouped(const mint_moe_apply_item *items,
   }
   return MINT_OK;
 }
+
+// ---- backward of per-expert LoRA tensors (packed MoE pools) -------------------------------
+// Workspace: u and v ([T*K][r_max] fp32, pair order), then the streamed shrink's parts for dy . B^T and
+// for x . A.
+extern "C" size_t mint_moe_lora_backward_workspace_bytes(const mint_pool *pool, int32_t T, int32_t K) {
+  if (!pool || T <= 0 || K < 1 || pool->desc.num_experts < 1) return 0;
+  if (!mint_stream_moe_supported(pool->desc.r_max, 0)) return 0;
+  const size_t parts = align256(mint_stream_moe_workspace_bytes(
+      (int64_t)T * K, (int64_t)pool->desc.num_slots * pool->desc.num_experts, pool->desc.r_max));
+  return 2 * align256((size_t)T * K * pool->desc.r_max * sizeof(float)) + 2 * parts;
+}
+
+extern "C" int32_t mint_moe_lora_backward(const mint_pool *pool, const mint_slot_table *table, const void *plan_dev,
+                                          int32_t T, int32_t K, const void *x_dev, int64_t ldx, int64_t x_rows,
+                                          const int32_t *x_row_dev, const float *pair_weight_dev,
+                                          const void *dy_dev, int64_t lddy, void *dx_dev, int64_t lddx,
+                                          float *dA_dev, float *dB_dev, void *workspace_dev, size_t workspace_bytes,
+                                          int32_t *status_dev, mint_stream_t stream) {
+  const char *who = "moe_backward";
+  if (!pool || !table || !plan_dev || !status_dev) return mint_fail(MINT_ERR_INVALID_ARG, "%s: null argument", who);
+  if (T < 0 || K < 1 || (int64_t)T * K > kMaxItems) return mint_fail(MINT_ERR_INVALID_ARG, "%s: T=%d K=%d", who, T, K);
+  if ((dA_dev == nullptr) != (dB_dev == nullptr))
+    return mint_fail(MINT_ERR_INVALID_ARG, "%s: dA_dev and dB_dev are given together or not at all", who);
+  if (!dx_dev && !dA_dev) return mint_fail(MINT_ERR_INVALID_ARG, "%s: nothing to compute", who);
+  MoEArgs a;
+  bool streamed = false;
+  // (the forward checks; y stands for dy here: same width, same row per pair)
+  int32_t st = fill_moe(pool, table, T, K, x_dev, ldx, x_rows, x_row_dev, pair_weight_dev, const_cast<void *>(dy_dev),
+                        lddy, workspace_dev, workspace_bytes, status_dev, who, a, streamed);
+  if (st) return st;
+  if (T == 0) return MINT_OK;
+  if (!streamed)
+    return mint_fail(MINT_ERR_UNSUPPORTED, "%s: pools of r_max 8, 16, 32 or 64 and ranks up to 64 only", who);
+  if (dx_dev && (st = check_act(dx_dev, lddx, pool->desc.d, "dx_dev", who))) return st;
+  const size_t need = mint_moe_lora_backward_workspace_bytes(pool, T, K);
+  if (!workspace_dev || workspace_bytes < need)
+    return mint_fail(MINT_ERR_WORKSPACE_TOO_SMALL, "%s: workspace %zu < %zu", who, workspace_bytes, need);
+  if ((reinterpret_cast<uintptr_t>(workspace_dev) & 255) != 0)
+    return mint_fail(MINT_ERR_MISALIGNED, "%s: workspace_dev must be 256-byte aligned", who);
+  const int64_t pairs = (int64_t)T * K;
+  const int32_t E = pool->desc.num_experts, r_max = pool->desc.r_max;
+  char *w = static_cast<char *>(workspace_dev);
+  float *u = reinterpret_cast<float *>(w);
+  w += align256((size_t)pairs * r_max * sizeof(float));
+  float *v = reinterpret_cast<float *>(w);
+  w += align256((size_t)pairs * r_max * sizeof(float));
+  void *parts_u = w;
+  w += align256(mint_stream_moe_workspace_bytes(pairs, (int64_t)pool->desc.num_slots * E, r_max));
+  void *parts_v = w;
+  const TableDev tab = table_dev(table);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // u = w * dy . B^T: B's blocks are rank rows of n elements, and row p of dy belongs to pair p
+  MoEArgs au = a;
+  au.A = a.B;
+  au.d = a.n;
+  au.x = static_cast<const uint16_t *>(dy_dev);
+  au.ldx = lddy;
+  au.x_rows = pairs;
+  au.x_row = nullptr;
+  if ((st = mint_launch_stream_moe_shrink_v(&au, 1, true, tab, plan_dev, &parts_u, &u, s))) return st;
+  if (dx_dev &&
+      (st = mint_launch_moe_dx(a.A, u, static_cast<uint16_t *>(dx_dev), lddx, a.d, r_max, T, K, E, tab, plan_dev,
+                               status_dev, s)))
+    return st;
+  if (!dA_dev) return MINT_OK;
+  // v = w * x . A, then both weight gradients in one launch
+  if ((st = mint_launch_stream_moe_shrink_v(&a, 1, false, tab, plan_dev, &parts_v, &v, s))) return st;
+  GradJobHost jobs[2];
+  jobs[0].coef = u;
+  jobs[0].act = a.x;
+  jobs[0].ld = ldx;
+  jobs[0].out = dA_dev;
+  jobs[0].width = a.d;
+  jobs[0].r_max = r_max;
+  jobs[0].row_map = x_row_dev;
+  jobs[0].act_rows = x_rows;
+  jobs[0].packed = 1;
+  jobs[1].coef = v;
+  jobs[1].act = static_cast<const uint16_t *>(dy_dev);
+  jobs[1].ld = lddy;
+  jobs[1].out = dB_dev;
+  jobs[1].width = a.n;
+  jobs[1].r_max = r_max;
+  return mint_launch_grad_weights(jobs, 2, T, tab, plan_dev, status_dev, s, K, E);
+}

@@ -49,27 +49,32 @@ struct GradJob {
   const float *coef;      // [T][r_max] fp32, token order: u (for dA) or v (for dB)
   const uint16_t *act;    // [T][ld] bf16: x (for dA) or dy (for dB)
   int64_t ld;
-  float *out;             // [slots][r_max][width] fp32, accumulated into
+  float *out;             // [blocks][r_max][width] fp32, accumulated into (packed: [blocks][width][r_max]);
+                          // block = slot, or slot * experts + expert
+  const int32_t *row_map; // row of act that item p reads (nullptr: p)
+  int64_t act_rows;       // rows of act: an item whose row is outside is left out
   int32_t width, r_max;
   int32_t block0;         // first of its groups of kBlocksPerCta column blocks in the grid's second dimension
-  int32_t pad;
+  int32_t packed;
 };
 
 struct GradParams {
   GradJob job[kMaxJobs];
   int32_t njobs, T;
+  int32_t K, E;           // items per token and experts of a MoE plan (1, 0: dense)
   int32_t *status;
   TableDev tab;
   PlanView pv;
 };
 
 __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_constant__ GradParams P) {
-  __shared__ int32_t tok[kTokenBatch];
+  __shared__ int32_t tok[kTokenBatch];    // staged items (tokens, or (token, k) pairs)
+  __shared__ int32_t arow[kTokenBatch];   // the row of act each of them reads
   __shared__ float cf[kTokenBatch][kRankChunk];
   const int tid = threadIdx.x;
   pdl_launch_dependents();
   // (before the wait: the plan and the slot table, complete before this call's first kernel started)
-  if (!plan_ok(P.pv.header, P.T, 1, P.tab.num_slots, 0, P.tab.gen_lo, P.tab.gen_hi,
+  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.E, P.tab.gen_lo, P.tab.gen_hi,
                (blockIdx.x == 0 && blockIdx.y == 0) ? P.status : nullptr)) {
     pdl_wait();
     return;
@@ -91,12 +96,18 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
     if (tid == 0) report(P.status, MINT_ERR_RANK_TOO_LARGE, slot);
     return;
   }
-  float *out_slot = p.out + (size_t)slot * p.r_max * p.width;
+  const int block = P.E > 0 ? slot * P.E + P.pv.seg_expert[seg] : slot;
+  float *out_slot = p.out + (size_t)block * p.r_max * p.width;
   const bool one_batch = len <= kTokenBatch;   // the usual case of a decode batch: staged once per rank chunk
   // stages the token indices and the coefficients of tokens [b0, b0 + nb) for ranks k0 .. k0 + kc - 1
   auto stage = [&](int b0, int nb, int k0, int kc) {
     __syncthreads();   // what was staged before has been read
-    if (tid < nb) tok[tid] = P.pv.perm[off + b0 + tid];
+    if (tid < nb) {
+      const int item = P.pv.perm[off + b0 + tid];
+      tok[tid] = item;
+      const int r_ = p.row_map ? p.row_map[item] : item;
+      arow[tid] = (r_ >= 0 && r_ < p.act_rows) ? r_ : -1;   // (reported by the shrink that made the coefficients)
+    }
     __syncthreads();
     for (int i = tid; i < nb * kRankChunk; i += kThreads) {
       const int j = i / kRankChunk, k = i - j * kRankChunk;
@@ -107,7 +118,11 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
   {
     // the gradient rows this CTA will add to, on their way into L2 while the tokens are walked
     const int col = ((int)blockIdx.y - p.block0) * kBlocksPerCta * kColsPerCta + tid * kColsPerThread;
-    if ((tid & 7) == 0 && col < p.width)
+    if (p.packed) {   // [width][r_max]: this thread's four columns are 4 r_max consecutive floats
+      if (col < p.width)
+        for (int i = 0; i < 4 * p.r_max; i += 32)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(out_slot + (size_t)col * p.r_max + i));
+    } else if ((tid & 7) == 0 && col < p.width)
       for (int k = 0; k < rank; ++k)
         asm volatile("prefetch.global.L2 [%0];" ::"l"(out_slot + (size_t)k * p.width + col));
   }
@@ -130,7 +145,8 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
         if (col_ok) {
 #pragma unroll 4
           for (int j = 0; j < nb; ++j) {
-            const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p.act + (int64_t)tok[j] * p.ld + col));
+            if (arow[j] < 0) continue;
+            const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p.act + (int64_t)arow[j] * p.ld + col));
             const float a[4] = {bf16lo(q.x), bf16hi(q.x), bf16lo(q.y), bf16hi(q.y)};
 #pragma unroll
             for (int k = 0; k < kRankChunk; ++k) {
@@ -141,7 +157,16 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
           }
         }
       }
-      if (col_ok) {
+      if (col_ok && p.packed) {
+#pragma unroll
+        for (int e = 0; e < kColsPerThread; ++e)
+#pragma unroll
+          for (int k = 0; k < kRankChunk; ++k)
+            if (k < kc) {
+              float *dst = out_slot + (size_t)(col + e) * p.r_max + k0 + k;
+              *dst = fmaf(scale, acc[k][e], *dst);
+            }
+      } else if (col_ok) {
 #pragma unroll
         for (int k = 0; k < kRankChunk; ++k)
           if (k < kc) {
@@ -158,10 +183,85 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
   }
 }
 
+// ---- dx of per-expert LoRA tensors in the packed layout -------------------------------
+// dx[p, :] += s * u[p, :rank] . A[slot][expert]^T with A stored [d][r_max] (a column of d is r_max
+// consecutive values).  One CTA per (tile of at most 32 pairs of one (expert, slot), 1024 columns
+// of d): the tile's u (already times the routing weight) waits in shared memory times s, a thread
+// holds the r_max weights of its column(s) in registers and walks the tile's pairs.  CUDA cores:
+// 2 r_max flops per 2 bytes of dx read and written.
+struct MoeDxParams {
+  const uint16_t *A;      // [slot][E][d][r_max]
+  const float *u;         // [T*K][r_max], pair order
+  uint16_t *dx;           // [T*K][lddx] bf16, accumulated into
+  int64_t lddx;
+  int32_t d, r_max, T, K, E;
+  int32_t *status;
+  TableDev tab;
+  PlanView pv;
+};
+
+constexpr int kDxColsPerCta = 1024;
+
+template <int RM>
+__global__ void __launch_bounds__(kThreads) moe_dx_kernel(const __grid_constant__ MoeDxParams P) {
+  constexpr int kCols = RM <= 16 ? 2 : 1;   // columns per thread
+  __shared__ float us[32][RM];
+  __shared__ int32_t row[32];
+  const int tid = threadIdx.x;
+  pdl_launch_dependents();
+  if (!plan_ok(P.pv.header, P.T, P.K, P.tab.num_slots, P.E, P.tab.gen_lo, P.tab.gen_hi, nullptr) ||
+      (int)blockIdx.x >= P.pv.header[PH_NCHUNK1]) {
+    pdl_wait();
+    return;
+  }
+  const TileDesc t = P.pv.tile_desc[blockIdx.x];
+  const uint16_t *A_blk = P.A + ((size_t)t.slot * P.E + t.expert) * (size_t)P.d * RM;
+  if (tid < 32) row[tid] = tid < t.len ? P.pv.perm[t.off + tid] : 0;
+  pdl_wait();   // u and dx belong to earlier kernels until here
+  __syncthreads();
+  for (int i = tid; i < 32 * RM; i += kThreads) {
+    const int l = i / RM, k = i - l * RM;
+    us[l][k] = (l < t.len && k < t.rank) ? t.scale * P.u[(size_t)row[l] * RM + k] : 0.f;
+  }
+  __syncthreads();
+  const int c_end = min(P.d, ((int)blockIdx.y + 1) * kDxColsPerCta);
+  for (int c = (int)blockIdx.y * kDxColsPerCta + tid * kCols; c < c_end; c += kThreads * kCols) {
+    float a[kCols][RM];
+#pragma unroll
+    for (int e = 0; e < kCols; ++e)
+#pragma unroll
+      for (int k8 = 0; k8 < RM; k8 += 8) {
+        float f[8];
+        unpack8(__ldg(reinterpret_cast<const uint4 *>(A_blk + (size_t)(c + e) * RM + k8)), f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a[e][k8 + k] = k8 + k < t.rank ? f[k] : 0.f;   // (padding may hold anything)
+      }
+    for (int l = 0; l < t.len; ++l) {
+      float acc[kCols];
+#pragma unroll
+      for (int e = 0; e < kCols; ++e) acc[e] = 0.f;
+#pragma unroll
+      for (int k = 0; k < RM; ++k) {
+        const float uk = us[l][k];
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) acc[e] = fmaf(uk, a[e][k], acc[e]);
+      }
+      uint16_t *dst = P.dx + (size_t)row[l] * P.lddx + c;
+      if (kCols == 2) {
+        const uint32_t old = *reinterpret_cast<const uint32_t *>(dst);
+        *reinterpret_cast<uint32_t *>(dst) = pack_bf16x2(bf16lo(old) + acc[0], bf16hi(old) + acc[kCols - 1]);
+      } else {
+        const uint32_t old = (uint32_t)*dst;
+        *dst = (uint16_t)(pack_bf16x2(bf16lo(old) + acc[0], 0.f) & 0xffffu);
+      }
+    }
+  }
+}
+
 }  // namespace
 
 int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, const TableDev &tab,
-                                 const void *plan_dev, int32_t *status, cudaStream_t s) {
+                                 const void *plan_dev, int32_t *status, cudaStream_t s, int32_t K, int32_t E) {
   if (T == 0 || njobs == 0) return MINT_OK;
   if (njobs > kMaxJobs) return mint_fail(MINT_ERR_INVALID_ARG, "weight gradients: at most %d tensors per launch", kMaxJobs);
   GradParams P = {};
@@ -174,15 +274,21 @@ int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, 
     j.out = jobs[i].out;
     j.width = jobs[i].width;
     j.r_max = jobs[i].r_max;
+    j.row_map = jobs[i].row_map;
+    j.act_rows = jobs[i].act_rows > 0 ? jobs[i].act_rows : ((int64_t)1 << 40);
+    j.packed = jobs[i].packed;
     j.block0 = blocks;
     blocks += (jobs[i].width + kBlocksPerCta * kColsPerCta - 1) / (kBlocksPerCta * kColsPerCta);
   }
   P.njobs = njobs;
   P.T = T;
+  P.K = K;
+  P.E = E;
   P.status = status;
   P.tab = tab;
-  P.pv = mint_plan_view(plan_dev, T, tab.num_slots);
-  const int64_t seg_ub = T < tab.num_slots ? T : tab.num_slots;
+  const int64_t items = (int64_t)T * K, key_space = (int64_t)tab.num_slots * (E > 0 ? E : 1);
+  P.pv = mint_plan_view(plan_dev, items, key_space);
+  const int64_t seg_ub = items < key_space ? items : key_space;
   const dim3 grid((unsigned)seg_ub, (unsigned)blocks);
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -195,4 +301,38 @@ int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, 
   // right after a plan or a bind kernel it waits for that kernel in full: it reads the plan at once
   cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
   return mint_check_cuda(cudaLaunchKernelEx(&cfg, grad_weight_kernel, P), "grad_weight launch");
+}
+
+
+// dx[p, :] += s * u[p, :] . A[slot][expert]^T for the pairs of a MoE plan (packed A, r_max 8, 16, 32 or 64).
+int32_t mint_launch_moe_dx(const uint16_t *A, const float *u, uint16_t *dx, int64_t lddx, int32_t d, int32_t r_max,
+                           int32_t T, int32_t K, int32_t E, const TableDev &tab, const void *plan_dev,
+                           int32_t *status, cudaStream_t s) {
+  const int64_t pairs = (int64_t)T * K, key_space = (int64_t)tab.num_slots * E;
+  const int64_t tiles = mint_tile_upper_bound(1, pairs, key_space);
+  if (tiles == 0) return MINT_OK;
+  MoeDxParams P = {};
+  P.A = A; P.u = u; P.dx = dx; P.lddx = lddx;
+  P.d = d; P.r_max = r_max; P.T = T; P.K = K; P.E = E;
+  P.status = status;
+  P.tab = tab;
+  P.pv = mint_plan_view(plan_dev, pairs, key_space);
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)((d + kDxColsPerCta - 1) / kDxColsPerCta));
+  cfg.blockDim = dim3(kThreads);
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+  cudaError_t e;
+  switch (r_max) {
+    case 8: e = cudaLaunchKernelEx(&cfg, moe_dx_kernel<8>, P); break;
+    case 16: e = cudaLaunchKernelEx(&cfg, moe_dx_kernel<16>, P); break;
+    case 32: e = cudaLaunchKernelEx(&cfg, moe_dx_kernel<32>, P); break;
+    case 64: e = cudaLaunchKernelEx(&cfg, moe_dx_kernel<64>, P); break;
+    default: return mint_fail(MINT_ERR_UNSUPPORTED, "MoE backward: r_max %d (8, 16, 32 or 64)", r_max);
+  }
+  return mint_check_cuda(e, "moe_dx launch");
 }

@@ -1293,19 +1293,14 @@ static int32_t stream_kernel_attributes() {
 // MoE expert LoRA apply on the streamed kernels: the plan's items are the
 // (token, k) pairs grouped by (expert, slot); the weight block of a tile is
 // (slot, expert); the shrink reads row x_row[p] of x, the expand updates row p of y.
-int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
-                               void *const *workspaces, cudaStream_t s) {
-  if (nprob < 1 || nprob > kMaxProblems)
-    return mint_fail(MINT_ERR_INVALID_ARG, "grouped MoE apply: 1..%d problems", kMaxProblems);
-  int32_t lanes = 0;
-  int32_t st = mint_device_lanes(&lanes);
-  if (st) return st;
-  if ((st = stream_kernel_attributes())) return st;
+// Kernel parameters of nprob MoE problems that share the plan, the row map and the pair weights
+// (share_x: consecutive problems that read one x through pools of one shape are shrunk together).
+static StreamParams moe_stream_params(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                                      void *const *workspaces, int32_t lanes, bool share_x) {
   const MoEArgs &a0 = args[0];
   const int64_t pairs = (int64_t)a0.T * a0.K;
   const int64_t key_space = (int64_t)tab.num_slots * a0.num_experts;
   const int64_t tiles = mint_tile_upper_bound(1, pairs, key_space);
-  if (tiles == 0) return MINT_OK;
   StreamParams P = {};
   int cb_s = 0, cb_e = 0, cb_widest = 0;
   for (int i = 0; i < nprob; ++i) {
@@ -1333,7 +1328,7 @@ int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &t
     cb_widest = std::max(cb_widest, kShrinkPieceBlocks + (a.d + kShrinkBlock - 1) / kShrinkBlock);
     if (i + 1 < nprob) {
       const MoEArgs &b = args[i + 1];
-      if (b.x == a.x && b.ldx == a.ldx && b.d == a.d && b.r_max == a.r_max && a.r_max <= 16) pb.dual = 1;
+      if (share_x && b.x == a.x && b.ldx == a.ldx && b.d == a.d && b.r_max == a.r_max && a.r_max <= 16) pb.dual = 1;
     }
   }
   P.nprob = nprob;
@@ -1352,6 +1347,20 @@ int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &t
   P.status = a0.status;
   P.tab = tab;
   P.pv = mint_plan_view(plan_dev, pairs, key_space);
+  return P;
+}
+
+int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
+                               void *const *workspaces, cudaStream_t s) {
+  if (nprob < 1 || nprob > kMaxProblems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "grouped MoE apply: 1..%d problems", kMaxProblems);
+  int32_t lanes = 0;
+  int32_t st = mint_device_lanes(&lanes);
+  if (st) return st;
+  if ((st = stream_kernel_attributes())) return st;
+  if (mint_tile_upper_bound(1, (int64_t)args[0].T * args[0].K, (int64_t)tab.num_slots * args[0].num_experts) == 0)
+    return MINT_OK;
+  const StreamParams P = moe_stream_params(args, nprob, tab, plan_dev, workspaces, lanes, true);
 
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -1422,7 +1431,9 @@ __global__ void __launch_bounds__(kThreads) gather_v_kernel(const __grid_constan
       for (int k = 0; k < 4; ++k) s += part[k];
     }
     const int l = i / d.rank, j = i - l * d.rank;
-    out.v[p][(size_t)P.pv.perm[d.off + l] * pb.r_max + j] = s;
+    const int item = P.pv.perm[d.off + l];
+    // (MoE: the pair's routing weight multiplies its row, as it does in the forward expand)
+    out.v[p][(size_t)item * pb.r_max + j] = P.pair_weight ? __ldg(P.pair_weight + item) * s : s;
   }
 }
 
@@ -1518,6 +1529,46 @@ int32_t mint_launch_stream(const DenseArgs *args, int nprob, const TableDev &tab
 int32_t mint_launch_stream_shrink_v(const DenseArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                     void *const *workspaces, float *const *v_out, cudaStream_t s) {
   return mint_launch_stream_phases(args, nprob, tab, plan_dev, workspaces, s, 1, v_out);
+}
+
+// The same for the (token, k) pairs of a MoE plan: v_out[i] ([T*K][r_max] fp32, pair order) = the pair's
+// routing weight times x[x_row[p]] . A[slot][expert] (packed pools, A as [d][r_max]) or, with rank_major,
+// times x[p] . A[slot][expert]^T for tensors stored as [slot][expert][r_max][d] -- which is how the backward
+// gets dy . B^T out of a pool's B.  Workspaces as for mint_launch_stream_moe.
+int32_t mint_launch_stream_moe_shrink_v(const MoEArgs *args, int nprob, bool rank_major, const TableDev &tab,
+                                        const void *plan_dev, void *const *workspaces, float *const *v_out,
+                                        cudaStream_t s) {
+  if (nprob < 1 || nprob > kMaxProblems)
+    return mint_fail(MINT_ERR_INVALID_ARG, "MoE shrink: 1..%d problems", kMaxProblems);
+  int32_t lanes = 0;
+  int32_t st = mint_device_lanes(&lanes);
+  if (st) return st;
+  if ((st = stream_kernel_attributes())) return st;
+  const int64_t tiles =
+      mint_tile_upper_bound(1, (int64_t)args[0].T * args[0].K, (int64_t)tab.num_slots * args[0].num_experts);
+  if (tiles == 0) return MINT_OK;
+  const StreamParams P = moe_stream_params(args, nprob, tab, plan_dev, workspaces, lanes, false);
+  GatherV out = {};
+  for (int i = 0; i < nprob; ++i) out.v[i] = v_out[i];
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)lanes);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kRingsBytes;
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
+  if (rank_major)
+    st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<false>, P), "shrink_stream launch");
+  else
+    st = mint_check_cuda(cudaLaunchKernelEx(&cfg, shrink_stream_kernel<true>, P), "shrink_stream (packed) launch");
+  if (st) return st;
+  cfg.gridDim = dim3((unsigned)tiles, (unsigned)nprob);
+  cfg.dynamicSmemBytes = 0;
+  cfg.numAttrs = 1;
+  return mint_check_cuda(cudaLaunchKernelEx(&cfg, gather_v_kernel, P, out), "gather_v launch");
 }
 
 // ---- fused apply without a caller-provided workspace -------------------------------

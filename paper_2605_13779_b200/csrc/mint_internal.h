@@ -252,11 +252,20 @@ struct GradJobHost {
   const float *coef;      // [T][r_max] fp32, token order
   const uint16_t *act;    // [T][ld] bf16
   int64_t ld;
-  float *out;             // [slots][r_max][width] fp32
+  float *out;             // [slots][r_max][width] fp32 (MoE: [slots][experts][r_max][width], or packed
+                          // [slots][experts][width][r_max])
   int32_t width, r_max;
+  const int32_t *row_map = nullptr;   // MoE: row of act that pair p reads (nullptr: p)
+  int64_t act_rows = 0;               // rows of act (0: not checked)
+  int32_t packed = 0;
 };
+// dx[p, :] += scale * u[p, :] . A[slot][expert]^T over the pairs of a MoE plan (A packed [slot][E][d][r_max])
+int32_t mint_launch_moe_dx(const uint16_t *A, const float *u, uint16_t *dx, int64_t lddx, int32_t d, int32_t r_max,
+                           int32_t T, int32_t K, int32_t E, const TableDev &tab, const void *plan_dev,
+                           int32_t *status, cudaStream_t s);
+// K, E: items per token and experts of the plan (1, 0 for dense plans)
 int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, const TableDev &tab,
-                                 const void *plan_dev, int32_t *status, cudaStream_t s);
+                                 const void *plan_dev, int32_t *status, cudaStream_t s, int32_t K = 1, int32_t E = 0);
 
 // x . A^T of up to 8 problems as tensors v_out[i] ([T][r_max] fp32, token order) through the streamed shrink
 // (bound ranks up to 64).  Entries of tokens without an adapter and of ranks at or above a slot's rank are
@@ -290,6 +299,11 @@ int32_t mint_launch_moe(const MoEArgs &a, const TableDev &tab, const void *plan_
 // nprob problems that share the plan, the row map and the pair weights (args[0]'s are used)
 int32_t mint_launch_stream_moe(const MoEArgs *args, int nprob, const TableDev &tab, const void *plan_dev,
                                void *const *workspaces, cudaStream_t s);
+// v_out[i] ([T*K][r_max] fp32, pair order) = routing weight times the pair's x row times A[slot][expert];
+// rank_major: the tensors behind args[i].A are stored [slot][expert][r_max][d] and row p of x belongs to pair p.
+int32_t mint_launch_stream_moe_shrink_v(const MoEArgs *args, int nprob, bool rank_major, const TableDev &tab,
+                                        const void *plan_dev, void *const *workspaces, float *const *v_out,
+                                        cudaStream_t s);
 
 int32_t mint_launch_table_init(int32_t *id_to_slot, int64_t catalog_size, int32_t *slot_rank,
                                float *slot_scale, int32_t num_slots, cudaStream_t s);
