@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the mixed-adapter LoRA apply on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3|config1|backward]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2|config5|config4|config3|config1|backward|moe_backward]
     python bench.py --impl reference ...        # the fp64 CPU oracle, timed on the host cores
 
 A step is a fixed number of passes of the whole hot path over one batch: each
@@ -493,6 +493,80 @@ def measure_backward(torch, dist, world, stream, peak, layers=6, short=False):
     return res
 
 
+def measure_moe_backward(torch, dist, world, stream, peak, short=False):
+    """The backward of config 4's three expert projections (per-pair dx, dA, dB of the packed tensors) at
+    full size, device-timed: one MoE plan, then mint_moe_lora_backward per projection; two sets of
+    tensors (about 2.5 GB each) are walked in turn."""
+    from oracle import backward as oracle_backward
+    from paper_2605_13779_b200 import accounting, binding as mb, harness, synth
+    wl = build_workload("config4", 0)
+    cases = wl["cases"]
+    P = cases[0].T * cases[0].K
+    base = [harness.upload_moe(c) for c in cases]
+    table, ids, ex, status = base[0].table, base[0].ids, base[0].expert_ids, mb.new_status()
+    dys = [synth.normal_bf16(synth.stream("bench/moe-backward", c.name), (P, c.n), 1.0) for c in cases]
+    sets = []
+    for si in range(2):
+        row = []
+        for dv, c, dy in zip(base, cases, dys):
+            pool = dv.pool if si == 0 else mb.Pool(dv.pool.A.clone(), dv.pool.B.clone(), c.d, c.n, c.r_max,
+                                                   dv.pool.num_slots, num_experts=c.E)
+            row.append((pool, dv.x if si == 0 else dv.x.clone(), mb.bf16_from_bits(dy),
+                        torch.zeros(P, c.d, dtype=torch.bfloat16, device="cuda"),
+                        torch.zeros(c.A.shape, dtype=torch.float32, device="cuda"),
+                        torch.zeros(c.B.shape, dtype=torch.float32, device="cuda"), dv.x_row))
+        sets.append(row)
+    nbytes = max(int(mb.load_library().mint_moe_lora_backward_workspace_bytes(dv.pool.handle, cases[0].T, cases[0].K))
+                 for dv in base)
+    ws = torch.empty(max(256, nbytes), dtype=torch.uint8, device="cuda")
+    plan = mb.Plan(cases[0].T, cases[0].K, table.num_slots, cases[0].E)
+    w = base[0].pair_weight
+
+    def one_pass():
+        for row in sets:
+            mb.mint_lora_plan(table, ids, status, expert_ids=ex, num_experts=cases[0].E, plan=plan)
+            for (pool, x, dy, dx, dA, dB, x_row) in row:
+                mb.mint_moe_lora_backward(pool, table, plan, x, dy, status, dx=dx, dA=dA, dB=dB, x_row=x_row,
+                                          pair_weight=w, workspace=ws)
+
+    one_pass()
+    torch.cuda.synchronize()
+    # parity of the first set's gate projection (all outputs started at zero) against the fp64 oracle
+    c, (_, _, _, dx, dA, dB, _) = cases[0], sets[0][0]
+    t = c.table
+    dx_ref, dA_ref, dB_ref, _ = oracle_backward.moe_lora_backward(c.ids, c.expert_ids, t.id_to_slot, t.slot_rank,
+                                                                  t.slot_scale, c.A, c.B, c.x, dys[0], x_row=c.x_row,
+                                                                  pair_weight=c.pair_weight)
+    dxg = harness.y_to_f64(dx)
+    par = {"max_abs_dx": float(np.abs(dxg - dx_ref).max()),
+           "rel_fro_dx": float(np.linalg.norm(dxg - dx_ref) / np.linalg.norm(dx_ref)),
+           "rel_fro_dA": float(np.linalg.norm(dA.cpu().numpy() - dA_ref) / np.linalg.norm(dA_ref)),
+           "rel_fro_dB": float(np.linalg.norm(dB.cpu().numpy() - dB_ref) / np.linalg.norm(dB_ref))}
+    par["within_tolerance"] = bool(par["max_abs_dx"] <= 3e-2 and par["rel_fro_dx"] <= 5e-3 and
+                                   par["rel_fro_dA"] <= 1e-4 and par["rel_fro_dB"] <= 1e-4)
+    del dx_ref, dA_ref, dB_ref, dxg
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(g, stream=stream):
+            one_pass()
+    est = time_graph(torch, dist, world, stream, g, 2, 2) / 2
+    steps = 2 if short else int(min(100, max(5, 150.0 / max(est, 1e-3))))
+    ms = time_graph(torch, dist, world, stream, g, steps, 3, name="moe_backward") / steps
+    st = status.cpu().numpy()
+    if st[0] != 0:
+        raise SystemExit(f"device status {mb.status_name(int(st[0]))} after the MoE backward loop")
+    layer_bytes = sum(accounting.algorithmic_bytes_moe_backward(c)["total"] for c in cases)
+    res = {"workload": "config4 layer: per-pair dx, dA, dB of gate, up and down (one call per projection, a plan per layer)",
+           "layers": len(sets), "us_per_layer": ms * 1e3 / len(sets), "bytes_per_layer": layer_bytes,
+           "GBps": layer_bytes / (ms * 1e-3 / len(sets)) / 1e9,
+           "roofline_frac": layer_bytes / (ms * 1e-3 / len(sets)) / 1e9 / peak,
+           "tokens_per_s": world * cases[0].T * len(sets) / (ms * 1e-3), "parity": par}
+    del g, sets, base, ws
+    gc.collect()
+    torch.cuda.empty_cache()
+    return res
+
+
 def measure_admission(torch, stream):
     """Admitting one adapter into the three expert projections of a 30B-A3B-shaped layer (128 experts):
     the packed representation (one call per projection) against one copy per tensor."""
@@ -551,9 +625,12 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     mb.load_library()
     peak, peak_src = hbm_peak()
-    if args.workload == "backward":   # the backward alone (the command profilers wrap): its own JSON line
-        res = measure_backward(torch, dist, 1, torch.cuda.Stream(), peak, layers=args.layers or 6,
-                               short=args.profile)
+    if args.workload in ("backward", "moe_backward"):   # a backward alone (the command profilers wrap): its own JSON line
+        if args.workload == "backward":
+            res = measure_backward(torch, dist, 1, torch.cuda.Stream(), peak, layers=args.layers or 6,
+                                   short=args.profile)
+        else:
+            res = measure_moe_backward(torch, dist, 1, torch.cuda.Stream(), peak, short=args.profile)
         if rank == 0:
             print(json.dumps(res))
         return
@@ -761,6 +838,8 @@ def run_gpu(args):
     admission = None if args.no_side_workloads else measure_admission(torch, stream)
     backward = (measure_backward(torch, dist, 1, stream, peak)
                 if (args.workload == "config2" and not args.no_side_workloads and rank == 0) else None)
+    moe_backward = (measure_moe_backward(torch, dist, 1, stream, peak)
+                    if (args.workload == "config2" and not args.no_side_workloads and rank == 0) else None)
     cpu_val, cores, sample = oracle_layer_seconds(wl)
 
     line = {
@@ -783,6 +862,7 @@ def run_gpu(args):
         "workloads": workloads,
         "admission": admission,
         "backward": backward,
+        "moe_backward": moe_backward,
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "layers_per_step": e2e_layers},

@@ -77,3 +77,20 @@ def algorithmic_bytes_moe(case: MoECase) -> dict:
     b["total"] = b["x"] + b["ab"] + b["y"] + b["ids"]
     b["flops"] = 2 * int(case.table.slot_rank[pair_slot[active]].sum()) * (case.d + case.n)
     return b
+
+
+def algorithmic_bytes_moe_backward(case: MoECase) -> dict:
+    """Backward of the MoE apply: x once per distinct row read, dy once per active pair, each touched
+    (slot, expert) A and B once, dx (one bf16 row per active pair) read + write, dA and dB of the touched
+    blocks read + write (fp32, true ranks), plus ids."""
+    f = algorithmic_bytes_moe(case)
+    b = {
+        "x": f["x"],
+        "dy": 2 * f["p_active"] * case.n,
+        "ab": f["ab"],
+        "dx": 4 * f["p_active"] * case.d,
+        "grads": 4 * f["ab"],            # fp32 read + write against bf16 read: 8 bytes per element against 2
+        "ids": f["ids"],
+    }
+    b["total"] = sum(b.values())
+    return b

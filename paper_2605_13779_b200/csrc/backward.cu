@@ -158,13 +158,20 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
         }
       }
       if (col_ok && p.packed) {
+        // [width][r_max]: the chunk's ranks of a column are eight consecutive floats (r_max is a multiple of
+        // 8); ranks at or above the slot's rank are written back as they were read
 #pragma unroll
         for (int e = 0; e < kColsPerThread; ++e)
 #pragma unroll
-          for (int k = 0; k < kRankChunk; ++k)
-            if (k < kc) {
-              float *dst = out_slot + (size_t)(col + e) * p.r_max + k0 + k;
-              *dst = fmaf(scale, acc[k][e], *dst);
+          for (int h = 0; h < kRankChunk / 4; ++h)
+            if (4 * h < kc) {
+              float4 *dst = reinterpret_cast<float4 *>(out_slot + (size_t)(col + e) * p.r_max + k0 + 4 * h);
+              float4 o = *dst;
+              if (4 * h + 0 < kc) o.x = fmaf(scale, acc[4 * h + 0][e], o.x);
+              if (4 * h + 1 < kc) o.y = fmaf(scale, acc[4 * h + 1][e], o.y);
+              if (4 * h + 2 < kc) o.z = fmaf(scale, acc[4 * h + 2][e], o.z);
+              if (4 * h + 3 < kc) o.w = fmaf(scale, acc[4 * h + 3][e], o.w);
+              *dst = o;
             }
       } else if (col_ok) {
 #pragma unroll
