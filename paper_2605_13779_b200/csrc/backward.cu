@@ -67,6 +67,9 @@ struct GradParams {
   PlanView pv;
 };
 
+// kGeneral: (slot, expert) blocks, a row map for the activations and the packed layout (MoE pools); the
+// dense instantiation carries none of that.
+template <bool kGeneral>
 __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_constant__ GradParams P) {
   __shared__ int32_t tok[kTokenBatch];    // staged items (tokens, or (token, k) pairs)
   __shared__ int32_t arow[kTokenBatch];   // the row of act each of them reads
@@ -96,7 +99,7 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
     if (tid == 0) report(P.status, MINT_ERR_RANK_TOO_LARGE, slot);
     return;
   }
-  const int block = P.E > 0 ? slot * P.E + P.pv.seg_expert[seg] : slot;
+  const int block = (kGeneral && P.E > 0) ? slot * P.E + P.pv.seg_expert[seg] : slot;
   float *out_slot = p.out + (size_t)block * p.r_max * p.width;
   const bool one_batch = len <= kTokenBatch;   // the usual case of a decode batch: staged once per rank chunk
   // stages the token indices and the coefficients of tokens [b0, b0 + nb) for ranks k0 .. k0 + kc - 1
@@ -105,20 +108,20 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
     if (tid < nb) {
       const int item = P.pv.perm[off + b0 + tid];
       tok[tid] = item;
-      const int r_ = p.row_map ? p.row_map[item] : item;
-      arow[tid] = (r_ >= 0 && r_ < p.act_rows) ? r_ : -1;   // (reported by the shrink that made the coefficients)
+      const int r_ = (kGeneral && p.row_map) ? p.row_map[item] : item;
+      arow[tid] = (!kGeneral || (r_ >= 0 && r_ < p.act_rows)) ? r_ : ~0;   // (~0: out of range, reported by the shrink; it counts as zero)
     }
     __syncthreads();
     for (int i = tid; i < nb * kRankChunk; i += kThreads) {
       const int j = i / kRankChunk, k = i - j * kRankChunk;
-      cf[j][k] = k < kc ? p.coef[(size_t)tok[j] * p.r_max + k0 + k] : 0.f;
+      cf[j][k] = (k < kc && (!kGeneral || arow[j] >= 0)) ? p.coef[(size_t)tok[j] * p.r_max + k0 + k] : 0.f;
     }
     __syncthreads();
   };
   {
     // the gradient rows this CTA will add to, on their way into L2 while the tokens are walked
     const int col = ((int)blockIdx.y - p.block0) * kBlocksPerCta * kColsPerCta + tid * kColsPerThread;
-    if (p.packed) {   // [width][r_max]: this thread's four columns are 4 r_max consecutive floats
+    if (kGeneral && p.packed) {   // [width][r_max]: this thread's four columns are 4 r_max consecutive floats
       if (col < p.width)
         for (int i = 0; i < 4 * p.r_max; i += 32)
           asm volatile("prefetch.global.L2 [%0];" ::"l"(out_slot + (size_t)col * p.r_max + i));
@@ -145,8 +148,7 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
         if (col_ok) {
 #pragma unroll 4
           for (int j = 0; j < nb; ++j) {
-            if (arow[j] < 0) continue;
-            const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p.act + (int64_t)arow[j] * p.ld + col));
+            const uint2 q = __ldg(reinterpret_cast<const uint2 *>(p.act + (int64_t)(kGeneral ? max(arow[j], 0) : tok[j]) * p.ld + col));
             const float a[4] = {bf16lo(q.x), bf16hi(q.x), bf16lo(q.y), bf16hi(q.y)};
 #pragma unroll
             for (int k = 0; k < kRankChunk; ++k) {
@@ -157,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) grad_weight_kernel(const __grid_cons
           }
         }
       }
-      if (col_ok && p.packed) {
+      if (kGeneral && col_ok && p.packed) {
         // [width][r_max]: the chunk's ranks of a column are eight consecutive floats (r_max is a multiple of
         // 8); ranks at or above the slot's rank are written back as they were read
 #pragma unroll
@@ -307,7 +309,11 @@ int32_t mint_launch_grad_weights(const GradJobHost *jobs, int njobs, int32_t T, 
   cfg.attrs = attr;
   // right after a plan or a bind kernel it waits for that kernel in full: it reads the plan at once
   cfg.numAttrs = mint_take_tables_changed() ? 0 : 1;
-  return mint_check_cuda(cudaLaunchKernelEx(&cfg, grad_weight_kernel, P), "grad_weight launch");
+  bool general = E > 0;
+  for (int i = 0; i < njobs; ++i) general = general || jobs[i].row_map != nullptr || jobs[i].packed;
+  return mint_check_cuda(general ? cudaLaunchKernelEx(&cfg, grad_weight_kernel<true>, P)
+                                 : cudaLaunchKernelEx(&cfg, grad_weight_kernel<false>, P),
+                         "grad_weight launch");
 }
 
 
