@@ -500,13 +500,13 @@ def measure_moe_backward(torch, dist, world, stream, peak, short=False):
     from oracle import backward as oracle_backward
     from paper_2605_13779_b200 import accounting, binding as mb, harness, synth
     wl = build_workload("config4", 0)
-    cases = wl["cases"]
+    cases = wl["cases"][:1] if short else wl["cases"]   # (short: the gate projection alone, under a profiler)
     P = cases[0].T * cases[0].K
     base = [harness.upload_moe(c) for c in cases]
     table, ids, ex, status = base[0].table, base[0].ids, base[0].expert_ids, mb.new_status()
     dys = [synth.normal_bf16(synth.stream("bench/moe-backward", c.name), (P, c.n), 1.0) for c in cases]
     sets = []
-    for si in range(2):
+    for si in range(1 if short else 2):
         row = []
         for dv, c, dy in zip(base, cases, dys):
             pool = dv.pool if si == 0 else mb.Pool(dv.pool.A.clone(), dv.pool.B.clone(), c.d, c.n, c.r_max,
